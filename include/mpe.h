@@ -1,0 +1,160 @@
+/*
+ * mpe -- mixed-precision embedding tables behind an FP32 cache: the training
+ * step of "Mixed-Precision Embedding using a Cache" on one B200 (sm_100a).
+ *
+ * Every table stores its rows row-wise quantized (INT8 or packed INT4 codes plus
+ * an FP32 scale and bias per row; Section 3 "Precision", Appendix Eq. 3) and is
+ * fronted by a set-associative cache of FP32 rows (Section 3 "Cache Structure")
+ * managed by LRU or LFU priorities (Section 3 "Cache Replacement Policy",
+ * Algorithm 2).  One training step = mpe_forward (fetch + sum-pool) followed by
+ * mpe_backward (merge duplicate gradients, optimizer update in FP32, commit to
+ * cache or stochastic-round back to the table, admission/eviction).
+ *
+ * C ABI, no exceptions.  Every function returns 0 (MPE_OK) or a negative
+ * MPE_ERR_* code.  Pointers named d_* are device pointers on the handle's
+ * device, h_* are host pointers.  The handle owns all table state and all
+ * workspace; the caller owns every buffer it passes in, and device buffers need
+ * to stay alive only until the stream work enqueued by that call has finished.
+ * Calls on one handle must not overlap in time (no internal locking).
+ */
+#ifndef MPE_H
+#define MPE_H
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mpe_handle mpe_handle;
+typedef struct { int64_t num_rows; int32_t dim; } mpe_table_spec;
+
+enum { MPE_LRU = 0, MPE_LFU = 1 };
+enum { MPE_SGD = 0, MPE_ROWWISE_ADAGRAD = 1 };
+
+enum {
+    MPE_OK = 0,
+    MPE_ERR_ARG = -1,          /* NULL pointer, negative size, value out of range */
+    MPE_ERR_UNSUPPORTED = -2,  /* unequal dims, dim not a power of two in [4,128], bits not 8/4, ways not 2^k <= 32 */
+    MPE_ERR_CUDA = -3,         /* a CUDA runtime call failed (detail = cudaError_t) */
+    MPE_ERR_SEQUENCE = -4,     /* backward without a preceding forward, or step not strictly increasing */
+    MPE_ERR_INDEX = -5,        /* device saw row ids outside [0, num_rows) (detail = how many); they were dropped */
+    MPE_ERR_OFFSETS = -6,      /* device saw offsets that are not 0 = o[0] <= o[1] <= ... <= o[T*B] = total */
+    MPE_ERR_NOMEM = -7         /* allocation failed */
+};
+
+/*
+ * Create the tables, the caches and the policy state on `device`.
+ *   tables[num_tables]  row count and dimension of each table; all dims must be equal
+ *                       (a power of two in [4,128]); num_rows in [1, 2^31-2].
+ *   bits                8 or 4: width of the integer codes (Section 3 "Precision").
+ *   cache_fraction      in [0,1]; table t gets n_t = max(1, floor(cache_fraction*N_t + 1e-6) / ways) sets
+ *                       of `ways` FP32 rows (Section 3 "Cache Structure"); 0 = no cache at all.
+ *   ways                associativity alpha, a power of two <= 32; 0 selects 32 (Section 5.1).
+ *   policy              MPE_LRU (timestamp of last access = step number, per cached row) or
+ *                       MPE_LFU (access count per embedding row)  (Section 3 "Cache Replacement Policy").
+ *   optimizer           MPE_SGD (x <- x - lr*g, Section 3) or MPE_ROWWISE_ADAGRAD
+ *                       (G_row += mean(g^2); x <- x - lr/(sqrt(G_row)+eps)*g; Section 4.1 names a
+ *                       sparse AdaGrad without a formula, this is the build's reading).
+ *   init_lo, init_hi    rows start Uniform(init_lo, init_hi) drawn from a counter hash of
+ *                       (seed, table, row, column) and are quantized with round-to-nearest-even;
+ *                       the cache starts empty.
+ * On success *out receives the handle.  Allocates device memory (cudaMalloc).
+ */
+int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_tables, int32_t bits,
+               double cache_fraction, int32_t ways, int32_t policy, int32_t optimizer, float eps,
+               float init_lo, float init_hi, uint64_t seed, int32_t device);
+
+/* Size the per-step workspace for batches of up to max_batch samples and max_total_indices
+ * indices, so that later steps allocate nothing.  mpe_forward grows the workspace by itself
+ * (a synchronising reallocation) when a larger batch arrives. */
+int mpe_reserve(mpe_handle* h, int32_t max_batch, int64_t max_total_indices);
+
+/*
+ * Forward: x <- fetch(T, C, i) for every index, summed per bag (Section 3; multi-hot bags, Section 5.1).
+ *   d_indices[total_indices]  table-local row ids, int32, table-major: bag (t,b) is
+ *                             d_indices[d_offsets[t*batch+b] .. d_offsets[t*batch+b+1]).
+ *   d_offsets[T*batch+1]      non-decreasing, first 0, last total_indices.
+ *   d_out[batch][T*dim]       FP32, row-major; bag (t,b) lands in d_out[b][t*dim .. (t+1)*dim);
+ *                             an empty bag gives zeros; rows are added in index order starting from +0.
+ * The call sorts and de-duplicates the indices (Section 5.1), probes the cache tags, gathers FP32
+ * rows on hits and dequantizes (q*scale+bias, Algorithm 1) on misses.  It reads but never changes
+ * table, cache or policy state.  Work is enqueued on `cuda_stream` (a cudaStream_t; NULL = the
+ * default stream) and the call returns without waiting.  Row ids outside [0, num_rows) contribute
+ * nothing and raise the sticky MPE_ERR_INDEX.
+ */
+int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch,
+                int64_t total_indices, float* d_out, void* cuda_stream);
+
+/*
+ * Backward of the preceding mpe_forward, on the same stream: update(T, C, i, x) for every distinct
+ * row of the batch (Section 3, Algorithm 2).
+ *   d_grad_out[batch][T*dim]  gradient of the loss w.r.t. d_out, FP32.
+ *   lr                        learning rate.
+ *   step                      1 <= step < 2^32, strictly increasing over the handle's life; it is the LRU
+ *                             timestamp and part of the stochastic-rounding counter.
+ * Gradients of duplicate rows are merged first (Section 5.1) in a fixed radix-32 tree over index
+ * positions; priorities are updated; each row is updated once in FP32 from the value the forward
+ * fetched; rows that are (or become) cache resident are written to the cache verbatim, all others
+ * are re-quantized with stochastic rounding (Section 3 "Rounding"); an evicted row is down-converted
+ * the same way.  Must follow exactly one mpe_forward (else MPE_ERR_SEQUENCE).  Returns without waiting.
+ */
+int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step);
+
+/* One whole step from HOST buffers: copies indices, offsets and grad_out to the device, runs
+ * forward and backward, copies the pooled output back and waits for it.  Layouts as above.
+ * Uses the stream of the last mpe_forward (default stream if none). */
+int mpe_step_host(mpe_handle* h, const int32_t* h_indices, const int32_t* h_offsets, int32_t batch,
+                  int64_t total_indices, const float* h_grad_out, float* h_out, float lr, int64_t step);
+
+/* Write every cache-resident row back into the low-precision table with stochastic rounding; rows
+ * stay resident and unchanged.  Afterwards the table alone is a complete snapshot of the model.
+ * (The paper has no flush; it is the snapshot operation a trainer needs.) */
+int mpe_flush(mpe_handle* h);
+
+/* Waits for the handle's stream, then frees everything. */
+int mpe_destroy(mpe_handle* h);
+
+/* ---- observation (all of these wait for the handle's stream) --------------------------------- */
+/* Sticky device-detected condition since the last call of this function: *code is MPE_OK,
+ * MPE_ERR_INDEX or MPE_ERR_OFFSETS; *detail counts the offending items.  Clears the condition. */
+int mpe_last_error(mpe_handle* h, int32_t* code, int64_t* detail);
+/* Counters of table `table` accumulated by mpe_backward: out8 = {lookups, hits (per index),
+ * unique rows, unique hits, admissions, evictions, bypasses, steps}. */
+int mpe_stats(mpe_handle* h, int32_t table, uint64_t* out8);
+/* Bytes of each component of the appendix's memory accounting (Appendix Eq. 2-3), summed over
+ * tables: out6 = {low-precision table incl. scale/bias, FP32 cache, tags, LFU counters or LRU
+ * timestamps, optimizer state, the FP32 table this replaces}. */
+int mpe_memory_bytes(mpe_handle* h, uint64_t* out6);
+/* Geometry of table `table`'s cache. */
+int mpe_cache_geometry(mpe_handle* h, int32_t table, int32_t* n_sets, int32_t* ways);
+/* Figures of the last mpe_forward: out4 = {valid indices, distinct rows, dropped indices, rows whose
+ * multiplicity needs the multi-block gradient tree}. */
+int mpe_step_info(mpe_handle* h, int64_t* out4);
+/* Low-precision entries of n rows: h_codes[n][dim*bits/8] (INT4: column 2k in the low nibble of
+ * byte k), h_scale[n], h_bias[n].  The entry of a cache-resident row is stale until it is evicted
+ * or flushed. */
+int mpe_export_rows(mpe_handle* h, int32_t table, const int64_t* h_rows, int64_t n, uint8_t* h_codes,
+                    float* h_scale, float* h_bias);
+/* Whole cache of one table: h_tags[n_sets*ways] (-1 = empty), h_rows[n_sets*ways][dim],
+ * h_ts[n_sets*ways] (LRU timestamps; pass NULL to skip, zeros under LFU). */
+int mpe_export_cache(mpe_handle* h, int32_t table, int32_t* h_tags, float* h_rows, uint32_t* h_ts);
+/* Per-row auxiliary state of n rows: LFU counters and/or Adagrad accumulators (NULL to skip). */
+int mpe_export_aux(mpe_handle* h, int32_t table, const int64_t* h_rows, int64_t n, uint32_t* h_cnt,
+                   float* h_adagrad);
+
+/* ---- instrumentation ---------------------------------------------------------------------------- */
+/* Number of kernels this handle has launched so far. */
+int mpe_kernel_launches(mpe_handle* h, uint64_t* count);
+/* With profiling on, every kernel launch is bracketed by CUDA events on the launching stream. */
+int mpe_profile(mpe_handle* h, int32_t enable);
+/* Waits for the stream, then reports per kernel name the launches and the summed event time since
+ * profiling was switched on (or last read): up to `cap` entries, names are 32-byte C strings.
+ * *n receives the number of distinct kernels. */
+int mpe_profile_read(mpe_handle* h, int32_t cap, char* names /*[cap][32]*/, double* ms, uint64_t* launches,
+                     int32_t* n);
+const char* mpe_error_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,598 @@
+// Host side of the C ABI declared in include/mpe.h: state, workspace, and the
+// kernel sequence of one training step.  Nothing here computes on the host;
+// every step of the path runs in the kernels of mpe_kernels.cuh.
+#include "../../include/mpe.h"
+#include "mpe_kernels.cuh"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <vector>
+
+using namespace mpe;
+
+namespace {
+
+struct ProfRec { int name; cudaEvent_t a, b; };
+
+}  // namespace
+
+struct mpe_handle {
+    int device = 0, num_sms = 148;
+    int T = 0, dim = 0, bits = 0, ways = 0, policy = 0, optimizer = 0, code_bytes = 0;
+    float eps = 0, lo = 0, hi = 0;
+    uint64_t seed = 0;
+    std::vector<TableDev> tables;
+    int64_t total_rows = 0, total_sets = 0, total_slots = 0;
+    int32_t max_rows = 0, max_sets = 0;
+    State st{};
+    Work wk{};
+    TableDev* d_tables = nullptr;
+    // workspace
+    int64_t cap_L = 0, cap_bags = 0;
+    uint32_t *keyA = nullptr, *keyB = nullptr, *valA = nullptr, *valB = nullptr;
+    uint32_t *ckeyA = nullptr, *ckeyB = nullptr, *cvalA = nullptr, *cvalB = nullptr;
+    uint32_t *hist = nullptr, *block_sums = nullptr;
+    std::vector<void*> ws_allocs;
+    // staging for mpe_step_host
+    int32_t *sh_idx = nullptr, *sh_off = nullptr; float *sh_grad = nullptr, *sh_out = nullptr;
+    int64_t sh_cap_L = 0, sh_cap_off = 0, sh_cap_out = 0;
+    // step state
+    cudaStream_t stream = nullptr;
+    bool have_forward = false;
+    int64_t last_step = 0;
+    uint64_t steps = 0;
+    uint32_t epoch = 0;
+    int32_t B = 0; int64_t L = 0;
+    const uint32_t *skey = nullptr, *spos = nullptr;
+    // instrumentation
+    uint64_t launches = 0;
+    bool profiling = false;
+    std::vector<std::string> prof_names;
+    std::vector<ProfRec> prof_recs;
+    std::vector<cudaEvent_t> event_pool;
+    int last_cuda_error = 0;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = 0;
+    explicit DeviceGuard(int dev) { cudaGetDevice(&prev); if (prev != dev) cudaSetDevice(dev); else prev = -1; }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+#define CK(h, expr) do { cudaError_t e_ = (expr); if (e_ != cudaSuccess) { (h)->last_cuda_error = (int)e_; return e_ == cudaErrorMemoryAllocation ? MPE_ERR_NOMEM : MPE_ERR_CUDA; } } while (0)
+
+cudaEvent_t get_event(mpe_handle* h) {
+    if (!h->event_pool.empty()) { cudaEvent_t e = h->event_pool.back(); h->event_pool.pop_back(); return e; }
+    cudaEvent_t e; cudaEventCreate(&e); return e;
+}
+
+int prof_name(mpe_handle* h, const char* name) {
+    for (size_t i = 0; i < h->prof_names.size(); ++i) if (h->prof_names[i] == name) return (int)i;
+    h->prof_names.push_back(name);
+    return (int)h->prof_names.size() - 1;
+}
+
+struct LaunchScope {
+    mpe_handle* h; ProfRec rec{};
+    LaunchScope(mpe_handle* h_, const char* name) : h(h_) {
+        ++h->launches;
+        if (h->profiling) { rec.name = prof_name(h, name); rec.a = get_event(h); rec.b = get_event(h); cudaEventRecord(rec.a, h->stream); }
+    }
+    ~LaunchScope() { if (h->profiling) { cudaEventRecord(rec.b, h->stream); h->prof_recs.push_back(rec); } }
+};
+
+#define LAUNCH(h, name, kern, grid, block, smem, ...) \
+    do { LaunchScope ls_(h, name); kern<<<(grid), (block), (smem), (h)->stream>>>(__VA_ARGS__); } while (0)
+
+int grid_for(const mpe_handle* h, int64_t work_items, int64_t items_per_block, int blocks_per_sm) {
+    int64_t need = (work_items + items_per_block - 1) / items_per_block;
+    int64_t cap = (int64_t)h->num_sms * blocks_per_sm;
+    return (int)std::max<int64_t>(1, std::min(need, cap));
+}
+
+int bits_for(uint32_t v) { int b = 1; while (b < 32 && (v >> b) != 0) ++b; return b; }
+
+template <class T>
+int dmalloc(mpe_handle* h, T** p, int64_t n, std::vector<void*>* track) {
+    *p = nullptr;
+    cudaError_t e = cudaMalloc((void**)p, (size_t)std::max<int64_t>(n, 1) * sizeof(T));
+    if (e != cudaSuccess) { h->last_cuda_error = (int)e; return MPE_ERR_NOMEM; }
+    if (track) track->push_back(*p);
+    return MPE_OK;
+}
+
+void free_workspace(mpe_handle* h) {
+    for (void* p : h->ws_allocs) cudaFree(p);
+    h->ws_allocs.clear();
+    h->cap_L = 0; h->cap_bags = 0;
+}
+
+int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
+    // everything a step needs between its first and last kernel, sized for L indices
+    free_workspace(h);
+    auto* tr = &h->ws_allocs;
+    const int T = h->T;
+    const int64_t n = L + 1;
+    Work& w = h->wk;
+    int rc = MPE_OK;
+#define A(ptr, count) if ((rc = dmalloc(h, &(ptr), (count), tr)) != MPE_OK) return rc
+    A(h->keyA, n); A(h->keyB, n); A(h->valA, n); A(h->valB, n);
+    A(h->ckeyA, n); A(h->ckeyB, n); A(h->cvalA, n); A(h->cvalB, n);
+    const int64_t max_tiles = (L + SORT_TILE - 1) / SORT_TILE + T + 1;
+    A(h->hist, 256 * max_tiles);
+    A(h->block_sums, std::max<int64_t>(256 * max_tiles, n) / SCAN_TILE + 2);
+    A(w.ctr, 1);
+    A(w.table_start, T + 1); A(w.tile_base, T + 1); A(w.ustart, T + 1); A(w.ctile_base, T + 1);
+    A(w.bag_of, n); A(w.kidx, n); A(w.occ_loc, n); A(w.occ_b, n);
+    A(w.uniq_row, n); A(w.uniq_t, n); A(w.seg, n + 1); A(w.loc, n); A(w.final_loc, n); A(w.victim, n);
+    A(w.hot_base, n); A(w.uset, n);
+    const int64_t max_tasks = L / (HOT_SPAN / 2) + 2;
+    A(w.task_k, max_tasks); A(w.partial, max_tasks * h->dim);
+#undef A
+    CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), h->stream));
+    h->cap_L = L; h->cap_bags = bags;
+    return MPE_OK;
+}
+
+// device-wide exclusive prefix sum of data[0 .. *n_ptr) in place
+void scan_u32(mpe_handle* h, uint32_t* data, const uint32_t* n_ptr, int64_t n_upper) {
+    const int g = grid_for(h, n_upper, SCAN_TILE, 8);
+    LAUNCH(h, "scan_reduce", k_scan_reduce, g, SCAN_THREADS, 0, data, n_ptr, h->block_sums);
+    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, 1024, 0, h->block_sums, n_ptr, (uint32_t)SCAN_TILE, (uint32_t*)nullptr);
+    LAUNCH(h, "scan_apply", k_scan_apply, g, SCAN_THREADS, 0, data, n_ptr, (const uint32_t*)h->block_sums);
+}
+
+// stable sort of every segment [seg_start[t], seg_start[t+1]) by the low `key_bits` bits of the key;
+// returns which buffer pair holds the result (0 = A, 1 = B)
+int seg_sort(mpe_handle* h, uint32_t* kA, uint32_t* kB, uint32_t* vA, uint32_t* vB, const int32_t* seg_start,
+             int32_t* tile_base, uint32_t* hist_len, int key_bits, int64_t n_upper) {
+    const int T = h->T;
+    LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, seg_start, T, tile_base, hist_len, (const uint32_t*)&h->wk.ctr->abort);
+    const int64_t max_tiles = (n_upper + SORT_TILE - 1) / SORT_TILE + T;
+    const int g = grid_for(h, max_tiles, 1, 4);
+    const int passes = (key_bits + 7) / 8;
+    uint32_t *kin = kA, *kout = kB, *vin = nullptr, *vout = vB;
+    for (int p = 0; p < passes; ++p) {
+        LAUNCH(h, "sort_hist", k_sort_hist, g, SORT_THREADS, 0, (const uint32_t*)kin, seg_start, (const int32_t*)tile_base, T, 8 * p, h->hist);
+        scan_u32(h, h->hist, hist_len, 256 * max_tiles);
+        LAUNCH(h, "sort_scatter", k_sort_scatter, g, SORT_THREADS, 0, (const uint32_t*)kin, (const uint32_t*)vin, kout, vout,
+               seg_start, (const int32_t*)tile_base, T, 8 * p, (const uint32_t*)h->hist);
+        std::swap(kin, kout);
+        vin = vout; vout = (vout == vB) ? vA : vB;
+    }
+    return (passes & 1) ? 1 : 0;
+}
+
+int check_launch(mpe_handle* h) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { h->last_cuda_error = (int)e; return MPE_ERR_CUDA; }
+    return MPE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* mpe_error_string(int code) {
+    switch (code) {
+        case MPE_OK: return "ok";
+        case MPE_ERR_ARG: return "bad argument";
+        case MPE_ERR_UNSUPPORTED: return "unsupported configuration";
+        case MPE_ERR_CUDA: return "CUDA runtime error";
+        case MPE_ERR_SEQUENCE: return "call out of sequence";
+        case MPE_ERR_INDEX: return "row index out of range";
+        case MPE_ERR_OFFSETS: return "inconsistent offsets";
+        case MPE_ERR_NOMEM: return "out of memory";
+        default: return "unknown error";
+    }
+}
+
+int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_tables, int32_t bits,
+               double cache_fraction, int32_t ways, int32_t policy, int32_t optimizer, float eps,
+               float init_lo, float init_hi, uint64_t seed, int32_t device) {
+    if (!out || !tables || num_tables < 1) return MPE_ERR_ARG;
+    *out = nullptr;
+    if (!(cache_fraction >= 0.0 && cache_fraction <= 1.0)) return MPE_ERR_ARG;
+    if (policy != MPE_LRU && policy != MPE_LFU) return MPE_ERR_ARG;
+    if (optimizer != MPE_SGD && optimizer != MPE_ROWWISE_ADAGRAD) return MPE_ERR_ARG;
+    if (bits != 8 && bits != 4) return MPE_ERR_UNSUPPORTED;
+    if (ways == 0) ways = 32;
+    if (ways < 1 || ways > 32 || (ways & (ways - 1))) return MPE_ERR_UNSUPPORTED;
+    const int dim = tables[0].dim;
+    if (dim < 4 || dim > 128 || (dim & (dim - 1))) return MPE_ERR_UNSUPPORTED;
+    for (int t = 0; t < num_tables; ++t) {
+        if (tables[t].dim != dim) return MPE_ERR_UNSUPPORTED;
+        if (tables[t].num_rows < 1 || tables[t].num_rows > 0x7ffffffeLL) return MPE_ERR_ARG;
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return MPE_ERR_CUDA;
+
+    mpe_handle* h = new mpe_handle();
+    h->device = device;
+    DeviceGuard guard(device);
+    cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, device);
+    h->T = num_tables; h->dim = dim; h->bits = bits; h->ways = ways; h->policy = policy; h->optimizer = optimizer;
+    h->code_bytes = dim * bits / 8; h->eps = eps; h->lo = init_lo; h->hi = init_hi; h->seed = seed;
+    h->tables.resize(num_tables);
+    for (int t = 0; t < num_tables; ++t) {
+        TableDev& tb = h->tables[t];
+        tb.row_base = h->total_rows; tb.set_base = h->total_sets;
+        tb.N = (int32_t)tables[t].num_rows;
+        int64_t n = 0;
+        if (cache_fraction > 0.0) {
+            const int64_t cache_rows = (int64_t)std::floor(cache_fraction * (double)tables[t].num_rows + 1e-6);
+            n = std::max<int64_t>(1, cache_rows / ways);
+        }
+        tb.n_sets = (int32_t)n;
+        tb.salt = table_salt(seed, (uint32_t)t);
+        tb.pad = 0;
+        h->total_rows += tb.N; h->total_sets += n;
+        h->max_rows = std::max(h->max_rows, tb.N); h->max_sets = std::max(h->max_sets, tb.n_sets);
+    }
+    h->total_slots = h->total_sets * ways;
+    if (h->total_slots > 0x7fffffffLL) { delete h; return MPE_ERR_UNSUPPORTED; }
+
+    State& s = h->st;
+    s.T = num_tables; s.dim = dim; s.lanes = dim / 4; s.ways = ways; s.policy = policy; s.optimizer = optimizer;
+    s.bits = bits; s.seed = seed; s.eps = eps;
+    int rc = MPE_OK;
+    auto fail = [&](int code) { mpe_destroy(h); return code; };
+    if ((rc = dmalloc(h, &h->d_tables, num_tables, nullptr)) != MPE_OK) return fail(rc);
+    s.tables = h->d_tables;
+    if ((rc = dmalloc(h, &s.codes, h->total_rows * h->code_bytes, nullptr)) != MPE_OK) return fail(rc);
+    if ((rc = dmalloc(h, &s.sb, h->total_rows, nullptr)) != MPE_OK) return fail(rc);
+    if (policy == MPE_LFU && (rc = dmalloc(h, &s.cnt, h->total_rows, nullptr)) != MPE_OK) return fail(rc);
+    if (optimizer == MPE_ROWWISE_ADAGRAD && (rc = dmalloc(h, &s.G, h->total_rows, nullptr)) != MPE_OK) return fail(rc);
+    if ((rc = dmalloc(h, &s.slab, h->total_slots * dim, nullptr)) != MPE_OK) return fail(rc);
+    if ((rc = dmalloc(h, &s.tags, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
+    if (policy == MPE_LRU && (rc = dmalloc(h, &s.ts, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
+    if ((rc = dmalloc(h, &s.hit_epoch, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
+    if ((rc = dmalloc(h, &s.hit_k, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
+    if ((rc = dmalloc(h, &s.stats, (int64_t)num_tables * 8, nullptr)) != MPE_OK) return fail(rc);
+#define CKC(expr) do { cudaError_t e_ = (expr); if (e_ != cudaSuccess) { h->last_cuda_error = (int)e_; return fail(MPE_ERR_CUDA); } } while (0)
+    CKC(cudaMemcpy(h->d_tables, h->tables.data(), sizeof(TableDev) * num_tables, cudaMemcpyHostToDevice));
+    if (s.cnt) CKC(cudaMemset(s.cnt, 0, sizeof(uint32_t) * h->total_rows));
+    if (s.G) CKC(cudaMemset(s.G, 0, sizeof(float) * h->total_rows));
+    CKC(cudaMemset(s.slab, 0, sizeof(float) * std::max<int64_t>(1, h->total_slots * dim)));
+    if (s.ts) CKC(cudaMemset(s.ts, 0, sizeof(uint32_t) * std::max<int64_t>(1, h->total_slots)));
+    CKC(cudaMemset(s.hit_epoch, 0, sizeof(uint32_t) * std::max<int64_t>(1, h->total_slots)));
+    CKC(cudaMemset(s.stats, 0, sizeof(unsigned long long) * 8 * num_tables));
+    LAUNCH(h, "fill_tags", k_fill_i32, grid_for(h, h->total_slots, 256, 8), 256, 0, s.tags, h->total_slots, -1);
+    for (int t = 0; t < num_tables; ++t) {
+        const int g = grid_for(h, h->tables[t].N, 256 / s.lanes, 8);
+        if (bits == 8) LAUNCH(h, "init_table", k_init_table<8>, g, 256, 0, s, t, init_lo, init_hi);
+        else LAUNCH(h, "init_table", k_init_table<4>, g, 256, 0, s, t, init_lo, init_hi);
+    }
+    CKC(cudaGetLastError());
+    CKC(cudaDeviceSynchronize());
+#undef CKC
+    *out = h;
+    return MPE_OK;
+}
+
+int mpe_reserve(mpe_handle* h, int32_t max_batch, int64_t max_total_indices) {
+    if (!h || max_batch < 0 || max_total_indices < 0 || max_total_indices > 0x7ffffff0LL) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    const int64_t bags = (int64_t)h->T * max_batch;
+    if (max_total_indices <= h->cap_L && bags <= h->cap_bags && h->wk.ctr) return MPE_OK;
+    if (h->have_forward) return MPE_ERR_SEQUENCE;     // a pending backward still needs the old workspace
+    CK(h, cudaStreamSynchronize(h->stream));
+    return alloc_workspace(h, std::max(max_total_indices, h->cap_L), std::max(bags, h->cap_bags));
+}
+
+int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch,
+                int64_t total_indices, float* d_out, void* cuda_stream) {
+    if (!h || !d_offsets || batch < 0 || total_indices < 0 || total_indices > 0x7ffffff0LL) return MPE_ERR_ARG;
+    if ((total_indices > 0 && !d_indices) || (batch > 0 && !d_out)) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (stream != h->stream) { CK(h, cudaStreamSynchronize(h->stream)); h->stream = stream; }
+    h->have_forward = false;
+    const int64_t bags = (int64_t)h->T * batch;
+    if (total_indices > h->cap_L || bags > h->cap_bags || !h->wk.ctr) {
+        int rc = mpe_reserve(h, batch, total_indices);
+        if (rc != MPE_OK) return rc;
+    }
+    const State& s = h->st;
+    Work& w = h->wk;
+    const int T = h->T;
+    const uint32_t L = (uint32_t)total_indices;
+    h->B = batch; h->L = total_indices; ++h->epoch;
+
+    LAUNCH(h, "prelude", k_prelude, 1, 32, 0, w, d_offsets, T, batch, L);
+    LAUNCH(h, "make_keys", k_make_keys, grid_for(h, bags, 8, 8), 256, 0, s, w, d_indices, d_offsets, batch, h->keyA);
+    // sort the row indices of the mini-batch (Section 5.1), table by table
+    const int which = seg_sort(h, h->keyA, h->keyB, h->valA, h->valB, w.table_start, w.tile_base, &w.ctr->hist_len,
+                               bits_for((uint32_t)h->max_rows), total_indices);
+    h->skey = which ? h->keyB : h->keyA;
+    h->spos = which ? h->valB : h->valA;
+    // distinct rows
+    const int gs = grid_for(h, total_indices, SCAN_TILE, 8);
+    LAUNCH(h, "unique_count", k_unique<false>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
+    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, 1024, 0, h->block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);
+    LAUNCH(h, "unique_write", k_unique<true>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
+    LAUNCH(h, "ustart", k_ustart, 1, 256, 0, w, T);
+    // tag lookup, then fetch + pool
+    LAUNCH(h, "probe", k_probe, grid_for(h, total_indices, 256 / s.ways, 8), 256, 0, s, w, h->epoch);
+    LAUNCH(h, "broadcast", k_broadcast, grid_for(h, total_indices, 256, 8), 256, 0, s, w, h->spos, batch);
+    const int gp = grid_for(h, bags, 256 / s.lanes, 8);
+    if (h->bits == 8) LAUNCH(h, "pool", k_pool<8>, gp, 256, 0, s, w, d_indices, d_offsets, batch, d_out);
+    else LAUNCH(h, "pool", k_pool<4>, gp, 256, 0, s, w, d_indices, d_offsets, batch, d_out);
+    int rc = check_launch(h);
+    if (rc != MPE_OK) return rc;
+    h->have_forward = true;
+    return MPE_OK;
+}
+
+int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step) {
+    if (!h || (!d_grad_out && h->B > 0)) return MPE_ERR_ARG;
+    if (!h->have_forward) return MPE_ERR_SEQUENCE;
+    if (step < 1 || step > 0xffffffffLL) return MPE_ERR_ARG;
+    if (step <= h->last_step) return MPE_ERR_SEQUENCE;
+    DeviceGuard guard(h->device);
+    const State& s = h->st;
+    Work& w = h->wk;
+    const int64_t L = h->L;
+    const int B = h->B;
+
+    LAUNCH(h, "priority", k_priority, grid_for(h, L, 256, 8), 256, 0, s, w, (uint32_t)step, h->ckeyA);
+    if (h->max_sets > 0) {
+        // group the rows that missed by cache set, keeping ascending row id inside a set
+        const int which = seg_sort(h, h->ckeyA, h->ckeyB, h->cvalA, h->cvalB, w.ustart, w.ctile_base, &w.ctr->chist_len,
+                                   bits_for((uint32_t)h->max_sets), L);
+        const uint32_t* ck = which ? h->ckeyB : h->ckeyA;
+        const uint32_t* cv = which ? h->cvalB : h->cvalA;
+        LAUNCH(h, "policy", k_policy, grid_for(h, L, 256 / s.ways, 8), 256, 0, s, w, ck, cv, (uint32_t)step, h->epoch);
+    }
+    LAUNCH(h, "hot_partial", k_hot_partial, grid_for(h, L / HOT_SPAN + 1, 1, 4), 256, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
+    const int gu = grid_for(h, L, 256 / s.lanes, 8);
+    for (int phase = 1; phase <= (h->max_sets > 0 ? 2 : 1); ++phase) {
+        if (h->bits == 8) LAUNCH(h, phase == 1 ? "update" : "update_admit", k_update<8>, gu, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step, phase);
+        else LAUNCH(h, phase == 1 ? "update" : "update_admit", k_update<4>, gu, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step, phase);
+    }
+    int rc = check_launch(h);
+    if (rc != MPE_OK) return rc;
+    h->have_forward = false;
+    h->last_step = step;
+    ++h->steps;
+    return MPE_OK;
+}
+
+int mpe_step_host(mpe_handle* h, const int32_t* h_indices, const int32_t* h_offsets, int32_t batch,
+                  int64_t total_indices, const float* h_grad_out, float* h_out, float lr, int64_t step) {
+    if (!h || !h_offsets || batch < 0 || total_indices < 0) return MPE_ERR_ARG;
+    if ((total_indices > 0 && !h_indices) || (batch > 0 && (!h_grad_out || !h_out))) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    const int64_t noff = (int64_t)h->T * batch + 1, nout = (int64_t)batch * h->T * h->dim;
+    if (total_indices > h->sh_cap_L || noff > h->sh_cap_off || nout > h->sh_cap_out) {
+        CK(h, cudaStreamSynchronize(h->stream));
+        cudaFree(h->sh_idx); cudaFree(h->sh_off); cudaFree(h->sh_grad); cudaFree(h->sh_out);
+        h->sh_idx = nullptr; h->sh_off = nullptr; h->sh_grad = nullptr; h->sh_out = nullptr;
+        h->sh_cap_L = std::max(total_indices, h->sh_cap_L); h->sh_cap_off = std::max(noff, h->sh_cap_off);
+        h->sh_cap_out = std::max(nout, h->sh_cap_out);
+        int rc;
+        if ((rc = dmalloc(h, &h->sh_idx, h->sh_cap_L, nullptr)) != MPE_OK) return rc;
+        if ((rc = dmalloc(h, &h->sh_off, h->sh_cap_off, nullptr)) != MPE_OK) return rc;
+        if ((rc = dmalloc(h, &h->sh_grad, h->sh_cap_out, nullptr)) != MPE_OK) return rc;
+        if ((rc = dmalloc(h, &h->sh_out, h->sh_cap_out, nullptr)) != MPE_OK) return rc;
+    }
+    cudaStream_t st = h->stream;
+    if (total_indices) CK(h, cudaMemcpyAsync(h->sh_idx, h_indices, sizeof(int32_t) * total_indices, cudaMemcpyHostToDevice, st));
+    CK(h, cudaMemcpyAsync(h->sh_off, h_offsets, sizeof(int32_t) * noff, cudaMemcpyHostToDevice, st));
+    if (nout) CK(h, cudaMemcpyAsync(h->sh_grad, h_grad_out, sizeof(float) * nout, cudaMemcpyHostToDevice, st));
+    int rc = mpe_forward(h, h->sh_idx, h->sh_off, batch, total_indices, h->sh_out, (void*)st);
+    if (rc != MPE_OK) return rc;
+    rc = mpe_backward(h, h->sh_grad, lr, step);
+    if (rc != MPE_OK) return rc;
+    if (nout) CK(h, cudaMemcpyAsync(h_out, h->sh_out, sizeof(float) * nout, cudaMemcpyDeviceToHost, st));
+    CK(h, cudaStreamSynchronize(st));
+    return MPE_OK;
+}
+
+int mpe_flush(mpe_handle* h) {
+    if (!h) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    const State& s = h->st;
+    for (int t = 0; t < h->T; ++t) {
+        const int64_t nslot = (int64_t)h->tables[t].n_sets * h->ways;
+        if (nslot == 0) continue;
+        const int g = grid_for(h, nslot, 256 / s.lanes, 8);
+        if (h->bits == 8) LAUNCH(h, "flush", k_flush<8>, g, 256, 0, s, t, (uint64_t)h->last_step);
+        else LAUNCH(h, "flush", k_flush<4>, g, 256, 0, s, t, (uint64_t)h->last_step);
+    }
+    return check_launch(h);
+}
+
+int mpe_destroy(mpe_handle* h) {
+    if (!h) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    cudaStreamSynchronize(h->stream);
+    free_workspace(h);
+    State& s = h->st;
+    cudaFree(h->d_tables); cudaFree(s.codes); cudaFree(s.sb); cudaFree(s.cnt); cudaFree(s.G); cudaFree(s.slab);
+    cudaFree(s.tags); cudaFree(s.ts); cudaFree(s.hit_epoch); cudaFree(s.hit_k); cudaFree(s.stats);
+    cudaFree(h->sh_idx); cudaFree(h->sh_off); cudaFree(h->sh_grad); cudaFree(h->sh_out);
+    for (auto& r : h->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (auto e : h->event_pool) cudaEventDestroy(e);
+    delete h;
+    return MPE_OK;
+}
+
+int mpe_last_error(mpe_handle* h, int32_t* code, int64_t* detail) {
+    if (!h || !code || !detail) return MPE_ERR_ARG;
+    *code = MPE_OK; *detail = 0;
+    if (!h->wk.ctr) return MPE_OK;
+    DeviceGuard guard(h->device);
+    CK(h, cudaStreamSynchronize(h->stream));
+    Counters c;
+    CK(h, cudaMemcpy(&c, h->wk.ctr, sizeof(c), cudaMemcpyDeviceToHost));
+    if (c.err[ERR_OFFSETS]) { *code = MPE_ERR_OFFSETS; *detail = (int64_t)c.err[ERR_OFFSETS]; }
+    else if (c.err[ERR_INDEX]) { *code = MPE_ERR_INDEX; *detail = (int64_t)c.err[ERR_INDEX]; }
+    CK(h, cudaMemset(&h->wk.ctr->err[0], 0, sizeof(c.err)));
+    return MPE_OK;
+}
+
+int mpe_stats(mpe_handle* h, int32_t table, uint64_t* out8) {
+    if (!h || !out8 || table < 0 || table >= h->T) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    CK(h, cudaStreamSynchronize(h->stream));
+    CK(h, cudaMemcpy(out8, h->st.stats + (int64_t)table * 8, 8 * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+    out8[7] = h->steps;
+    return MPE_OK;
+}
+
+int mpe_memory_bytes(mpe_handle* h, uint64_t* out6) {
+    if (!h || !out6) return MPE_ERR_ARG;
+    const uint64_t N = (uint64_t)h->total_rows, slots = (uint64_t)h->total_slots, d = (uint64_t)h->dim;
+    out6[0] = N * ((uint64_t)h->bits * d + 64) / 8;                  // E x (bitwidth x D + 64) bits
+    out6[1] = slots * 4 * d;                                         // 4 alpha n d bytes
+    out6[2] = slots * 4;                                             // one INT32 tag per cached row
+    uint64_t pv = 0;
+    for (const TableDev& tb : h->tables)
+        if (tb.n_sets > 0) pv += h->policy == MPE_LFU ? (uint64_t)tb.N * 4 : (uint64_t)tb.n_sets * h->ways * 4;
+    out6[3] = pv;                                                    // INT32 counter per embedding row (LFU) / per cached row (LRU)
+    out6[4] = h->optimizer == MPE_ROWWISE_ADAGRAD ? N * 4 : 0;
+    out6[5] = N * 4 * d;
+    return MPE_OK;
+}
+
+int mpe_cache_geometry(mpe_handle* h, int32_t table, int32_t* n_sets, int32_t* ways) {
+    if (!h || table < 0 || table >= h->T || !n_sets || !ways) return MPE_ERR_ARG;
+    *n_sets = h->tables[table].n_sets; *ways = h->ways;
+    return MPE_OK;
+}
+
+int mpe_step_info(mpe_handle* h, int64_t* out4) {
+    if (!h || !out4) return MPE_ERR_ARG;
+    out4[0] = out4[1] = out4[2] = out4[3] = 0;
+    if (!h->wk.ctr) return MPE_OK;
+    DeviceGuard guard(h->device);
+    CK(h, cudaStreamSynchronize(h->stream));
+    Counters c;
+    CK(h, cudaMemcpy(&c, h->wk.ctr, sizeof(c), cudaMemcpyDeviceToHost));
+    if (c.abort) return MPE_OK;
+    std::vector<int32_t> us(h->T + 1), urow(1);
+    out4[0] = (int64_t)c.L - (int64_t)c.dropped;
+    // distinct rows: the sort puts each table's out-of-range ids into one pseudo row; leave those out
+    int64_t pseudo = 0;
+    if (c.dropped) {
+        CK(h, cudaMemcpy(us.data(), h->wk.ustart, sizeof(int32_t) * (h->T + 1), cudaMemcpyDeviceToHost));
+        for (int t = 0; t < h->T; ++t) {
+            if (us[t + 1] == us[t]) continue;
+            CK(h, cudaMemcpy(urow.data(), h->wk.uniq_row + us[t + 1] - 1, sizeof(int32_t), cudaMemcpyDeviceToHost));
+            if (urow[0] >= h->tables[t].N) ++pseudo;
+        }
+    }
+    out4[1] = (int64_t)c.U - pseudo;
+    out4[2] = (int64_t)c.dropped;
+    out4[3] = (int64_t)c.hot_rows;
+    return MPE_OK;
+}
+
+int mpe_export_rows(mpe_handle* h, int32_t table, const int64_t* h_rows, int64_t n, uint8_t* h_codes,
+                    float* h_scale, float* h_bias) {
+    if (!h || table < 0 || table >= h->T || n < 0 || (n > 0 && (!h_rows || !h_codes || !h_scale || !h_bias))) return MPE_ERR_ARG;
+    if (n == 0) return MPE_OK;
+    DeviceGuard guard(h->device);
+    CK(h, cudaStreamSynchronize(h->stream));
+    int64_t* d_rows = nullptr; uint8_t* d_codes = nullptr; float *d_s = nullptr, *d_b = nullptr;
+    int rc = MPE_OK;
+    if ((rc = dmalloc(h, &d_rows, n, nullptr)) == MPE_OK && (rc = dmalloc(h, &d_codes, n * h->code_bytes, nullptr)) == MPE_OK &&
+        (rc = dmalloc(h, &d_s, n, nullptr)) == MPE_OK && (rc = dmalloc(h, &d_b, n, nullptr)) == MPE_OK) {
+        cudaMemcpy(d_rows, h_rows, sizeof(int64_t) * n, cudaMemcpyHostToDevice);
+        cudaMemset(d_codes, 0, (size_t)n * h->code_bytes); cudaMemset(d_s, 0, sizeof(float) * n); cudaMemset(d_b, 0, sizeof(float) * n);
+        LAUNCH(h, "gather_rows", k_gather_rows, grid_for(h, n, 256, 8), 256, 0, h->st, table, (const int64_t*)d_rows, n, h->code_bytes,
+               d_codes, d_s, d_b, (uint32_t*)nullptr, (float*)nullptr);
+        cudaMemcpy(h_codes, d_codes, (size_t)n * h->code_bytes, cudaMemcpyDeviceToHost);
+        cudaMemcpy(h_scale, d_s, sizeof(float) * n, cudaMemcpyDeviceToHost);
+        cudaMemcpy(h_bias, d_b, sizeof(float) * n, cudaMemcpyDeviceToHost);
+        rc = check_launch(h);
+    }
+    cudaFree(d_rows); cudaFree(d_codes); cudaFree(d_s); cudaFree(d_b);
+    return rc;
+}
+
+int mpe_export_cache(mpe_handle* h, int32_t table, int32_t* h_tags, float* h_rows, uint32_t* h_ts) {
+    if (!h || table < 0 || table >= h->T) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    CK(h, cudaStreamSynchronize(h->stream));
+    const TableDev& tb = h->tables[table];
+    const int64_t nslot = (int64_t)tb.n_sets * h->ways, first = tb.set_base * h->ways;
+    if (nslot == 0) return MPE_OK;
+    if (h_tags) CK(h, cudaMemcpy(h_tags, h->st.tags + first, sizeof(int32_t) * nslot, cudaMemcpyDeviceToHost));
+    if (h_rows) CK(h, cudaMemcpy(h_rows, h->st.slab + first * h->dim, sizeof(float) * nslot * h->dim, cudaMemcpyDeviceToHost));
+    if (h_ts) {
+        if (h->st.ts) CK(h, cudaMemcpy(h_ts, h->st.ts + first, sizeof(uint32_t) * nslot, cudaMemcpyDeviceToHost));
+        else memset(h_ts, 0, sizeof(uint32_t) * nslot);
+    }
+    return MPE_OK;
+}
+
+int mpe_export_aux(mpe_handle* h, int32_t table, const int64_t* h_rows, int64_t n, uint32_t* h_cnt, float* h_adagrad) {
+    if (!h || table < 0 || table >= h->T || n < 0 || (n > 0 && !h_rows)) return MPE_ERR_ARG;
+    if (n == 0 || (!h_cnt && !h_adagrad)) return MPE_OK;
+    DeviceGuard guard(h->device);
+    CK(h, cudaStreamSynchronize(h->stream));
+    int64_t* d_rows = nullptr; uint32_t* d_c = nullptr; float* d_g = nullptr;
+    int rc = MPE_OK;
+    if ((rc = dmalloc(h, &d_rows, n, nullptr)) == MPE_OK && (rc = dmalloc(h, &d_c, n, nullptr)) == MPE_OK &&
+        (rc = dmalloc(h, &d_g, n, nullptr)) == MPE_OK) {
+        cudaMemcpy(d_rows, h_rows, sizeof(int64_t) * n, cudaMemcpyHostToDevice);
+        cudaMemset(d_c, 0, sizeof(uint32_t) * n); cudaMemset(d_g, 0, sizeof(float) * n);
+        LAUNCH(h, "gather_rows", k_gather_rows, grid_for(h, n, 256, 8), 256, 0, h->st, table, (const int64_t*)d_rows, n, h->code_bytes,
+               (uint8_t*)nullptr, (float*)nullptr, (float*)nullptr, d_c, d_g);
+        if (h_cnt) cudaMemcpy(h_cnt, d_c, sizeof(uint32_t) * n, cudaMemcpyDeviceToHost);
+        if (h_adagrad) cudaMemcpy(h_adagrad, d_g, sizeof(float) * n, cudaMemcpyDeviceToHost);
+        rc = check_launch(h);
+    }
+    cudaFree(d_rows); cudaFree(d_c); cudaFree(d_g);
+    return rc;
+}
+
+int mpe_kernel_launches(mpe_handle* h, uint64_t* count) {
+    if (!h || !count) return MPE_ERR_ARG;
+    *count = h->launches;
+    return MPE_OK;
+}
+
+int mpe_profile(mpe_handle* h, int32_t enable) {
+    if (!h) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    CK(h, cudaStreamSynchronize(h->stream));
+    for (auto& r : h->prof_recs) { h->event_pool.push_back(r.a); h->event_pool.push_back(r.b); }
+    h->prof_recs.clear();
+    h->profiling = enable != 0;
+    return MPE_OK;
+}
+
+int mpe_profile_read(mpe_handle* h, int32_t cap, char* names, double* ms, uint64_t* launches, int32_t* n) {
+    if (!h || cap < 0 || !n || (cap > 0 && (!names || !ms || !launches))) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    CK(h, cudaStreamSynchronize(h->stream));
+    std::vector<double> t(h->prof_names.size(), 0.0);
+    std::vector<uint64_t> c(h->prof_names.size(), 0);
+    for (auto& r : h->prof_recs) {
+        float e = 0.f;
+        cudaEventElapsedTime(&e, r.a, r.b);
+        t[r.name] += e; c[r.name] += 1;
+        h->event_pool.push_back(r.a); h->event_pool.push_back(r.b);
+    }
+    h->prof_recs.clear();
+    int32_t k = 0;
+    for (size_t i = 0; i < h->prof_names.size() && k < cap; ++i) {
+        if (!c[i]) continue;
+        std::memset(names + 32 * k, 0, 32);
+        std::strncpy(names + 32 * k, h->prof_names[i].c_str(), 31);
+        ms[k] = t[i]; launches[k] = c[i]; ++k;
+    }
+    *n = k;
+    return MPE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,124 @@
+// Device-side building blocks: counter hash, set hash, row loads, the row-wise
+// min-max quantizer with nearest-even or stochastic rounding (Section 3
+// "Precision"/"Rounding", Algorithm 1).  Every FP32 operation that feeds a stored
+// code is spelled with an explicit rounding intrinsic so that the compiler can
+// neither contract nor reorder it.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mpe {
+
+constexpr uint32_t DOMAIN_INIT = 1, DOMAIN_SR = 2, DOMAIN_FLUSH = 3;
+constexpr int LOC_MISS = -1;      // unique row not cache resident
+constexpr int LOC_INVALID = -2;   // pseudo row collecting out-of-range indices
+
+__host__ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
+    x ^= x >> 16; x *= 0x7feb352dU; x ^= x >> 15; x *= 0x846ca68bU; x ^= x >> 16;
+    return x;
+}
+__host__ __device__ __forceinline__ uint32_t absorb(uint32_t h, uint32_t w) { return mix32((h ^ w) + 0x9E3779B9U); }
+
+// per-(row, step) key of the counter-based generator; one mixing round per column follows
+__host__ __device__ __forceinline__ uint32_t rowkey(uint64_t seed, uint32_t domain, uint32_t table, uint32_t row, uint64_t step) {
+    uint32_t h = 0x243F6A88U;
+    h = absorb(h, (uint32_t)seed); h = absorb(h, (uint32_t)(seed >> 32));
+    h = absorb(h, domain); h = absorb(h, table); h = absorb(h, row);
+    h = absorb(h, (uint32_t)step); h = absorb(h, (uint32_t)(step >> 32));
+    return h;
+}
+__device__ __forceinline__ float uniform01(uint32_t key, uint32_t column) {
+    uint32_t bits = mix32(key ^ (column * 0x9E3779B9U + 0x7F4A7C15U));
+    return __uint2float_rn(bits >> 8) * 0x1p-24f;   // exact
+}
+__host__ __device__ __forceinline__ uint32_t table_salt(uint64_t seed, uint32_t table) {
+    uint32_t h = 0x13198A2EU;
+    h = absorb(h, (uint32_t)seed); h = absorb(h, (uint32_t)(seed >> 32)); h = absorb(h, table);
+    return h;
+}
+// h : row -> set (Section 3 "Cache Structure")
+__device__ __forceinline__ int set_of(uint32_t row, uint32_t salt, int n_sets) {
+    return (int)(((uint64_t)mix32(row ^ salt) * (uint64_t)(uint32_t)n_sets) >> 32);
+}
+
+// A row of `dim` values is handled by dim/4 consecutive lanes, four columns per lane.
+__device__ __forceinline__ uint32_t group_mask(int lanes_per_row) {
+    const int lane = threadIdx.x & 31;
+    return lanes_per_row == 32 ? 0xffffffffU : (((1U << lanes_per_row) - 1U) << (lane & ~(lanes_per_row - 1)));
+}
+
+// RO = the table is not written by the running kernel, so the read-only data path may serve the loads
+template <int BITS, bool RO>
+__device__ __forceinline__ float4 dequant4(const uint8_t* codes, const float2* sb, int64_t grow, int dim, int sub) {
+    // up-conversion q*s + b (Algorithm 1, last line of the loop)
+    float2 p;
+    uint32_t q;
+    if (RO) {
+        p = __ldg(sb + grow);
+        if (BITS == 8) q = __ldg(reinterpret_cast<const uint32_t*>(codes + grow * dim) + sub);
+        else           q = __ldg(reinterpret_cast<const uint16_t*>(codes + grow * (dim >> 1)) + sub);
+    } else {
+        p = sb[grow];
+        if (BITS == 8) q = reinterpret_cast<const uint32_t*>(codes + grow * dim)[sub];
+        else           q = reinterpret_cast<const uint16_t*>(codes + grow * (dim >> 1))[sub];
+    }
+    float4 x;
+    if (BITS == 8) {
+        x.x = __fmaf_rn(__uint2float_rn(q & 255u), p.x, p.y);
+        x.y = __fmaf_rn(__uint2float_rn((q >> 8) & 255u), p.x, p.y);
+        x.z = __fmaf_rn(__uint2float_rn((q >> 16) & 255u), p.x, p.y);
+        x.w = __fmaf_rn(__uint2float_rn(q >> 24), p.x, p.y);
+    } else {
+        x.x = __fmaf_rn(__uint2float_rn(q & 15u), p.x, p.y);
+        x.y = __fmaf_rn(__uint2float_rn((q >> 4) & 15u), p.x, p.y);
+        x.z = __fmaf_rn(__uint2float_rn((q >> 8) & 15u), p.x, p.y);
+        x.w = __fmaf_rn(__uint2float_rn((q >> 12) & 15u), p.x, p.y);
+    }
+    return x;
+}
+
+__device__ __forceinline__ float4 add4(float4 a, float4 b) {
+    return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
+}
+
+template <int BITS, bool STOCHASTIC>
+__device__ __forceinline__ uint32_t quant1(float x, float mn, float inv, float qmax, uint32_t key, uint32_t column) {
+    float y = __fmul_rn(__fsub_rn(x, mn), inv);           // (x - b)/s as (x - b) * (1/s)
+    y = fminf(fmaxf(y, 0.0f), qmax);
+    if (STOCHASTIC) {
+        const float f = floorf(y);
+        const float p = __fsub_rn(y, f);                   // exact
+        const float u = uniform01(key, column);
+        return (uint32_t)f + (u < p ? 1u : 0u);            // x+ with probability p: expectation y
+    }
+    return (uint32_t)rintf(y);                             // nearest, ties to even
+}
+
+// Down-convert one FP32 row (four columns per lane) into the low-precision table.
+template <int BITS, bool STOCHASTIC>
+__device__ __forceinline__ void quantize_store(float4 x, uint8_t* __restrict__ codes, float2* __restrict__ sb,
+                                               int64_t grow, int dim, int sub, int lanes_per_row, uint32_t key) {
+    const uint32_t mask = group_mask(lanes_per_row);
+    float mn = fminf(fminf(x.x, x.y), fminf(x.z, x.w));
+    float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
+    for (int o = lanes_per_row >> 1; o > 0; o >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(mask, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(mask, mx, o));
+    }
+    mn = __fadd_rn(mn, 0.0f);                              // -0 -> +0
+    const float qmax = (float)((1 << BITS) - 1);
+    float s = __fdiv_rn(__fsub_rn(mx, mn), qmax);          // s = (max - min)/(2^N - 1)
+    float inv = 0.0f;
+    if (s >= 1.17549435e-38f) inv = __fdiv_rn(1.0f, s);
+    if (inv == 0.0f) s = 0.0f;
+    const uint32_t c = 4u * (uint32_t)sub;
+    const uint32_t q0 = quant1<BITS, STOCHASTIC>(x.x, mn, inv, qmax, key, c);
+    const uint32_t q1 = quant1<BITS, STOCHASTIC>(x.y, mn, inv, qmax, key, c + 1);
+    const uint32_t q2 = quant1<BITS, STOCHASTIC>(x.z, mn, inv, qmax, key, c + 2);
+    const uint32_t q3 = quant1<BITS, STOCHASTIC>(x.w, mn, inv, qmax, key, c + 3);
+    if (BITS == 8) reinterpret_cast<uint32_t*>(codes + grow * dim)[sub] = q0 | (q1 << 8) | (q2 << 16) | (q3 << 24);
+    else reinterpret_cast<uint16_t*>(codes + grow * (dim >> 1))[sub] = (uint16_t)(q0 | (q1 << 4) | (q2 << 8) | (q3 << 12));
+    if (sub == 0) sb[grow] = make_float2(s, mn);
+}
+
+}  // namespace mpe

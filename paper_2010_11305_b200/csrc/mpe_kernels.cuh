@@ -1,0 +1,585 @@
+// Kernels of the training step.  Naming follows the paper: T = low-precision
+// table, C = FP32 cache, I_C = tags, PV = priority values, I_U = distinct rows
+// of the batch (Section 3, Algorithm 2, Section 5.1).
+#pragma once
+#include "mpe_device.cuh"
+#include "mpe_sort.cuh"
+
+namespace mpe {
+
+constexpr int HOT_SPAN = 1024;        // occurrences covered by one multi-block gradient task (two tree levels)
+constexpr int ERR_INDEX = 0, ERR_OFFSETS = 1;
+
+struct TableDev {
+    int64_t row_base;    // first row of this table in the concatenated store
+    int64_t set_base;    // first set of this table in the concatenated cache
+    int32_t N;           // rows
+    int32_t n_sets;      // cache sets (0 = no cache)
+    uint32_t salt;       // of the set hash
+    int32_t pad;
+};
+
+struct Counters {
+    uint32_t L;            // indices in this batch
+    uint32_t U;            // distinct (table,row) pairs incl. one pseudo row per table that had bad indices
+    uint32_t hist_len;     // 256 * number of sort tiles (main sort)
+    uint32_t chist_len;    // same for the candidate sort
+    uint32_t hot_rows;
+    uint32_t hot_tasks;
+    uint32_t abort;        // offsets were inconsistent: every later kernel of the step returns at once
+    uint32_t pad;
+    unsigned long long dropped;      // out-of-range indices in this batch
+    unsigned long long err[2];       // sticky: ERR_INDEX, ERR_OFFSETS
+};
+
+struct State {
+    int T, dim, lanes, ways, policy, optimizer, bits;
+    uint64_t seed;
+    float eps;
+    const TableDev* tables;
+    uint8_t* codes;        // [sum N][dim*bits/8]
+    float2* sb;            // [sum N] (scale, bias)
+    uint32_t* cnt;         // LFU: [sum N]
+    float* G;              // Adagrad: [sum N]
+    float* slab;           // [slots][dim]
+    int32_t* tags;         // [slots], -1 empty
+    uint32_t* ts;          // LRU: [slots]
+    uint32_t* hit_epoch;   // [slots] forward call in which the slot was last hit
+    int32_t* hit_k;        // [slots] unique-row index of that hit
+    unsigned long long* stats;   // [T][8]
+};
+
+struct Work {
+    Counters* ctr;
+    int32_t *table_start, *tile_base, *ustart, *ctile_base;   // [T+1]
+    int32_t* bag_of;       // [L] bag of every index position
+    uint32_t* kidx;        // [L] unique-row index of the i-th sorted element
+    int32_t* occ_loc;      // [L] by position: cache slot, LOC_MISS or LOC_INVALID
+    int32_t* occ_b;        // [L] by sorted order: sample of the element
+    int32_t *uniq_row, *uniq_t, *seg, *loc, *final_loc, *victim, *hot_base, *uset;   // per unique row
+    int32_t* task_k;       // [hot tasks]
+    float* partial;        // [hot tasks][dim]
+};
+
+// ---------------------------------------------------------------------------------------------
+// step prologue
+// ---------------------------------------------------------------------------------------------
+__global__ void k_prelude(Work w, const int32_t* __restrict__ offsets, int T, int B, uint32_t L) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        Counters* c = w.ctr;
+        c->L = L; c->U = 0; c->hot_rows = 0; c->hot_tasks = 0; c->abort = 0; c->dropped = 0;
+        bool bad = offsets[0] != 0 || offsets[(int64_t)T * B] != (int32_t)L;
+        int32_t prev = 0;
+        w.table_start[0] = 0;
+        for (int t = 1; t < T; ++t) {
+            int32_t v = offsets[(int64_t)t * B];
+            if (v < prev || v > (int32_t)L) { bad = true; v = prev; }
+            w.table_start[t] = v; prev = v;
+        }
+        w.table_start[T] = (int32_t)L;
+        if (bad) { c->abort = 1; atomicAdd(&c->err[ERR_OFFSETS], 1ULL); }
+    }
+}
+
+// keys for the sort: the row id, or N_t for an id outside [0, N_t); one warp per bag
+__global__ void k_make_keys(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets,
+                            int B, uint32_t* __restrict__ keys) {
+    const int lane = threadIdx.x & 31;
+    const int64_t nbags = (int64_t)s.T * B;
+    const int64_t nw = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int32_t L = (int32_t)w.ctr->L;
+    for (int64_t bag = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); bag < nbags; bag += nw) {
+        const int32_t lo = offsets[bag], hi = offsets[bag + 1];
+        if (lo < 0 || hi < lo || hi > L) {
+            if (lane == 0) { w.ctr->abort = 1; atomicAdd(&w.ctr->err[ERR_OFFSETS], 1ULL); }
+            continue;
+        }
+        const int t = (int)(bag / B);
+        const int32_t N = s.tables[t].N;
+        int bad = 0;
+        for (int32_t p = lo + lane; p < hi; p += 32) {
+            const int32_t r = indices[p];
+            const bool ok = r >= 0 && r < N;
+            keys[p] = ok ? (uint32_t)r : (uint32_t)N;
+            w.bag_of[p] = (int32_t)bag;
+            bad += !ok;
+        }
+        bad = __reduce_add_sync(0xffffffffU, bad);
+        if (lane == 0 && bad) { atomicAdd(&w.ctr->dropped, (unsigned long long)bad); atomicAdd(&w.ctr->err[ERR_INDEX], (unsigned long long)bad); }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// distinct rows of the sorted batch (I_U), multiplicities, element -> distinct-row map
+// ---------------------------------------------------------------------------------------------
+template <bool WRITE>
+__global__ void __launch_bounds__(SCAN_THREADS)
+k_unique(Work w, int T, const uint32_t* __restrict__ skey, uint32_t* __restrict__ block_sums) {
+    __shared__ uint32_t tmp[SCAN_THREADS / 32 + 1];
+    if (w.ctr->abort) return;
+    const uint32_t n = w.ctr->L;
+    const uint32_t nblk = (n + SCAN_TILE - 1) / SCAN_TILE;
+    for (uint32_t b = blockIdx.x; b < nblk; b += gridDim.x) {
+        const uint32_t base = b * SCAN_TILE + threadIdx.x * SCAN_ITEMS;
+        uint32_t flag[SCAN_ITEMS];
+        int tcur[SCAN_ITEMS];
+        uint32_t sum = 0;
+        if (base < n) {
+            int t = find_segment(w.table_start, T, (int32_t)base);
+            while (w.table_start[t + 1] <= (int32_t)base) ++t;     // skip empty tables that start here
+            uint32_t prev = base > 0 ? skey[base - 1] : 0;
+#pragma unroll
+            for (int i = 0; i < SCAN_ITEMS; ++i) {
+                const uint32_t e = base + i;
+                flag[i] = 0; tcur[i] = t;
+                if (e < n) {
+                    while (w.table_start[t + 1] <= (int32_t)e) ++t;
+                    tcur[i] = t;
+                    const uint32_t k = skey[e];
+                    flag[i] = (e == (uint32_t)w.table_start[t] || k != prev) ? 1u : 0u;
+                    prev = k;
+                    sum += flag[i];
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < SCAN_ITEMS; ++i) { flag[i] = 0; tcur[i] = 0; }
+        }
+        uint32_t total;
+        uint32_t ex = block_exclusive_scan<SCAN_THREADS>(sum, &total, tmp);
+        if (!WRITE) {
+            if (threadIdx.x == 0) block_sums[b] = total;
+        } else {
+            ex += block_sums[b];
+#pragma unroll
+            for (int i = 0; i < SCAN_ITEMS; ++i) {
+                const uint32_t e = base + i;
+                if (e < n) {
+                    ex += flag[i];
+                    const uint32_t k = ex - 1;
+                    w.kidx[e] = k;
+                    if (flag[i]) { w.uniq_row[k] = (int32_t)skey[e]; w.uniq_t[k] = tcur[i]; w.seg[k] = (int32_t)e; }
+                }
+            }
+        }
+    }
+}
+
+__global__ void k_ustart(Work w, int T) {
+    if (w.ctr->abort) return;
+    const uint32_t L = w.ctr->L, U = w.ctr->U;
+    for (int t = blockIdx.x * blockDim.x + threadIdx.x; t <= T; t += gridDim.x * blockDim.x) {
+        const int32_t s = w.table_start[t];
+        w.ustart[t] = (uint32_t)s < L ? (int32_t)w.kidx[s] : (int32_t)U;
+        if (t == 0) w.seg[U] = (int32_t)L;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// cache tag lookup: one group of `ways` lanes per distinct row (Section 3 "Cache Structure")
+// ---------------------------------------------------------------------------------------------
+__global__ void k_probe(State s, Work w, uint32_t epoch) {
+    if (w.ctr->abort) return;
+    const int ways = s.ways;
+    const int lane = threadIdx.x & 31, way = lane & (ways - 1);
+    const uint32_t gmask = group_mask(ways);
+    const int64_t U = w.ctr->U;
+    const int64_t gpb = blockDim.x / ways, ng = gpb * gridDim.x;
+    for (int64_t k = blockIdx.x * gpb + threadIdx.x / ways; k < U; k += ng) {
+        const int t = w.uniq_t[k];
+        const int32_t row = w.uniq_row[k];
+        const TableDev tb = s.tables[t];
+        int loc = LOC_MISS, set = 0;
+        if (row >= tb.N) loc = LOC_INVALID;
+        else if (tb.n_sets > 0) {
+            set = set_of((uint32_t)row, tb.salt, tb.n_sets);
+            const int64_t slot = (tb.set_base + set) * ways + way;
+            const bool match = s.tags[slot] == row;
+            const uint32_t hit = __ballot_sync(gmask, match) & gmask;
+            if (hit) {
+                loc = (int)((tb.set_base + set) * ways + (__ffs(hit) - 1 - (lane & ~(ways - 1))));
+                if (match) { s.hit_epoch[slot] = epoch; s.hit_k[slot] = (int32_t)k; }
+            }
+        }
+        if (way == 0) { w.loc[k] = loc; w.final_loc[k] = loc; w.uset[k] = set; }
+    }
+}
+
+// per sorted element: where its row lives (by index position) and which sample it belongs to
+__global__ void k_broadcast(State s, Work w, const uint32_t* __restrict__ spos, int B) {
+    if (w.ctr->abort) return;
+    const int64_t L = w.ctr->L;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < L; i += (int64_t)gridDim.x * blockDim.x) {
+        const uint32_t k = w.kidx[i];
+        const uint32_t p = spos[i];
+        w.occ_loc[p] = w.loc[k];
+        w.occ_b[i] = w.bag_of[p] - w.uniq_t[k] * B;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// forward: fetch + sum-pool, one group of dim/4 lanes per bag (Section 3 fetch; Algorithm 1 up-conversion)
+// ---------------------------------------------------------------------------------------------
+template <int BITS, bool RO>
+__device__ __forceinline__ float4 fetch4(const State& s, const TableDev& tb, int32_t row, int loc, int sub) {
+    if (loc >= 0) {
+        const float4* src = reinterpret_cast<const float4*>(s.slab + (int64_t)loc * s.dim) + sub;
+        return RO ? __ldg(src) : *src;
+    }
+    return dequant4<BITS, RO>(s.codes, s.sb, tb.row_base + row, s.dim, sub);
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(256)
+k_pool(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int B,
+       float* __restrict__ out) {
+    const int lanes = s.lanes;
+    const int sub = threadIdx.x & (lanes - 1);
+    const int64_t nbags = (int64_t)s.T * B;
+    const int64_t gpb = blockDim.x / lanes, ng = gpb * gridDim.x;
+    const bool abort = w.ctr->abort != 0;
+    for (int64_t bag = blockIdx.x * gpb + threadIdx.x / lanes; bag < nbags; bag += ng) {
+        const int t = (int)(bag / B);
+        const int b = (int)(bag - (int64_t)t * B);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (!abort) {
+            const TableDev tb = s.tables[t];
+            const int32_t lo = offsets[bag], hi = offsets[bag + 1];
+            for (int32_t p = lo; p < hi; p += 4) {
+                int loc[4]; int32_t row[4]; float4 x[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) if (p + u < hi) { loc[u] = w.occ_loc[p + u]; row[u] = indices[p + u]; }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) if (p + u < hi && loc[u] != LOC_INVALID) x[u] = fetch4<BITS, true>(s, tb, row[u], loc[u], sub);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) if (p + u < hi && loc[u] != LOC_INVALID) acc = add4(acc, x[u]);
+            }
+        }
+        reinterpret_cast<float4*>(out + ((int64_t)b * s.T + t) * s.dim)[sub] = acc;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// backward 1: "Update PV[i]" for every i in I_U (Algorithm 2), candidate keys, hot-row tasks, counters
+// ---------------------------------------------------------------------------------------------
+__global__ void k_priority(State s, Work w, uint32_t step, uint32_t* __restrict__ ckey) {
+    if (w.ctr->abort) return;
+    const int64_t U = w.ctr->U;
+    const int64_t U32 = (U + 31) & ~31LL;
+    for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < U32; k += (int64_t)gridDim.x * blockDim.x) {
+        int t = -1; unsigned long long m = 0, hitm = 0, uh = 0, un = 0;
+        if (k < U) {
+            t = w.uniq_t[k];
+            const TableDev tb = s.tables[t];
+            const int32_t row = w.uniq_row[k];
+            const int loc = w.loc[k];
+            const uint32_t mult = (uint32_t)(w.seg[k + 1] - w.seg[k]);
+            uint32_t key = (uint32_t)tb.n_sets;              // sorts behind every real set: not a candidate
+            int hb = -1;
+            if (loc != LOC_INVALID) {
+                m = mult; un = 1;
+                if (s.policy == 1) {                         // LFU: access count of the row, saturating
+                    uint32_t* c = s.cnt + tb.row_base + row;
+                    const uint32_t old = *c;
+                    *c = old + mult < old ? 0xffffffffU : old + mult;
+                } else if (loc >= 0) {
+                    s.ts[loc] = step;                        // LRU: time stamp of the cached row
+                }
+                if (loc >= 0) { hitm = mult; uh = 1; }
+                else if (tb.n_sets > 0) key = (uint32_t)w.uset[k];
+                if (mult > (uint32_t)HOT_SPAN) {
+                    const uint32_t nt = (mult + HOT_SPAN - 1) / HOT_SPAN;
+                    hb = (int)atomicAdd(&w.ctr->hot_tasks, nt);
+                    atomicAdd(&w.ctr->hot_rows, 1u);
+                    for (uint32_t j = 0; j < nt; ++j) w.task_k[hb + j] = (int32_t)k;
+                }
+            }
+            ckey[k] = key;
+            w.hot_base[k] = hb;
+        }
+        // counters: one atomic per warp when the warp sits inside one table
+        const int t0 = __shfl_sync(0xffffffffU, t, 0);
+        const bool same = __all_sync(0xffffffffU, t == t0 || t < 0);
+        if (same && t0 >= 0) {
+            for (int o = 16; o > 0; o >>= 1) {
+                m += __shfl_xor_sync(0xffffffffU, m, o); hitm += __shfl_xor_sync(0xffffffffU, hitm, o);
+                uh += __shfl_xor_sync(0xffffffffU, uh, o); un += __shfl_xor_sync(0xffffffffU, un, o);
+            }
+            if ((threadIdx.x & 31) == 0) {
+                unsigned long long* st = s.stats + (int64_t)t0 * 8;
+                atomicAdd(st + 0, m); atomicAdd(st + 1, hitm); atomicAdd(st + 2, un); atomicAdd(st + 3, uh);
+            }
+        } else if (t >= 0) {
+            unsigned long long* st = s.stats + (int64_t)t * 8;
+            atomicAdd(st + 0, m); atomicAdd(st + 1, hitm); atomicAdd(st + 2, un); atomicAdd(st + 3, uh);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// backward 2: admission / eviction, integer only.  One group of `ways` lanes walks the miss
+// candidates of one set in ascending row id (Algorithm 2: j <- argmin PV; PV[i] <= PV[j] -> bypass,
+// else replace j by i in I_C[s]).  No row value is read or written here.
+// ---------------------------------------------------------------------------------------------
+__global__ void k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __restrict__ cval,
+                         uint32_t step, uint32_t epoch) {
+    if (w.ctr->abort) return;
+    const int ways = s.ways;
+    const int lane = threadIdx.x & 31, way = lane & (ways - 1);
+    const uint32_t gmask = group_mask(ways);
+    const int64_t U = w.ctr->U;
+    const int64_t gpb = blockDim.x / ways, ng = gpb * gridDim.x;
+    for (int64_t j = blockIdx.x * gpb + threadIdx.x / ways; j < U; j += ng) {
+        const uint32_t key = ckey[j];
+        const int t = w.uniq_t[cval[j]];
+        const TableDev tb = s.tables[t];
+        if (key >= (uint32_t)tb.n_sets) continue;                       // not a candidate
+        if (j != w.ustart[t] && ckey[j - 1] == key) continue;           // not the first candidate of its set
+        const int64_t slot = (tb.set_base + key) * ways + way;
+        int32_t tag = s.tags[slot];
+        uint32_t pri = 0;
+        if (tag >= 0) pri = s.policy == 1 ? s.cnt[tb.row_base + tag] : s.ts[slot];
+        int32_t cand = -1, vict = -1;
+        uint32_t n_admit = 0, n_evict = 0, n_bypass = 0;
+        const int64_t jend = w.ustart[t + 1];
+        for (int64_t jj = j; jj < jend && ckey[jj] == key; ++jj) {
+            const int32_t kk = (int32_t)cval[jj];
+            const int32_t row = w.uniq_row[kk];
+            const uint32_t pv = s.policy == 1 ? s.cnt[tb.row_base + row] : step;
+            // empty ways rank below every priority; ties go to the lowest way
+            unsigned long long mine = tag < 0 ? (unsigned long long)way : ((((unsigned long long)pri + 1ULL) << 8) | (unsigned long long)way);
+            unsigned long long best = mine;
+            for (int o = ways >> 1; o > 0; o >>= 1) {
+                const unsigned long long other = __shfl_xor_sync(gmask, best, o);
+                best = other < best ? other : best;
+            }
+            const int jw = (int)(best & 255ULL);
+            const unsigned long long jp = best >> 8;                   // 0 = empty, else PV[j] + 1
+            bool replace = jp == 0 || (unsigned long long)pv + 1ULL > jp;
+            if (ways == 1 && s.policy == 0) replace = true;              // direct-mapped LRU never compares
+            if (replace) {
+                ++n_admit;
+                if (jp != 0) ++n_evict;
+                if (way == jw) {
+                    if (tag >= 0 && cand < 0) {
+                        // a row that was resident when the step began leaves the cache
+                        if (s.hit_epoch[slot] == epoch) { w.final_loc[s.hit_k[slot]] = LOC_MISS; vict = -1; }
+                        else vict = tag;
+                    }
+                    tag = row; pri = pv; cand = kk;
+                }
+            } else {
+                ++n_bypass;
+            }
+        }
+        if (cand >= 0) {
+            s.tags[slot] = tag;
+            if (s.policy == 0) s.ts[slot] = step;
+            w.final_loc[cand] = (int32_t)slot;
+            w.victim[cand] = vict;
+        }
+        if (way == 0) {
+            unsigned long long* st = s.stats + (int64_t)t * 8;
+            if (n_admit) atomicAdd(st + 4, (unsigned long long)n_admit);
+            if (n_evict) atomicAdd(st + 5, (unsigned long long)n_evict);
+            if (n_bypass) atomicAdd(st + 6, (unsigned long long)n_bypass);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// backward 3: merged gradient of one distinct row (Section 5.1), radix-32 tree over index positions
+// ---------------------------------------------------------------------------------------------
+// up to 32 consecutive occurrences, added left to right
+__device__ __forceinline__ float4 sum_occurrences(const Work& w, const float* __restrict__ grad, int64_t col, int64_t stride,
+                                                  int32_t first, int len) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j0 = 0; j0 < len; j0 += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (j0 + u < len) v[u] = __ldg(reinterpret_cast<const float4*>(grad + (int64_t)w.occ_b[first + j0 + u] * stride + col));
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (j0 + u < len) acc = (j0 + u == 0) ? v[u] : add4(acc, v[u]);
+    }
+    return acc;
+}
+
+// LEVEL 0 adds up to 32 terms left to right; LEVEL l adds up to 32 results of LEVEL l-1
+template <int LEVEL, class Term>
+__device__ __forceinline__ float4 tree_reduce(const Term& term, int64_t first, int64_t n) {
+    if constexpr (LEVEL == 0) {
+        float4 acc = term(first);
+        for (int64_t j = 1; j < n; ++j) acc = add4(acc, term(first + j));
+        return acc;
+    } else {
+        int64_t span = 32;
+        for (int l = 1; l < LEVEL; ++l) span *= 32;
+        float4 acc = tree_reduce<LEVEL - 1>(term, first, n < span ? n : span);
+        for (int64_t c = span; c < n; c += span)
+            acc = add4(acc, tree_reduce<LEVEL - 1>(term, first + c, n - c < span ? n - c : span));
+        return acc;
+    }
+}
+
+// rows with more than HOT_SPAN occurrences: one block per HOT_SPAN occurrences computes two tree levels
+__global__ void __launch_bounds__(256)
+k_hot_partial(State s, Work w, const float* __restrict__ grad, int B) {
+    extern __shared__ float chunk_sums[];     // [32][dim]
+    if (w.ctr->abort) return;
+    const int lanes = s.lanes, dim = s.dim;
+    const int sub = threadIdx.x & (lanes - 1), grp = threadIdx.x / lanes, ngrp = blockDim.x / lanes;
+    const uint32_t ntask = w.ctr->hot_tasks;
+    const int64_t stride = (int64_t)s.T * dim;
+    for (uint32_t task = blockIdx.x; task < ntask; task += gridDim.x) {
+        const int32_t k = w.task_k[task];
+        const int32_t j = (int32_t)task - w.hot_base[k];
+        const int32_t first = w.seg[k] + j * HOT_SPAN;
+        const int32_t n = min(HOT_SPAN, w.seg[k + 1] - first);
+        const int nchunk = (n + 31) >> 5;
+        const int64_t col = (int64_t)w.uniq_t[k] * dim + 4 * sub;
+        for (int c = grp; c < nchunk; c += ngrp) {
+            const float4 v = sum_occurrences(w, grad, col, stride, first + 32 * c, min(32, n - 32 * c));
+            reinterpret_cast<float4*>(chunk_sums + c * dim)[sub] = v;
+        }
+        __syncthreads();
+        if (grp == 0) {
+            float4 acc = reinterpret_cast<const float4*>(chunk_sums)[sub];
+            for (int c = 1; c < nchunk; ++c) acc = add4(acc, reinterpret_cast<const float4*>(chunk_sums + c * dim)[sub]);
+            reinterpret_cast<float4*>(w.partial + (int64_t)task * dim)[sub] = acc;
+        }
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// backward 4: update(T, C, i, x).  phase 1: every distinct row except those that end the step as
+// new cache residents; phase 2: those, after the row they displace has been written back.
+// ---------------------------------------------------------------------------------------------
+template <int BITS>
+__global__ void __launch_bounds__(256)
+k_update(State s, Work w, const float* __restrict__ grad, int B, float lr, uint64_t step, int phase) {
+    if (w.ctr->abort) return;
+    const int lanes = s.lanes, dim = s.dim;
+    const int sub = threadIdx.x & (lanes - 1);
+    const uint32_t gmask = group_mask(lanes);
+    const int64_t U = w.ctr->U;
+    const int64_t gpb = blockDim.x / lanes, ng = gpb * gridDim.x;
+    const int64_t stride = (int64_t)s.T * dim;
+    for (int64_t k = blockIdx.x * gpb + threadIdx.x / lanes; k < U; k += ng) {
+        const int loc = w.loc[k];
+        if (loc == LOC_INVALID) continue;
+        const int floc = w.final_loc[k];
+        const bool newcomer = loc < 0 && floc >= 0;
+        if (newcomer != (phase == 2)) continue;
+        const int t = w.uniq_t[k];
+        const int32_t row = w.uniq_row[k];
+        const TableDev tb = s.tables[t];
+        const int64_t grow = tb.row_base + row;
+        const int32_t first = w.seg[k], m = w.seg[k + 1] - first;
+        const int64_t col = (int64_t)t * dim + 4 * sub;
+        // merged gradient
+        float4 g;
+        const int hb = w.hot_base[k];
+        if (hb < 0) {
+            auto chunk = [&](int64_t c) { return sum_occurrences(w, grad, col, stride, first + 32 * (int32_t)c, min(32, m - 32 * (int32_t)c)); };
+            g = tree_reduce<0>(chunk, 0, (m + 31) >> 5);
+        } else {
+            const float* part = w.partial + (int64_t)hb * dim + 4 * sub;
+            auto term = [&](int64_t j) { return *reinterpret_cast<const float4*>(part + j * dim); };
+            g = tree_reduce<4>(term, 0, (m + HOT_SPAN - 1) / HOT_SPAN);
+        }
+        // the value the forward fetched
+        const float4 x = fetch4<BITS, false>(s, tb, row, loc, sub);
+        // optimizer, full precision
+        float mult = lr;
+        if (s.optimizer == 1) {
+            float a = __fmul_rn(g.x, g.x);
+            a = __fmaf_rn(g.y, g.y, a); a = __fmaf_rn(g.z, g.z, a); a = __fmaf_rn(g.w, g.w, a);
+            for (int o = lanes >> 1; o > 0; o >>= 1) a = __fadd_rn(a, __shfl_xor_sync(gmask, a, o));
+            const float Gold = s.G[grow];
+            __syncwarp(gmask);                               // every lane has read G before lane 0 replaces it
+            const float Gn = __fadd_rn(Gold, __fmul_rn(a, __fdiv_rn(1.0f, (float)dim)));
+            if (sub == 0) s.G[grow] = Gn;
+            mult = __fdiv_rn(lr, __fadd_rn(__fsqrt_rn(Gn), s.eps));
+        }
+        float4 xn;
+        xn.x = __fmaf_rn(-mult, g.x, x.x); xn.y = __fmaf_rn(-mult, g.y, x.y);
+        xn.z = __fmaf_rn(-mult, g.z, x.z); xn.w = __fmaf_rn(-mult, g.w, x.w);
+        if (floc >= 0) {
+            float4* dst = reinterpret_cast<float4*>(s.slab + (int64_t)floc * dim) + sub;
+            if (phase == 2) {
+                const int32_t v = w.victim[k];
+                if (v >= 0)   // the displaced row is down-converted and placed back in T
+                    quantize_store<BITS, true>(*dst, s.codes, s.sb, tb.row_base + v, dim, sub, lanes,
+                                               rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)v, step));
+            }
+            *dst = xn;       // cached rows keep full precision, a newcomer enters verbatim
+        } else {
+            quantize_store<BITS, true>(xn, s.codes, s.sb, grow, dim, sub, lanes,
+                                       rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)row, step));
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// create / flush / export
+// ---------------------------------------------------------------------------------------------
+template <int BITS>
+__global__ void k_init_table(State s, int t, float lo, float hi) {
+    const int lanes = s.lanes;
+    const int sub = threadIdx.x & (lanes - 1);
+    const TableDev tb = s.tables[t];
+    const int64_t gpb = blockDim.x / lanes, ng = gpb * gridDim.x;
+    const float width = __fsub_rn(hi, lo);
+    for (int64_t row = blockIdx.x * gpb + threadIdx.x / lanes; row < tb.N; row += ng) {
+        const uint32_t key = rowkey(s.seed, DOMAIN_INIT, (uint32_t)t, (uint32_t)row, 0);
+        float4 x;
+        x.x = __fmaf_rn(uniform01(key, 4 * sub + 0), width, lo);
+        x.y = __fmaf_rn(uniform01(key, 4 * sub + 1), width, lo);
+        x.z = __fmaf_rn(uniform01(key, 4 * sub + 2), width, lo);
+        x.w = __fmaf_rn(uniform01(key, 4 * sub + 3), width, lo);
+        quantize_store<BITS, false>(x, s.codes, s.sb, tb.row_base + row, s.dim, sub, lanes, 0u);
+    }
+}
+
+template <int BITS>
+__global__ void k_flush(State s, int t, uint64_t step) {
+    const int lanes = s.lanes;
+    const int sub = threadIdx.x & (lanes - 1);
+    const TableDev tb = s.tables[t];
+    const int64_t nslot = (int64_t)tb.n_sets * s.ways;
+    const int64_t gpb = blockDim.x / lanes, ng = gpb * gridDim.x;
+    for (int64_t i = blockIdx.x * gpb + threadIdx.x / lanes; i < nslot; i += ng) {
+        const int64_t slot = tb.set_base * s.ways + i;
+        const int32_t tag = s.tags[slot];
+        if (tag < 0) continue;
+        const float4 x = reinterpret_cast<const float4*>(s.slab + slot * s.dim)[sub];
+        quantize_store<BITS, true>(x, s.codes, s.sb, tb.row_base + tag, s.dim, sub, lanes,
+                                   rowkey(s.seed, DOMAIN_FLUSH, (uint32_t)t, (uint32_t)tag, step));
+    }
+}
+
+__global__ void k_gather_rows(State s, int t, const int64_t* __restrict__ rows, int64_t n, int code_bytes,
+                              uint8_t* __restrict__ codes, float* __restrict__ scale, float* __restrict__ bias,
+                              uint32_t* __restrict__ cnt, float* __restrict__ G) {
+    const TableDev tb = s.tables[t];
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = rows[i];
+        if (r < 0 || r >= tb.N) continue;
+        const int64_t g = tb.row_base + r;
+        if (codes) {
+            for (int c = 0; c < code_bytes; ++c) codes[i * code_bytes + c] = s.codes[g * code_bytes + c];
+            scale[i] = s.sb[g].x; bias[i] = s.sb[g].y;
+        }
+        if (cnt) cnt[i] = s.cnt ? s.cnt[g] : 0u;
+        if (G) G[i] = s.G ? s.G[g] : 0.0f;
+    }
+}
+
+__global__ void k_fill_i32(int32_t* p, int64_t n, int32_t v) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) p[i] = v;
+}
+
+}  // namespace mpe

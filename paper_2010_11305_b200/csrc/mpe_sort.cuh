@@ -1,0 +1,228 @@
+// Segmented stable LSD radix sort and device-wide prefix sums.
+//
+// The batch's indices arrive grouped by table, so sorting "by (table, row)"
+// (Section 5.1: sort the row indices of the mini-batch, then merge duplicates)
+// only has to order the rows inside each table's segment.  Every pass sorts by
+// an 8-bit digit with per-(table, digit, tile) counters, so one pass over the
+// whole array sorts all segments at once and never moves a key out of its
+// segment.  No kernel here waits on another block: a pass is histogram ->
+// prefix sum -> scatter, three ordinary launches.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mpe {
+
+constexpr int SORT_THREADS = 256;
+constexpr int SORT_ITEMS = 16;
+constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;   // 4096 keys per block
+constexpr int SCAN_THREADS = 256;
+constexpr int SCAN_ITEMS = 16;
+constexpr int SCAN_TILE = SCAN_THREADS * SCAN_ITEMS;
+
+// ---- block-wide exclusive prefix sum of one value per thread -----------------
+template <int THREADS>
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* total, uint32_t* smem /*[THREADS/32 + 1]*/) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t n = __shfl_up_sync(0xffffffffU, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (lane == 31) smem[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = lane < THREADS / 32 ? smem[lane] : 0;
+        uint32_t winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            uint32_t n = __shfl_up_sync(0xffffffffU, winc, o);
+            if (lane >= o) winc += n;
+        }
+        if (lane < THREADS / 32) smem[lane] = winc - w;
+        if (lane == THREADS / 32 - 1) smem[THREADS / 32] = winc;
+    }
+    __syncthreads();
+    const uint32_t r = smem[warp] + inc - v;
+    *total = smem[THREADS / 32];
+    __syncthreads();
+    return r;
+}
+
+// ---- segment -> tile bookkeeping ----------------------------------------------
+// tile_base[t] = number of SORT_TILE-sized tiles of segments 0..t-1; tile_base[T] = total.
+// A non-zero *skip (the step was abandoned) yields zero tiles, which turns the whole sort into a no-op.
+__global__ void k_tile_setup(const int32_t* __restrict__ seg_start, int T, int32_t* __restrict__ tile_base,
+                             uint32_t* __restrict__ hist_len, const uint32_t* __restrict__ skip) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const bool off = *skip != 0;
+        int32_t acc = 0;
+        for (int t = 0; t < T; ++t) {
+            tile_base[t] = acc;
+            int32_t len = off ? 0 : seg_start[t + 1] - seg_start[t];
+            acc += (len + SORT_TILE - 1) / SORT_TILE;
+        }
+        tile_base[T] = acc;
+        *hist_len = (uint32_t)acc * 256u;
+    }
+}
+
+__device__ __forceinline__ int find_segment(const int32_t* __restrict__ base, int T, int32_t v) {
+    // largest t in [0,T) with base[t] <= v  (base non-decreasing, base[0] <= v < base[T])
+    int lo = 0, hi = T;
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (base[mid] <= v) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// ---- pass 1 of 3: per-(table, digit, tile) counts ------------------------------
+__global__ void __launch_bounds__(SORT_THREADS)
+k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base,
+            int T, int shift, uint32_t* __restrict__ hist) {
+    __shared__ uint32_t cnt[256];
+    const int ntiles = tile_base[T];
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int t = find_segment(tile_base, T, tile);
+        const int local = tile - tile_base[t];
+        const int nt = tile_base[t + 1] - tile_base[t];
+        const int32_t start = seg_start[t] + local * SORT_TILE;
+        const int32_t end = min(start + SORT_TILE, seg_start[t + 1]);
+        cnt[threadIdx.x] = 0;
+        __syncthreads();
+        for (int32_t i = start + threadIdx.x; i < end; i += SORT_THREADS)
+            atomicAdd(&cnt[(keys[i] >> shift) & 255u], 1u);
+        __syncthreads();
+        hist[(size_t)256 * tile_base[t] + (size_t)threadIdx.x * nt + local] = cnt[threadIdx.x];
+        __syncthreads();
+    }
+}
+
+// ---- pass 3 of 3: stable scatter ------------------------------------------------
+// vals_in == nullptr means "the payload is the element's position" (first pass).
+__global__ void __launch_bounds__(SORT_THREADS)
+k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
+               uint32_t* __restrict__ keys_out, uint32_t* __restrict__ vals_out,
+               const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base, int T, int shift,
+               const uint32_t* __restrict__ hist_scanned) {
+    constexpr int WARPS = SORT_THREADS / 32;
+    __shared__ uint32_t wcnt[WARPS][256];      // per-warp digit counters, then per-warp digit bases
+    __shared__ uint32_t dstart[256];           // first tile-local position of each digit
+    __shared__ uint32_t gbase[256];            // first global position of each digit of this tile
+    __shared__ uint32_t skey[SORT_TILE];
+    __shared__ uint32_t sval[SORT_TILE];
+    __shared__ uint32_t scan_tmp[SORT_THREADS / 32 + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int ntiles = tile_base[T];
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int t = find_segment(tile_base, T, tile);
+        const int local = tile - tile_base[t];
+        const int nt = tile_base[t + 1] - tile_base[t];
+        const int32_t start = seg_start[t] + local * SORT_TILE;
+        const int32_t count = min(SORT_TILE, seg_start[t + 1] - start);
+        for (int i = threadIdx.x; i < WARPS * 256; i += SORT_THREADS) (&wcnt[0][0])[i] = 0;
+        gbase[threadIdx.x] = hist_scanned[(size_t)256 * tile_base[t] + (size_t)threadIdx.x * nt + local];
+        __syncthreads();
+        // warp w owns elements [w*512, w*512+512) of the tile, item i of lane l is w*512 + i*32 + l,
+        // so "item order, then lane order" is the original order
+        uint32_t key[SORT_ITEMS], val[SORT_ITEMS], rank[SORT_ITEMS];
+#pragma unroll
+        for (int i = 0; i < SORT_ITEMS; ++i) {
+            const int e = warp * (32 * SORT_ITEMS) + i * 32 + lane;
+            const bool ok = e < count;
+            key[i] = ok ? keys_in[start + e] : 0xffffffffU;
+            val[i] = ok ? (vals_in ? vals_in[start + e] : (uint32_t)(start + e)) : 0u;
+            const uint32_t dg = (key[i] >> shift) & 255u;
+            const uint32_t peers = __match_any_sync(0xffffffffU, dg);
+            const uint32_t before = wcnt[warp][dg];
+            __syncwarp();
+            if ((peers & ((1u << lane) - 1u)) == 0) wcnt[warp][dg] = before + __popc(peers);
+            __syncwarp();
+            rank[i] = before + __popc(peers & ((1u << lane) - 1u));
+        }
+        __syncthreads();
+        // digit d (= threadIdx.x): exclusive sum over warps, then over digits
+        uint32_t tot = 0;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) { uint32_t c = wcnt[w][threadIdx.x]; wcnt[w][threadIdx.x] = tot; tot += c; }
+        uint32_t all;
+        const uint32_t ds = block_exclusive_scan<SORT_THREADS>(tot, &all, scan_tmp);
+        dstart[threadIdx.x] = ds;
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < SORT_ITEMS; ++i) {
+            const uint32_t dg = (key[i] >> shift) & 255u;
+            const uint32_t pos = dstart[dg] + wcnt[warp][dg] + rank[i];
+            skey[pos] = key[i];
+            sval[pos] = val[i];
+        }
+        __syncthreads();
+        // padding keys (0xffffffff, digit 255) follow every real key of the tile, so positions [0,count) are real
+        for (int j = threadIdx.x; j < count; j += SORT_THREADS) {
+            const uint32_t k = skey[j];
+            const uint32_t dg = (k >> shift) & 255u;
+            const uint32_t dst = gbase[dg] + ((uint32_t)j - dstart[dg]);
+            keys_out[dst] = k;
+            vals_out[dst] = sval[j];
+        }
+        __syncthreads();
+    }
+}
+
+// ---- device-wide exclusive prefix sum over uint32 (length read from device memory) ------------
+__global__ void __launch_bounds__(SCAN_THREADS)
+k_scan_reduce(const uint32_t* __restrict__ in, const uint32_t* __restrict__ n_ptr, uint32_t* __restrict__ block_sums) {
+    __shared__ uint32_t tmp[SCAN_THREADS / 32 + 1];
+    const uint32_t n = *n_ptr;
+    const uint32_t nblk = (n + SCAN_TILE - 1) / SCAN_TILE;
+    for (uint32_t b = blockIdx.x; b < nblk; b += gridDim.x) {
+        uint32_t s = 0;
+        const uint32_t base = b * SCAN_TILE + threadIdx.x * SCAN_ITEMS;
+#pragma unroll
+        for (int i = 0; i < SCAN_ITEMS; ++i) if (base + i < n) s += in[base + i];
+        uint32_t total;
+        block_exclusive_scan<SCAN_THREADS>(s, &total, tmp);
+        if (threadIdx.x == 0) block_sums[b] = total;
+    }
+}
+
+// one block: exclusive scan of block_sums[0..nblk) in place; the grand total goes to *total_out
+__global__ void __launch_bounds__(1024)
+k_scan_block_sums(uint32_t* __restrict__ block_sums, const uint32_t* __restrict__ n_ptr, uint32_t tile,
+                  uint32_t* __restrict__ total_out) {
+    __shared__ uint32_t tmp[1024 / 32 + 1];
+    const uint32_t n = *n_ptr;
+    const uint32_t nblk = (n + tile - 1) / tile;
+    uint32_t carry = 0;
+    for (uint32_t base = 0; base < nblk; base += 1024) {
+        const uint32_t i = base + threadIdx.x;
+        const uint32_t v = i < nblk ? block_sums[i] : 0;
+        uint32_t total;
+        const uint32_t ex = block_exclusive_scan<1024>(v, &total, tmp);
+        if (i < nblk) block_sums[i] = carry + ex;
+        carry += total;
+    }
+    if (threadIdx.x == 0 && total_out) *total_out = carry;
+}
+
+__global__ void __launch_bounds__(SCAN_THREADS)
+k_scan_apply(uint32_t* __restrict__ data, const uint32_t* __restrict__ n_ptr, const uint32_t* __restrict__ block_sums) {
+    __shared__ uint32_t tmp[SCAN_THREADS / 32 + 1];
+    const uint32_t n = *n_ptr;
+    const uint32_t nblk = (n + SCAN_TILE - 1) / SCAN_TILE;
+    for (uint32_t b = blockIdx.x; b < nblk; b += gridDim.x) {
+        uint32_t v[SCAN_ITEMS];
+        uint32_t s = 0;
+        const uint32_t base = b * SCAN_TILE + threadIdx.x * SCAN_ITEMS;
+#pragma unroll
+        for (int i = 0; i < SCAN_ITEMS; ++i) { v[i] = base + i < n ? data[base + i] : 0; s += v[i]; }
+        uint32_t total;
+        uint32_t ex = block_exclusive_scan<SCAN_THREADS>(s, &total, tmp) + block_sums[b];
+#pragma unroll
+        for (int i = 0; i < SCAN_ITEMS; ++i) { if (base + i < n) data[base + i] = ex; ex += v[i]; }
+    }
+}
+
+}  // namespace mpe

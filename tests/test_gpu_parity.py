@@ -1,0 +1,268 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle
+on the same seeded inputs.  Integer state (codes, tags, timestamps, counters,
+statistics) and the FP32 scale/bias/cached rows must be bit-equal; pooled
+outputs must be within 1e-5 of the sum of absolute terms (they are bit-equal
+too, because both sides add in index order)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2010_11305_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_cuda():
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device; run them with -m gpu on a GPU box")
+
+
+def _cfg(**kw):
+    base = dict(name="t", num_rows=[1000], dim=16, bits=8, cache_fraction=0.05, ways=8, policy=wl.LRU, optimizer=wl.SGD,
+                lr=0.05, batch=64, bag=("fixed", 4), zipf=[1.05], steps=4, seed=1)
+    base.update(kw)
+    return wl.Config(**base)
+
+
+def test_config1_all_steps():
+    from parity_util import run_parity
+    cfg = wl.config(1)
+    h, o, info = run_parity(cfg, cfg.steps)
+    assert info[0][0] == 512 and 0 < info[0][1] <= 512
+
+
+def test_config2_lfu_many_tables():
+    from parity_util import run_parity
+    cfg = wl.config(2)
+    run_parity(cfg, 12, check_every=4)
+
+
+@pytest.mark.parametrize("bits,policy,opt,ways,dim", [
+    (8, wl.LRU, wl.SGD, 8, 16), (4, wl.LRU, wl.ROWWISE_ADAGRAD, 16, 64), (4, wl.LFU, wl.SGD, 32, 128),
+    (8, wl.LFU, wl.ROWWISE_ADAGRAD, 32, 64), (4, wl.LFU, wl.SGD, 2, 32), (8, wl.LRU, wl.SGD, 1, 8),
+    (4, wl.LFU, wl.SGD, 1, 4), (8, wl.LRU, wl.SGD, 4, 128),
+])
+def test_small_tables_every_variant(bits, policy, opt, ways, dim):
+    """Small tables with a skewed stream: many hits, admissions, evictions, bypasses and chains per step."""
+    from parity_util import run_parity
+    cfg = _cfg(num_rows=[3000, 500, 7], dim=dim, bits=bits, policy=policy, optimizer=opt, ways=ways, cache_fraction=0.1,
+               batch=96, bag=("poisson", 6.0), zipf=[1.1, 0.9, None], steps=8, seed=bits + ways)
+    h, o, _ = run_parity(cfg, 8)
+    s = h.stats(0)
+    assert s[3] > 0 and s[4] > 0 and s[5] > 0 and s[6] > 0     # hits, admissions, evictions, bypasses all occurred
+
+
+def test_config3_scaled_and_ragged():
+    from parity_util import run_parity
+    cfg = wl.scaled(wl.config(3), rows_div=100, batch_div=8, steps=6)
+    run_parity(cfg, 6, check_every=2)
+
+
+def test_config4_scaled_hot_rows():
+    """Poisson bags capped at 100, per-table skew, LFU, INT4 d=128; the hottest rows exceed 1024 occurrences."""
+    from parity_util import run_parity
+    cfg = wl.scaled(wl.config(4), rows_div=50, batch_div=8, tables=6, steps=4)
+    h, o, info = run_parity(cfg, 4, check_every=2)
+    assert info[0][3] > 0        # rows that needed the multi-block gradient tree
+
+
+def test_config5_points():
+    from parity_util import run_parity
+    pts = list(wl.sweep5())
+    for cfg in (pts[2], pts[len(pts) // 2 + 5], pts[-1]):
+        cfg = wl.scaled(cfg, rows_div=20, batch_div=4, steps=4)
+        run_parity(cfg, 4, check_every=2)
+
+
+def test_no_cache_is_pure_low_precision_training():
+    from parity_util import run_parity
+    run_parity(_cfg(cache_fraction=0.0, bits=4, dim=32), 4)
+
+
+def test_very_hot_row_uses_three_tree_levels():
+    """One row with > 32768 occurrences in a batch: partial sums of 1024, then of 32768, then the rest."""
+    from parity_util import make_pair, compare_state
+    cfg = _cfg(num_rows=[50], dim=8, batch=40000, bag=("fixed", 1), zipf=[3.0], cache_fraction=0.2, ways=2)
+    h, o = make_pair(cfg)
+    st = wl.Stream(cfg, "cpu")
+    rng = np.random.default_rng(0)
+    for step in (1, 2):
+        idx, off, grad = st.batch(step)
+        assert np.bincount(idx.numpy()).max() > 32768
+        out = torch.empty(cfg.batch, cfg.dim, device="cuda")
+        h.forward(idx.cuda(), off.cuda(), cfg.batch, out)
+        ref = o.forward(idx.numpy(), off.numpy(), cfg.batch)
+        assert np.array_equal(out.cpu().numpy(), ref)
+        h.backward(grad.cuda(), 0.01, step)
+        o.backward(grad.numpy(), 0.01, step)
+        compare_state(h, o, cfg, [0], rng)
+
+
+def test_empty_bags_empty_batch_and_duplicates_inside_a_bag():
+    from parity_util import make_pair, compare_state
+    cfg = _cfg(num_rows=[40, 40], dim=16, batch=5, cache_fraction=0.25, ways=2)
+    h, o = make_pair(cfg)
+    rng = np.random.default_rng(0)
+    bags = [[[1, 1, 1], [], [2, 3, 2], [], []], [[], [], [], [], []]]
+    idx = np.array([r for tb in bags for bag in tb for r in bag], np.int32)
+    off = np.cumsum([0] + [len(bag) for tb in bags for bag in tb]).astype(np.int32)
+    grad = rng.normal(0, 0.1, (5, 32)).astype(np.float32)
+    out = torch.full((5, 32), 7.0, device="cuda")
+    h.forward(torch.tensor(idx).cuda(), torch.tensor(off).cuda(), 5, out)
+    ref = o.forward(idx, off, 5)
+    assert np.array_equal(out.cpu().numpy(), ref) and np.all(ref[1] == 0) and np.all(ref[:, 16:] == 0)
+    h.backward(torch.tensor(grad).cuda(), 0.1, 1)
+    o.backward(grad, 0.1, 1)
+    compare_state(h, o, cfg, [0, 1], rng)
+    # a batch with no index at all
+    off0 = np.zeros(11, np.int32)
+    out = torch.full((5, 32), 7.0, device="cuda")
+    h.forward(torch.zeros(0, dtype=torch.int32, device="cuda"), torch.tensor(off0).cuda(), 5, out)
+    o.forward(np.zeros(0, np.int32), off0, 5)
+    assert torch.all(out == 0)
+    h.backward(torch.tensor(grad).cuda(), 0.1, 2)
+    o.backward(grad, 0.1, 2)
+    compare_state(h, o, cfg, [0, 1], rng)
+    assert h.last_error() == (0, 0)
+
+
+def test_out_of_range_indices_are_dropped_and_reported():
+    from parity_util import make_pair, compare_state
+    from paper_2010_11305_b200 import binding as mpe
+    cfg = _cfg(num_rows=[100, 30], dim=8, batch=4, cache_fraction=0.2, ways=4)
+    h, o = make_pair(cfg)
+    rng = np.random.default_rng(1)
+    idx = np.array([5, 100, 7, -1, 5, 99, 2 ** 31 - 1, 0, 29, 30, 3, 3, -7, 12], np.int32)
+    off = np.array([0, 2, 4, 6, 8, 10, 12, 13, 14], np.int32)
+    grad = rng.normal(0, 0.1, (4, 16)).astype(np.float32)
+    for step in (1, 2):
+        out = torch.empty(4, 16, device="cuda")
+        h.forward(torch.tensor(idx).cuda(), torch.tensor(off).cuda(), 4, out)
+        ref = o.forward(idx, off, 4)
+        assert np.array_equal(out.cpu().numpy(), ref)
+        info = h.step_info()
+        assert info[0] == 9 and info[2] == 5 and info[1] == 7
+        h.backward(torch.tensor(grad).cuda(), 0.1, step)
+        o.backward(grad, 0.1, step)
+        assert h.last_error() == (mpe.ERR_INDEX, 5)
+        assert h.last_error() == (0, 0)
+        compare_state(h, o, cfg, [0, 1], rng)
+    assert o.dropped() == 10
+
+
+def test_bad_offsets_are_refused_without_touching_state():
+    from parity_util import make_pair, compare_state
+    from paper_2010_11305_b200 import binding as mpe
+    cfg = _cfg(num_rows=[100], dim=8, batch=4)
+    h, o = make_pair(cfg)
+    rng = np.random.default_rng(1)
+    idx = torch.tensor([1, 2, 3, 4, 5, 6], dtype=torch.int32).cuda()
+    grad = torch.ones(4, 8, device="cuda")
+    for step, bad in enumerate(([0, 2, 1, 4, 6], [1, 2, 3, 4, 6], [0, 2, 3, 4, 5], [0, 2, 9, 4, 6], [0, -2, 3, 4, 6]), start=1):
+        out = torch.full((4, 8), 3.0, device="cuda")
+        h.forward(idx, torch.tensor(bad, dtype=torch.int32).cuda(), 4, out)
+        if step % 2:
+            h.backward(grad, 0.1, step)        # the abandoned step's backward must be a no-op too
+        code, detail = h.last_error()
+        assert code == mpe.ERR_OFFSETS and detail >= 1
+        assert torch.all(out == 0)
+    rows = np.arange(100)
+    codes, scale, bias = h.export_rows(0, rows)
+    rc, rs, rb = o.rows(0, rows)
+    assert np.array_equal(codes, rc) and np.array_equal(scale, rs) and np.array_equal(bias, rb)
+    assert np.all(h.export_cache(0)[0] == -1) and np.all(h.stats(0)[:7] == 0)
+    # and the handle still works afterwards
+    good = torch.tensor([0, 2, 3, 4, 6], dtype=torch.int32).cuda()
+    out = torch.empty(4, 8, device="cuda")
+    h.forward(idx, good, 4, out)
+    ref = o.forward(idx.cpu().numpy(), good.cpu().numpy(), 4)
+    assert np.array_equal(out.cpu().numpy(), ref)
+    h.backward(grad, 0.1, 10)
+    o.backward(grad.cpu().numpy(), 0.1, 10)
+    assert h.last_error() == (0, 0)
+    tags, crow, ts = h.export_cache(0)
+    otags, ocrow, ots = o.cache(0)
+    assert np.array_equal(tags, otags) and np.array_equal(crow, ocrow) and np.array_equal(ts, ots)
+    del rng, compare_state
+
+
+def test_sequence_and_argument_errors():
+    from paper_2010_11305_b200 import binding as mpe
+    with pytest.raises(mpe.MpeError) as e:
+        mpe.Mpe([100], 12, 8, 0.1, 8, mpe.LRU)
+    assert e.value.code == mpe.ERR_UNSUPPORTED
+    with pytest.raises(mpe.MpeError):
+        mpe.Mpe([100], 16, 3, 0.1, 8, mpe.LRU)
+    with pytest.raises(mpe.MpeError):
+        mpe.Mpe([100], 16, 8, 0.1, 6, mpe.LRU)
+    with pytest.raises(mpe.MpeError):
+        mpe.Mpe([100], 16, 8, 1.5, 8, mpe.LRU)
+    h = mpe.Mpe([100], 16, 8, 0.1, 8, mpe.LRU)
+    g = torch.zeros(2, 16, device="cuda")
+    with pytest.raises(mpe.MpeError) as e:
+        h.backward(g, 0.1, 1)
+    assert e.value.code == mpe.ERR_SEQUENCE
+    idx = torch.tensor([1, 2], dtype=torch.int32).cuda()
+    off = torch.tensor([0, 1, 2], dtype=torch.int32).cuda()
+    out = torch.empty(2, 16, device="cuda")
+    h.forward(idx, off, 2, out)
+    h.backward(g, 0.1, 5)
+    h.forward(idx, off, 2, out)
+    with pytest.raises(mpe.MpeError) as e:
+        h.backward(g, 0.1, 5)          # step must increase
+    assert e.value.code == mpe.ERR_SEQUENCE
+    h.backward(g, 0.1, 6)
+
+
+def test_step_is_deterministic_and_forward_is_read_only():
+    from paper_2010_11305_b200 import binding as mpe
+    cfg = wl.scaled(wl.config(4), rows_div=100, batch_div=16, tables=3)
+    st = wl.Stream(cfg, "cpu")
+    results = []
+    for rep in range(2):
+        h = mpe.Mpe(cfg.num_rows, cfg.dim, cfg.bits, cfg.cache_fraction, cfg.ways, cfg.policy, seed=cfg.seed)
+        for step in (1, 2, 3):
+            idx, off, grad = (x.cuda() for x in st.batch(step))
+            out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, device="cuda")
+            h.forward(idx, off, cfg.batch, out)
+            out2 = torch.empty_like(out)
+            h.forward(idx, off, cfg.batch, out2)       # a second forward sees the same state
+            assert torch.equal(out, out2)
+            h.backward(grad, cfg.lr, step)
+        rows = np.arange(0, cfg.num_rows[0], 3)
+        results.append((h.export_rows(0, rows), h.export_cache(0), out.cpu().numpy()))
+    (r0, c0, o0), (r1, c1, o1) = results
+    assert all(np.array_equal(a, b) for a, b in zip(r0, r1))
+    assert all(np.array_equal(a, b) for a, b in zip(c0, c1))
+    assert np.array_equal(o0, o1)
+
+
+def test_host_buffer_step_matches_device_step():
+    from parity_util import make_pair, compare_state
+    cfg = _cfg(num_rows=[2000, 300], dim=32, bits=4, batch=64, zipf=[1.05, 1.2], policy=wl.LFU, ways=4)
+    h, o = make_pair(cfg)
+    st = wl.Stream(cfg, "cpu")
+    rng = np.random.default_rng(0)
+    for step in (1, 2, 3):
+        idx, off, grad = st.batch(step)
+        out = np.zeros((cfg.batch, cfg.num_tables * cfg.dim), np.float32)
+        h.step_host(idx.numpy(), off.numpy(), cfg.batch, grad.numpy(), out, cfg.lr, step)
+        ref = o.forward(idx.numpy(), off.numpy(), cfg.batch)
+        o.backward(grad.numpy(), cfg.lr, step)
+        assert np.array_equal(out, ref)
+    compare_state(h, o, cfg, [0, 1], rng)
+
+
+def test_memory_accounting_matches_the_appendix_table():
+    import os
+    from paper_2010_11305_b200 import binding as mpe
+    rows = [l.split() for l in open(os.path.join(os.path.dirname(__file__), "golden", "compression_factor_table.txt"))
+            if not l.startswith("#")]
+    for bits, ratio, factor in rows:
+        if int(bits) == 2:
+            continue
+        h = mpe.Mpe([320_000], 128, int(bits), float(ratio), 32, mpe.LFU)
+        m = h.memory_bytes().astype(np.float64)
+        assert abs((m[0] + m[1] + m[2] + m[3]) / m[5] - float(factor)) < 6e-6
+        h.close()
