@@ -1,0 +1,326 @@
+"""Benchmark of the cached mixed-precision embedding training step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl ours|reference]
+
+One "step" is mpe_forward + mpe_backward over one batch of the chosen
+configuration (default: configuration 4, the largest one, 64 tables x 5M rows x
+dim 128, packed INT4, 1% FP32 cache, LFU).  Inputs are seeded synthetic Zipf
+streams generated on the device before the timed region (every batch is far
+larger than L2).  Timing uses CUDA events on the stream the kernels are launched
+on.  With N > 1 (torchrun) every rank trains its own shard of tables of the
+same size (weak scaling, no data-path collective) and rank 0 reports the
+aggregate.  Prints ONE JSON line.
+
+--impl reference times the CPU oracle (oracle/) on the host cores on a bounded
+sample of the same workload.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+from paper_2010_11305_b200 import workloads as wl  # noqa: E402
+
+METRIC = "embedding rows/sec per training step (fwd+bwd+cache) and % of 8 TB/s HBM"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, gpu_index):
+        self.q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+                  "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def describe(cfg):
+    pol = "LFU" if cfg.policy == wl.LFU else "LRU"
+    opt = "row-wise Adagrad" if cfg.optimizer == wl.ROWWISE_ADAGRAD else "SGD"
+    return (f"{cfg.name}: {cfg.num_tables} tables x {max(cfg.num_rows):,} rows x dim {cfg.dim}, INT{cfg.bits} row-wise, "
+            f"cache {cfg.cache_fraction:g} x rows, {cfg.ways or 32}-way {pol}, batch {cfg.batch}, bags {cfg.bag}, {opt}")
+
+
+def byte_model(cfg, L, U, U_hit, occ_hit, admissions, evictions, passes_main, passes_cand):
+    """Algorithmic bytes of one step, per kernel (what the method itself has to move, counted per access)."""
+    d, T, B = cfg.dim, cfg.num_tables, cfg.batch
+    rb = d * cfg.bits // 8 + 8      # codes + FP32 scale + FP32 bias
+    fb = 4 * d
+    occ_miss, U_miss = L - occ_hit, U - U_hit
+    out_bytes = 4 * B * T * d
+    m = {}
+    m["make_keys"] = 4 * L + 4 * T * B + 8 * L
+    m["sort_hist"] = passes_main * 4 * L + passes_cand * 4 * U
+    m["sort_scatter"] = passes_main * 16 * L + passes_cand * 16 * U
+    m["unique_count"] = 4 * L
+    m["unique_write"] = 8 * L + 12 * U
+    m["probe"] = 8 * U + 4 * cfg.ways * U + 12 * U
+    m["broadcast"] = 20 * L
+    m["pool"] = 8 * L + occ_hit * fb + occ_miss * rb + out_bytes
+    m["priority"] = 16 * U + (8 * U if cfg.policy == wl.LFU else 4 * U_hit) + 8 * U
+    m["policy"] = U_miss * (8 + 4 + (4 if cfg.policy == wl.LFU else 0) + 8) + admissions * 8 * cfg.ways
+    grad_bytes = L * (fb + 4)
+    m["update"] = grad_bytes + 28 * U + U_hit * 2 * fb + (U_miss - admissions) * 2 * rb
+    m["update_admit"] = 8 * U + admissions * (rb + fb) + evictions * (fb + rb)
+    if cfg.optimizer == wl.ROWWISE_ADAGRAD:
+        m["update"] += 8 * U
+    return m
+
+
+def run_ours(args, cfg, rank, world, local_rank):
+    from paper_2010_11305_b200 import binding as mpe
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    # every rank owns its own shard of tables (same shapes, different seed): weak scaling
+    cfg.seed = cfg.seed + 7919 * rank
+    stream_gen = wl.Stream(cfg, dev)
+    h = mpe.Mpe(cfg.num_rows, cfg.dim, cfg.bits, cfg.cache_fraction, cfg.ways, cfg.policy, cfg.optimizer, cfg.eps,
+                cfg.init_lo, cfg.init_hi, cfg.seed, local_rank)
+    n_e2e = min(args.steps, args.e2e_steps)
+    total_steps = args.warmup + args.steps + n_e2e
+    batches = [stream_gen.batch(s) for s in range(1, total_steps + 1)]
+    maxL = max(b[0].numel() for b in batches)
+    h.reserve(cfg.batch, maxL)
+    out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, dtype=torch.float32, device=dev)
+    cs = torch.cuda.current_stream(dev)
+    sp = cs.cuda_stream
+
+    def step(i):
+        idx, off, grad = batches[i]
+        h.forward(idx, off, cfg.batch, out, sp)
+        h.backward(grad, cfg.lr, i + 1)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize(dev)
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    stats0 = np.sum([h.stats(t) for t in range(cfg.num_tables)], axis=0).astype(np.int64)
+    launches0 = h.kernel_launches()
+    h.profile(True)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(cs)
+    for i in range(args.warmup, args.warmup + args.steps):
+        step(i)
+    e1.record(cs)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    prof = h.profile_read()
+    h.profile(False)
+    launches = h.kernel_launches() - launches0
+    stats1 = np.sum([h.stats(t) for t in range(cfg.num_tables)], axis=0).astype(np.int64)
+    code, detail = h.last_error()
+    assert code == 0, f"device error {code} ({detail})"
+    ds = stats1 - stats0
+    K = args.steps
+    L, occ_hit, U, U_hit, adm, evi = (ds[i] / K for i in (0, 1, 2, 3, 4, 5))
+
+    # end to end through the host-buffer entry point: pinned host inputs, H2D + step + D2H inside the timed region
+    h_batches = []
+    for i in range(args.warmup + args.steps, total_steps):
+        idx, off, grad = batches[i]
+        h_batches.append((idx.cpu().pin_memory(), off.cpu().pin_memory(), grad.cpu().pin_memory()))
+    h_out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, dtype=torch.float32).pin_memory()
+    barrier()
+    t0 = time.perf_counter()
+    e2e_rows = 0
+    for j, (idx, off, grad) in enumerate(h_batches):
+        h.step_host(idx, off, cfg.batch, grad, h_out, cfg.lr, args.warmup + args.steps + j + 1)
+        e2e_rows += idx.numel()
+    torch.cuda.synchronize(dev)
+    e2e_s = time.perf_counter() - t0
+    h2d = float(np.mean([(a.numel() + b.numel() + c.numel()) * 4 for a, b, c in h_batches])) if h_batches else 0.0
+    d2h = float(h_out.numel() * 4)
+
+    # aggregate over ranks: total rows / max time
+    rows_timed = float(ds[0])
+    if world > 1:
+        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device=dev)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        r = torch.tensor([rows_timed, float(e2e_rows)], dtype=torch.float64, device=dev)
+        torch.distributed.all_reduce(r, op=torch.distributed.ReduceOp.SUM)
+        ms, e2e_s = float(t[0]), float(t[1])
+        rows_timed, e2e_rows = float(r[0]), float(r[1])
+    if rank != 0:
+        return None
+
+    passes_main = (max(cfg.num_rows).bit_length() + 7) // 8
+    max_sets = max(h.cache_geometry(t)[0] for t in range(cfg.num_tables))
+    passes_cand = (max(max_sets, 1).bit_length() + 7) // 8 if max_sets else 0
+    model = byte_model(cfg, L, U, U_hit, occ_hit, adm, evi, passes_main, passes_cand)
+    step_bytes = float(sum(model.values()))
+    ms_step = ms / K
+    top = max(prof.items(), key=lambda kv: kv[1][0]) if prof else (None, (0.0, 0))
+    peak, peak_kind = measured_peaks()
+    roof = None
+    if top[0] is not None:
+        name, (tms, n) = top
+        per_launch_ms = tms / n
+        launches_per_step = n / K
+        bytes_per_launch = model.get(name, 0.0) / max(launches_per_step, 1e-9)
+        achieved = bytes_per_launch / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms > 0 else 0.0
+        roof = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None, "bytes_per_launch": bytes_per_launch, "ms_per_launch": per_launch_ms,
+                "share_of_step": tms / ms}
+    result = {
+        "metric": METRIC, "value": rows_timed / (ms * 1e-3), "unit": "rows/s", "n_gpus": world, "steps": K,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": describe(cfg), "l2": "inputs larger than L2; a new batch every step",
+                   "sharding": "each rank trains its own tables (no data-path collective)" if world > 1 else "one GPU"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_rows / e2e_s if e2e_s > 0 else None, "unit": "rows/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": len(h_batches)},
+        "gpu_launches": int(launches),
+        "roofline": roof,
+        "effective": {"bytes_per_step": step_bytes, "gbs": step_bytes / (ms_step * 1e-3) / 1e9,
+                      "frac_of_8TBs": step_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                      "frac_of_measured_copy": step_bytes / (ms_step * 1e-3) / 1e9 / peak},
+        "per_step": {"indices": L, "distinct_rows": U, "distinct_hits": U_hit, "index_hit_rate": occ_hit / max(L, 1),
+                     "admissions": adm, "evictions": evi},
+        "kernels_ms_per_step": {k: v[0] / K for k, v in sorted(prof.items(), key=lambda kv: -kv[1][0])},
+    }
+    return result
+
+
+def sample_tables(cfg, budget_rows):
+    """How many tables of the configuration the CPU oracle can process in the time budget (~10-30 s)."""
+    per_table = cfg.batch * (cfg.bag[1] if cfg.bag[0] != "fixed" else cfg.bag[1])
+    n = int(max(1, min(cfg.num_tables, budget_rows // max(per_table, 1))))
+    return list(range(n))
+
+
+def run_oracle(cfg, steps, warmup, stream_device, budget_rows=3_000_000):
+    """The CPU oracle, as it stands, on the host cores: `steps` steps over a sample of the tables."""
+    from oracle import mpe_oracle as orc
+    tables = sample_tables(cfg, budget_rows // max(steps + warmup, 1))
+    o = orc.Oracle(cfg.num_rows, cfg.dim, cfg.bits, cfg.cache_fraction, cfg.ways, cfg.policy, cfg.optimizer, cfg.eps,
+                   cfg.init_lo, cfg.init_hi, cfg.seed)
+    mask = np.zeros(cfg.num_tables, np.uint8)
+    mask[tables] = 1
+    o.set_table_mask(mask)
+    st = wl.Stream(cfg, stream_device)
+    rows, secs = 0, 0.0
+    for s in range(1, warmup + steps + 1):
+        idx, off, grad = (x.cpu().numpy() for x in st.batch(s))
+        t0 = time.perf_counter()
+        o.forward(idx, off, cfg.batch)
+        o.backward(grad, cfg.lr, s)
+        dt = time.perf_counter() - t0
+        if s > warmup:
+            secs += dt
+            rows += int(sum(off[(t + 1) * cfg.batch] - off[t * cfg.batch] for t in tables))
+    return {"value": rows / secs if secs > 0 else None, "unit": "rows/s", "cores": 1, "kind": "oracle",
+            "sample": f"{len(tables)} of {cfg.num_tables} tables, {steps} step(s) after {warmup} warm-up, "
+                      f"{rows} index rows in {secs:.1f} s; untouched rows are materialised on first use",
+            "seconds": secs, "rows": rows}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=4)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg = wl.config(args.config)
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        dev = "cuda" if torch.cuda.is_available() else "cpu"
+        r = run_oracle(cfg, args.steps, min(args.warmup, 1), dev, budget_rows=2_000_000)
+        line = {"metric": METRIC, "impl": "reference", "value": r["value"], "unit": "rows/s", "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * r["seconds"] / max(args.steps, 1),
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": describe(cfg)},
+                "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+                "e2e": {"value": r["value"], "unit": "rows/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    result = run_ours(args, cfg, rank, world, local_rank)
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            cfg0 = wl.config(args.config)
+            r = run_oracle(cfg0, 1, 0, torch.device("cuda", local_rank))
+            result["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        print(json.dumps(result))
+    if world > 1:
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
