@@ -284,12 +284,21 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tables", type=int, default=None, help="profiling aid: keep only the first TABLES tables")
+    ap.add_argument("--rows-div", type=int, default=1, help="profiling aid: divide every table's row count")
+    ap.add_argument("--batch-div", type=int, default=1, help="profiling aid: divide the batch size")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    cfg = wl.config(args.config)
+    def make_cfg():
+        c = wl.config(args.config)
+        if args.tables is not None or args.rows_div != 1 or args.batch_div != 1:
+            c = wl.scaled(c, rows_div=args.rows_div, batch_div=args.batch_div, tables=args.tables)
+        return c
+
+    cfg = make_cfg()
 
     if args.impl == "reference":
         if rank != 0:
@@ -313,7 +322,7 @@ def main():
     result = run_ours(args, cfg, rank, world, local_rank)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            cfg0 = wl.config(args.config)
+            cfg0 = make_cfg()
             r = run_oracle(cfg0, 1, 0, torch.device("cuda", local_rank))
             result["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
         print(json.dumps(result))
