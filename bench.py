@@ -111,8 +111,7 @@ def byte_model(cfg, L, U, U_hit, occ_hit, admissions, evictions, passes_main, pa
     m["priority"] = 16 * U + (8 * U if cfg.policy == wl.LFU else 4 * U_hit) + 8 * U
     m["policy"] = U_miss * (8 + 4 + (4 if cfg.policy == wl.LFU else 0) + 8) + admissions * 8 * cfg.ways
     grad_bytes = L * (fb + 4)
-    m["update"] = grad_bytes + 28 * U + U_hit * 2 * fb + (U_miss - admissions) * 2 * rb
-    m["update_admit"] = 8 * U + admissions * (rb + fb) + evictions * (fb + rb)
+    m["update"] = grad_bytes + 32 * U + U_hit * 2 * fb + (U_miss - admissions) * 2 * rb + admissions * (rb + fb) + evictions * (fb + rb)
     if cfg.optimizer == wl.ROWWISE_ADAGRAD:
         m["update"] += 8 * U
     return m

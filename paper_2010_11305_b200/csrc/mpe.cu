@@ -10,6 +10,7 @@
 #include <cstring>
 #include <map>
 #include <string>
+#include <type_traits>
 #include <vector>
 
 using namespace mpe;
@@ -133,7 +134,7 @@ int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
     A(w.uniq_row, n); A(w.uniq_t, n); A(w.seg, n + 1); A(w.loc, n); A(w.final_loc, n); A(w.victim, n);
     A(w.hot_base, n); A(w.uset, n);
     const int64_t max_tasks = L / (HOT_SPAN / 2) + 2;
-    A(w.task_k, max_tasks); A(w.partial, max_tasks * h->dim);
+    A(w.task_k, max_tasks); A(w.partial, max_tasks * h->dim); A(w.hot_k, L / HOT_SPAN + 2); A(w.defer_k, n);
 #undef A
     CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), h->stream));
     h->cap_L = L; h->cap_bags = bags;
@@ -167,6 +168,23 @@ int seg_sort(mpe_handle* h, uint32_t* kA, uint32_t* kB, uint32_t* vA, uint32_t* 
         vin = vout; vout = (vout == vB) ? vA : vB;
     }
     return (passes & 1) ? 1 : 0;
+}
+
+// call f(integral_constant<BITS>, integral_constant<LANES>) for the handle's code width and lanes per row
+template <class F>
+void dispatch(int bits, int lanes, F&& f) {
+    auto by_lanes = [&](auto bc) {
+        switch (lanes) {
+            case 1: f(bc, std::integral_constant<int, 1>{}); break;
+            case 2: f(bc, std::integral_constant<int, 2>{}); break;
+            case 4: f(bc, std::integral_constant<int, 4>{}); break;
+            case 8: f(bc, std::integral_constant<int, 8>{}); break;
+            case 16: f(bc, std::integral_constant<int, 16>{}); break;
+            default: f(bc, std::integral_constant<int, 32>{}); break;
+        }
+    };
+    if (bits == 8) by_lanes(std::integral_constant<int, 8>{});
+    else by_lanes(std::integral_constant<int, 4>{});
 }
 
 int check_launch(mpe_handle* h) {
@@ -322,8 +340,10 @@ int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offset
     LAUNCH(h, "probe", k_probe, grid_for(h, total_indices, 256 / s.ways, 8), 256, 0, s, w, h->epoch);
     LAUNCH(h, "broadcast", k_broadcast, grid_for(h, total_indices, 256, 8), 256, 0, s, w, h->spos, batch);
     const int gp = grid_for(h, bags, 256 / s.lanes, 8);
-    if (h->bits == 8) LAUNCH(h, "pool", k_pool<8>, gp, 256, 0, s, w, d_indices, d_offsets, batch, d_out);
-    else LAUNCH(h, "pool", k_pool<4>, gp, 256, 0, s, w, d_indices, d_offsets, batch, d_out);
+    dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
+        auto kern = k_pool<decltype(bc)::value, decltype(lc)::value>;
+        LAUNCH(h, "pool", kern, gp, 256, 0, s, w, d_indices, d_offsets, batch, d_out);
+    });
     int rc = check_launch(h);
     if (rc != MPE_OK) return rc;
     h->have_forward = true;
@@ -350,12 +370,21 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
         const uint32_t* cv = which ? h->cvalB : h->cvalA;
         LAUNCH(h, "policy", k_policy, grid_for(h, L, 256 / s.ways, 8), 256, 0, s, w, ck, cv, (uint32_t)step, h->epoch);
     }
-    LAUNCH(h, "hot_partial", k_hot_partial, grid_for(h, L / HOT_SPAN + 1, 1, 4), 256, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
-    const int gu = grid_for(h, L, 256 / s.lanes, 8);
-    for (int phase = 1; phase <= (h->max_sets > 0 ? 2 : 1); ++phase) {
-        if (h->bits == 8) LAUNCH(h, phase == 1 ? "update" : "update_admit", k_update<8>, gu, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step, phase);
-        else LAUNCH(h, phase == 1 ? "update" : "update_admit", k_update<4>, gu, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step, phase);
-    }
+    const int gu = grid_for(h, (L + 31) / 32, 8, 3);
+    const int gh = grid_for(h, L / HOT_SPAN + 1, 256 / s.lanes, 4);
+    dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
+        constexpr int BITS = decltype(bc)::value, LANES = decltype(lc)::value;
+        auto hot = k_hot_partial<LANES>;
+        auto upd = k_update<BITS, LANES>;
+        auto lst = k_update_list<BITS, LANES>;
+        LAUNCH(h, "hot_partial", hot, grid_for(h, L / HOT_SPAN + 1, 1, 4), 256, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
+        LAUNCH(h, "update", upd, gu, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step);
+        LAUNCH(h, "update_hot", lst, gh, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step, (const int32_t*)w.hot_k,
+               (const uint32_t*)&w.ctr->hot_rows, 0);
+        if (h->max_sets > 0)
+            LAUNCH(h, "update_deferred", lst, gh, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step, (const int32_t*)w.defer_k,
+                   (const uint32_t*)&w.ctr->deferred, 1);
+    });
     int rc = check_launch(h);
     if (rc != MPE_OK) return rc;
     h->have_forward = false;

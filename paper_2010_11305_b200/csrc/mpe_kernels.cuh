@@ -27,7 +27,7 @@ struct Counters {
     uint32_t hot_rows;
     uint32_t hot_tasks;
     uint32_t abort;        // offsets were inconsistent: every later kernel of the step returns at once
-    uint32_t pad;
+    uint32_t deferred;     // newcomers that wait for the write-back of an updated row
     unsigned long long dropped;      // out-of-range indices in this batch
     unsigned long long err[2];       // sticky: ERR_INDEX, ERR_OFFSETS
 };
@@ -58,6 +58,8 @@ struct Work {
     int32_t* occ_b;        // [L] by sorted order: sample of the element
     int32_t *uniq_row, *uniq_t, *seg, *loc, *final_loc, *victim, *hot_base, *uset;   // per unique row
     int32_t* task_k;       // [hot tasks]
+    int32_t* hot_k;        // [hot rows]
+    int32_t* defer_k;      // [deferred newcomers]
     float* partial;        // [hot tasks][dim]
 };
 
@@ -67,7 +69,7 @@ struct Work {
 __global__ void k_prelude(Work w, const int32_t* __restrict__ offsets, int T, int B, uint32_t L) {
     if (threadIdx.x == 0 && blockIdx.x == 0) {
         Counters* c = w.ctr;
-        c->L = L; c->U = 0; c->hot_rows = 0; c->hot_tasks = 0; c->abort = 0; c->dropped = 0;
+        c->L = L; c->U = 0; c->hot_rows = 0; c->hot_tasks = 0; c->abort = 0; c->dropped = 0; c->deferred = 0;
         bool bad = offsets[0] != 0 || offsets[(int64_t)T * B] != (int32_t)L;
         int32_t prev = 0;
         w.table_start[0] = 0;
@@ -218,7 +220,9 @@ __global__ void k_broadcast(State s, Work w, const uint32_t* __restrict__ spos, 
 }
 
 // ---------------------------------------------------------------------------------------------
-// forward: fetch + sum-pool, one group of dim/4 lanes per bag (Section 3 fetch; Algorithm 1 up-conversion)
+// forward: fetch + sum-pool, one group of LANES = dim/4 lanes per bag (Section 3 fetch; Algorithm 1
+// up-conversion).  The group reads LANES (slot, row id) pairs with one coalesced load, hands them
+// round with shuffles, and keeps up to eight row loads in flight; rows are added in index order.
 // ---------------------------------------------------------------------------------------------
 template <int BITS, bool RO>
 __device__ __forceinline__ float4 fetch4(const State& s, const TableDev& tb, int32_t row, int loc, int sub) {
@@ -229,30 +233,39 @@ __device__ __forceinline__ float4 fetch4(const State& s, const TableDev& tb, int
     return dequant4<BITS, RO>(s.codes, s.sb, tb.row_base + row, s.dim, sub);
 }
 
-template <int BITS>
+template <int BITS, int LANES>
 __global__ void __launch_bounds__(256)
 k_pool(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int B,
        float* __restrict__ out) {
-    const int lanes = s.lanes;
-    const int sub = threadIdx.x & (lanes - 1);
+    constexpr int NB = LANES < 8 ? LANES : 8;
+    const int sub = threadIdx.x & (LANES - 1);
+    const int gbase = (threadIdx.x & 31) & ~(LANES - 1);
+    const uint32_t gmask = group_mask(LANES);
     const int64_t nbags = (int64_t)s.T * B;
-    const int64_t gpb = blockDim.x / lanes, ng = gpb * gridDim.x;
+    const int64_t gpb = blockDim.x / LANES, ng = gpb * gridDim.x;
     const bool abort = w.ctr->abort != 0;
-    for (int64_t bag = blockIdx.x * gpb + threadIdx.x / lanes; bag < nbags; bag += ng) {
+    for (int64_t bag = blockIdx.x * gpb + threadIdx.x / LANES; bag < nbags; bag += ng) {
         const int t = (int)(bag / B);
         const int b = (int)(bag - (int64_t)t * B);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (!abort) {
             const TableDev tb = s.tables[t];
             const int32_t lo = offsets[bag], hi = offsets[bag + 1];
-            for (int32_t p = lo; p < hi; p += 4) {
-                int loc[4]; int32_t row[4]; float4 x[4];
+            for (int32_t p0 = lo; p0 < hi; p0 += LANES) {
+                const int n = min(LANES, hi - p0);
+                int myloc = LOC_INVALID; int32_t myrow = 0;
+                if (sub < n) { myloc = w.occ_loc[p0 + sub]; myrow = indices[p0 + sub]; }
+                for (int u0 = 0; u0 < n; u0 += NB) {
+                    float4 x[NB]; int lc[NB];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) if (p + u < hi) { loc[u] = w.occ_loc[p + u]; row[u] = indices[p + u]; }
+                    for (int u = 0; u < NB; ++u) {
+                        lc[u] = __shfl_sync(gmask, myloc, gbase + u0 + u);
+                        const int32_t rw = __shfl_sync(gmask, myrow, gbase + u0 + u);
+                        if (u0 + u < n && lc[u] != LOC_INVALID) x[u] = fetch4<BITS, true>(s, tb, rw, lc[u], sub);
+                    }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) if (p + u < hi && loc[u] != LOC_INVALID) x[u] = fetch4<BITS, true>(s, tb, row[u], loc[u], sub);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) if (p + u < hi && loc[u] != LOC_INVALID) acc = add4(acc, x[u]);
+                    for (int u = 0; u < NB; ++u) if (u0 + u < n && lc[u] != LOC_INVALID) acc = add4(acc, x[u]);
+                }
             }
         }
         reinterpret_cast<float4*>(out + ((int64_t)b * s.T + t) * s.dim)[sub] = acc;
@@ -290,7 +303,7 @@ __global__ void k_priority(State s, Work w, uint32_t step, uint32_t* __restrict_
                 if (mult > (uint32_t)HOT_SPAN) {
                     const uint32_t nt = (mult + HOT_SPAN - 1) / HOT_SPAN;
                     hb = (int)atomicAdd(&w.ctr->hot_tasks, nt);
-                    atomicAdd(&w.ctr->hot_rows, 1u);
+                    w.hot_k[atomicAdd(&w.ctr->hot_rows, 1u)] = (int32_t)k;
                     for (uint32_t j = 0; j < nt; ++j) w.task_k[hb + j] = (int32_t)k;
                 }
             }
@@ -319,13 +332,18 @@ __global__ void k_priority(State s, Work w, uint32_t step, uint32_t* __restrict_
 // ---------------------------------------------------------------------------------------------
 // backward 2: admission / eviction, integer only.  One group of `ways` lanes walks the miss
 // candidates of one set in ascending row id (Algorithm 2: j <- argmin PV; PV[i] <= PV[j] -> bypass,
-// else replace j by i in I_C[s]).  No row value is read or written here.
+// else replace j by i in I_C[s]).  Lane w holds way w of the set; the candidates are fetched `ways`
+// at a time (one per lane) and handed round with shuffles.  No row value is read or written here.
 // ---------------------------------------------------------------------------------------------
-__global__ void k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __restrict__ cval,
-                         uint32_t step, uint32_t epoch) {
+constexpr int VICTIM_NONE = -1;       // the way was empty, or the displaced row writes itself back
+constexpr int VICTIM_DEFER = -2;      // the displaced row was hit in this step: the newcomer waits for its write-back
+
+__global__ void __launch_bounds__(256)
+k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __restrict__ cval,
+         uint32_t step, uint32_t epoch) {
     if (w.ctr->abort) return;
     const int ways = s.ways;
-    const int lane = threadIdx.x & 31, way = lane & (ways - 1);
+    const int lane = threadIdx.x & 31, way = lane & (ways - 1), gbase = lane & ~(ways - 1);
     const uint32_t gmask = group_mask(ways);
     const int64_t U = w.ctr->U;
     const int64_t gpb = blockDim.x / ways, ng = gpb * gridDim.x;
@@ -339,44 +357,58 @@ __global__ void k_policy(State s, Work w, const uint32_t* __restrict__ ckey, con
         int32_t tag = s.tags[slot];
         uint32_t pri = 0;
         if (tag >= 0) pri = s.policy == 1 ? s.cnt[tb.row_base + tag] : s.ts[slot];
-        int32_t cand = -1, vict = -1;
+        int32_t cand = -1, vict = VICTIM_NONE;
         uint32_t n_admit = 0, n_evict = 0, n_bypass = 0;
         const int64_t jend = w.ustart[t + 1];
-        for (int64_t jj = j; jj < jend && ckey[jj] == key; ++jj) {
-            const int32_t kk = (int32_t)cval[jj];
-            const int32_t row = w.uniq_row[kk];
-            const uint32_t pv = s.policy == 1 ? s.cnt[tb.row_base + row] : step;
-            // empty ways rank below every priority; ties go to the lowest way
-            unsigned long long mine = tag < 0 ? (unsigned long long)way : ((((unsigned long long)pri + 1ULL) << 8) | (unsigned long long)way);
-            unsigned long long best = mine;
-            for (int o = ways >> 1; o > 0; o >>= 1) {
-                const unsigned long long other = __shfl_xor_sync(gmask, best, o);
-                best = other < best ? other : best;
+        for (int64_t jj0 = j;; jj0 += ways) {
+            const int64_t jj = jj0 + way;
+            const bool valid = jj < jend && ckey[jj] == key;
+            int32_t ckk = 0, crow = 0; uint32_t cpv = step;
+            if (valid) {
+                ckk = (int32_t)cval[jj];
+                crow = w.uniq_row[ckk];
+                if (s.policy == 1) cpv = s.cnt[tb.row_base + crow];
             }
-            const int jw = (int)(best & 255ULL);
-            const unsigned long long jp = best >> 8;                   // 0 = empty, else PV[j] + 1
-            bool replace = jp == 0 || (unsigned long long)pv + 1ULL > jp;
-            if (ways == 1 && s.policy == 0) replace = true;              // direct-mapped LRU never compares
-            if (replace) {
-                ++n_admit;
-                if (jp != 0) ++n_evict;
-                if (way == jw) {
-                    if (tag >= 0 && cand < 0) {
-                        // a row that was resident when the step began leaves the cache
-                        if (s.hit_epoch[slot] == epoch) { w.final_loc[s.hit_k[slot]] = LOC_MISS; vict = -1; }
-                        else vict = tag;
-                    }
-                    tag = row; pri = pv; cand = kk;
+            const int n = __popc(__ballot_sync(gmask, valid) & gmask);   // the valid lanes are a prefix of the group
+            for (int u = 0; u < n; ++u) {
+                const int32_t kk = __shfl_sync(gmask, ckk, gbase + u);
+                const int32_t row = __shfl_sync(gmask, crow, gbase + u);
+                const uint32_t pv = __shfl_sync(gmask, cpv, gbase + u);
+                // empty ways rank below every priority; ties go to the lowest way
+                const unsigned long long mine = tag < 0 ? (unsigned long long)way
+                                                        : ((((unsigned long long)pri + 1ULL) << 8) | (unsigned long long)way);
+                unsigned long long best = mine;
+                for (int o = ways >> 1; o > 0; o >>= 1) {
+                    const unsigned long long other = __shfl_xor_sync(gmask, best, o);
+                    best = other < best ? other : best;
                 }
-            } else {
-                ++n_bypass;
+                const int jw = (int)(best & 255ULL);
+                const unsigned long long jp = best >> 8;                   // 0 = empty, else PV[j] + 1
+                bool replace = jp == 0 || (unsigned long long)pv + 1ULL > jp;
+                if (ways == 1 && s.policy == 0) replace = true;              // direct-mapped LRU never compares
+                if (replace) {
+                    ++n_admit;
+                    if (jp != 0) ++n_evict;
+                    if (way == jw) {
+                        if (tag >= 0 && cand < 0) {
+                            // a row that was resident when the step began leaves the cache
+                            if (s.hit_epoch[slot] == epoch) { w.final_loc[s.hit_k[slot]] = LOC_MISS; vict = VICTIM_DEFER; }
+                            else vict = tag;
+                        }
+                        tag = row; pri = pv; cand = kk;
+                    }
+                } else {
+                    ++n_bypass;
+                }
             }
+            if (n < ways) break;
         }
         if (cand >= 0) {
             s.tags[slot] = tag;
             if (s.policy == 0) s.ts[slot] = step;
             w.final_loc[cand] = (int32_t)slot;
             w.victim[cand] = vict;
+            if (vict == VICTIM_DEFER) w.defer_k[atomicAdd(&w.ctr->deferred, 1u)] = cand;
         }
         if (way == 0) {
             unsigned long long* st = s.stats + (int64_t)t * 8;
@@ -390,18 +422,26 @@ __global__ void k_policy(State s, Work w, const uint32_t* __restrict__ ckey, con
 // ---------------------------------------------------------------------------------------------
 // backward 3: merged gradient of one distinct row (Section 5.1), radix-32 tree over index positions
 // ---------------------------------------------------------------------------------------------
-// up to 32 consecutive occurrences, added left to right
-__device__ __forceinline__ float4 sum_occurrences(const Work& w, const float* __restrict__ grad, int64_t col, int64_t stride,
-                                                  int32_t first, int len) {
+// up to 32 consecutive occurrences, added left to right; the group reads LANES sample ids at a time
+template <int LANES>
+__device__ __forceinline__ float4 sum_chunk(const int32_t* __restrict__ occ_b, const float* __restrict__ grad, int64_t col,
+                                            int64_t stride, int32_t first, int len, uint32_t gmask, int gbase, int sub) {
+    constexpr int NB = LANES < 8 ? LANES : 8;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int j0 = 0; j0 < len; j0 += 8) {
-        float4 v[8];
+    for (int j0 = 0; j0 < len; j0 += LANES) {
+        const int n = min(LANES, len - j0);
+        const int32_t myb = sub < n ? occ_b[first + j0 + sub] : 0;
+        for (int u0 = 0; u0 < n; u0 += NB) {
+            float4 v[NB];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-            if (j0 + u < len) v[u] = __ldg(reinterpret_cast<const float4*>(grad + (int64_t)w.occ_b[first + j0 + u] * stride + col));
+            for (int u = 0; u < NB; ++u) {
+                const int32_t b = __shfl_sync(gmask, myb, gbase + u0 + u);
+                if (u0 + u < n) v[u] = __ldg(reinterpret_cast<const float4*>(grad + (int64_t)b * stride + col));
+            }
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-            if (j0 + u < len) acc = (j0 + u == 0) ? v[u] : add4(acc, v[u]);
+            for (int u = 0; u < NB; ++u)
+                if (u0 + u < n) acc = (j0 + u0 + u == 0) ? v[u] : add4(acc, v[u]);
+        }
     }
     return acc;
 }
@@ -424,12 +464,15 @@ __device__ __forceinline__ float4 tree_reduce(const Term& term, int64_t first, i
 }
 
 // rows with more than HOT_SPAN occurrences: one block per HOT_SPAN occurrences computes two tree levels
+template <int LANES>
 __global__ void __launch_bounds__(256)
 k_hot_partial(State s, Work w, const float* __restrict__ grad, int B) {
     extern __shared__ float chunk_sums[];     // [32][dim]
     if (w.ctr->abort) return;
-    const int lanes = s.lanes, dim = s.dim;
-    const int sub = threadIdx.x & (lanes - 1), grp = threadIdx.x / lanes, ngrp = blockDim.x / lanes;
+    const int dim = s.dim;
+    const int sub = threadIdx.x & (LANES - 1), grp = threadIdx.x / LANES, ngrp = blockDim.x / LANES;
+    const int gbase = (threadIdx.x & 31) & ~(LANES - 1);
+    const uint32_t gmask = group_mask(LANES);
     const uint32_t ntask = w.ctr->hot_tasks;
     const int64_t stride = (int64_t)s.T * dim;
     for (uint32_t task = blockIdx.x; task < ntask; task += gridDim.x) {
@@ -440,7 +483,7 @@ k_hot_partial(State s, Work w, const float* __restrict__ grad, int B) {
         const int nchunk = (n + 31) >> 5;
         const int64_t col = (int64_t)w.uniq_t[k] * dim + 4 * sub;
         for (int c = grp; c < nchunk; c += ngrp) {
-            const float4 v = sum_occurrences(w, grad, col, stride, first + 32 * c, min(32, n - 32 * c));
+            const float4 v = sum_chunk<LANES>(w.occ_b, grad, col, stride, first + 32 * c, min(32, n - 32 * c), gmask, gbase, sub);
             reinterpret_cast<float4*>(chunk_sums + c * dim)[sub] = v;
         }
         __syncthreads();
@@ -454,72 +497,123 @@ k_hot_partial(State s, Work w, const float* __restrict__ grad, int B) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// backward 4: update(T, C, i, x).  phase 1: every distinct row except those that end the step as
-// new cache residents; phase 2: those, after the row they displace has been written back.
+// backward 4: update(T, C, i, x) for one distinct row whose merged gradient g is known
 // ---------------------------------------------------------------------------------------------
-template <int BITS>
-__global__ void __launch_bounds__(256)
-k_update(State s, Work w, const float* __restrict__ grad, int B, float lr, uint64_t step, int phase) {
+template <int BITS, int LANES>
+__device__ __forceinline__ void apply_update(const State& s, const TableDev& tb, int t, int32_t row, int loc, int floc,
+                                             int32_t victim, float4 g, float4 x, float lr, uint64_t step, int sub, uint32_t gmask) {
+    const int dim = 4 * LANES;
+    const int64_t grow = tb.row_base + row;
+    float mult = lr;                                         // SGD: x <- x - lr * g
+    if (s.optimizer == 1) {                                  // row-wise Adagrad
+        float a = __fmul_rn(g.x, g.x);
+        a = __fmaf_rn(g.y, g.y, a); a = __fmaf_rn(g.z, g.z, a); a = __fmaf_rn(g.w, g.w, a);
+#pragma unroll
+        for (int o = LANES >> 1; o > 0; o >>= 1) a = __fadd_rn(a, __shfl_xor_sync(gmask, a, o));
+        const float Gold = s.G[grow];
+        __syncwarp(gmask);                                   // every lane has read G before lane 0 replaces it
+        const float Gn = __fadd_rn(Gold, __fmul_rn(a, __fdiv_rn(1.0f, (float)dim)));
+        if (sub == 0) s.G[grow] = Gn;
+        mult = __fdiv_rn(lr, __fadd_rn(__fsqrt_rn(Gn), s.eps));
+    }
+    float4 xn;
+    xn.x = __fmaf_rn(-mult, g.x, x.x); xn.y = __fmaf_rn(-mult, g.y, x.y);
+    xn.z = __fmaf_rn(-mult, g.z, x.z); xn.w = __fmaf_rn(-mult, g.w, x.w);
+    if (floc >= 0) {
+        float4* dst = reinterpret_cast<float4*>(s.slab + (int64_t)floc * dim) + sub;
+        if (loc < 0 && victim >= 0)     // the row this newcomer displaces is down-converted and placed back in T
+            quantize_store<BITS, true>(*dst, s.codes, s.sb, tb.row_base + victim, dim, sub, LANES,
+                                       rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)victim, step));
+        *dst = xn;                      // cached rows keep full precision, a newcomer enters verbatim
+    } else {
+        quantize_store<BITS, true>(xn, s.codes, s.sb, grow, dim, sub, LANES,
+                                   rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)row, step));
+    }
+}
+
+// Every distinct row with at most HOT_SPAN occurrences, except newcomers that wait for a write-back.
+// A warp stages the bookkeeping of 32 consecutive rows in shared memory with coalesced loads, then
+// its groups of LANES lanes take the rows one by one.
+template <int BITS, int LANES>
+__global__ void __launch_bounds__(256, 3)
+k_update(State s, Work w, const float* __restrict__ grad, int B, float lr, uint64_t step) {
+    __shared__ int32_t meta[8][32][8];
     if (w.ctr->abort) return;
-    const int lanes = s.lanes, dim = s.dim;
-    const int sub = threadIdx.x & (lanes - 1);
-    const uint32_t gmask = group_mask(lanes);
+    constexpr int dim = 4 * LANES, G = 32 / LANES;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int sub = lane & (LANES - 1), grp = lane / LANES, gbase = lane & ~(LANES - 1);
+    const uint32_t gmask = group_mask(LANES);
     const int64_t U = w.ctr->U;
-    const int64_t gpb = blockDim.x / lanes, ng = gpb * gridDim.x;
+    const int64_t nwarps = (int64_t)gridDim.x * 8;
     const int64_t stride = (int64_t)s.T * dim;
-    for (int64_t k = blockIdx.x * gpb + threadIdx.x / lanes; k < U; k += ng) {
-        const int loc = w.loc[k];
+    for (int64_t k0 = ((int64_t)blockIdx.x * 8 + warp) * 32; k0 < U; k0 += nwarps * 32) {
+        __syncwarp();
+        const int64_t k = k0 + lane;
+        if (k < U) {
+            const int32_t first = w.seg[k];
+            int32_t* mrow = meta[warp][lane];
+            mrow[0] = w.loc[k]; mrow[1] = w.final_loc[k]; mrow[2] = w.uniq_t[k]; mrow[3] = w.uniq_row[k];
+            mrow[4] = first; mrow[5] = w.seg[k + 1] - first; mrow[6] = w.hot_base[k]; mrow[7] = w.victim[k];
+        }
+        __syncwarp();
+        const int nrow = (int)min((int64_t)32, U - k0);
+        for (int r = grp; r < nrow; r += G) {
+            const int32_t* mrow = meta[warp][r];
+            const int loc = mrow[0], floc = mrow[1];
+            if (loc == LOC_INVALID || mrow[6] >= 0) continue;            // pseudo row; hot rows have their own kernel
+            const int32_t victim = mrow[7];
+            if (loc < 0 && floc >= 0 && victim == VICTIM_DEFER) continue;
+            const int t = mrow[2];
+            const int32_t row = mrow[3], first = mrow[4], m = mrow[5];
+            const TableDev tb = s.tables[t];
+            const float4 x = fetch4<BITS, false>(s, tb, row, loc, sub);  // the value the forward fetched
+            const int64_t col = (int64_t)t * dim + 4 * sub;
+            float4 g = sum_chunk<LANES>(w.occ_b, grad, col, stride, first, min(32, m), gmask, gbase, sub);
+            for (int32_t c = 32; c < m; c += 32)
+                g = add4(g, sum_chunk<LANES>(w.occ_b, grad, col, stride, first + c, min(32, m - c), gmask, gbase, sub));
+            apply_update<BITS, LANES>(s, tb, t, row, loc, floc, victim, g, x, lr, step, sub, gmask);
+        }
+    }
+}
+
+// Rows named by a list: the hot rows (gradient from the partial sums of k_hot_partial), and, in a
+// second launch, the newcomers whose slot had to be vacated by a row that was itself updated.
+template <int BITS, int LANES>
+__global__ void __launch_bounds__(256)
+k_update_list(State s, Work w, const float* __restrict__ grad, int B, float lr, uint64_t step,
+              const int32_t* __restrict__ list, const uint32_t* __restrict__ count, int deferred_pass) {
+    if (w.ctr->abort) return;
+    constexpr int dim = 4 * LANES;
+    const int lane = threadIdx.x & 31;
+    const int sub = lane & (LANES - 1), gbase = lane & ~(LANES - 1);
+    const uint32_t gmask = group_mask(LANES);
+    const int64_t n = *count;
+    const int64_t gpb = blockDim.x / LANES, ng = gpb * gridDim.x;
+    const int64_t stride = (int64_t)s.T * dim;
+    for (int64_t i = blockIdx.x * gpb + threadIdx.x / LANES; i < n; i += ng) {
+        const int32_t k = list[i];
+        const int loc = w.loc[k], floc = w.final_loc[k];
         if (loc == LOC_INVALID) continue;
-        const int floc = w.final_loc[k];
-        const bool newcomer = loc < 0 && floc >= 0;
-        if (newcomer != (phase == 2)) continue;
+        int32_t victim = (loc < 0 && floc >= 0) ? w.victim[k] : VICTIM_NONE;
+        if (!deferred_pass && victim == VICTIM_DEFER) continue;          // comes back in the deferred pass
         const int t = w.uniq_t[k];
         const int32_t row = w.uniq_row[k];
         const TableDev tb = s.tables[t];
-        const int64_t grow = tb.row_base + row;
         const int32_t first = w.seg[k], m = w.seg[k + 1] - first;
         const int64_t col = (int64_t)t * dim + 4 * sub;
-        // merged gradient
+        const float4 x = fetch4<BITS, false>(s, tb, row, loc, sub);
         float4 g;
         const int hb = w.hot_base[k];
         if (hb < 0) {
-            auto chunk = [&](int64_t c) { return sum_occurrences(w, grad, col, stride, first + 32 * (int32_t)c, min(32, m - 32 * (int32_t)c)); };
-            g = tree_reduce<0>(chunk, 0, (m + 31) >> 5);
+            g = sum_chunk<LANES>(w.occ_b, grad, col, stride, first, min(32, m), gmask, gbase, sub);
+            for (int32_t c = 32; c < m; c += 32)
+                g = add4(g, sum_chunk<LANES>(w.occ_b, grad, col, stride, first + c, min(32, m - c), gmask, gbase, sub));
         } else {
             const float* part = w.partial + (int64_t)hb * dim + 4 * sub;
             auto term = [&](int64_t j) { return *reinterpret_cast<const float4*>(part + j * dim); };
             g = tree_reduce<4>(term, 0, (m + HOT_SPAN - 1) / HOT_SPAN);
         }
-        // the value the forward fetched
-        const float4 x = fetch4<BITS, false>(s, tb, row, loc, sub);
-        // optimizer, full precision
-        float mult = lr;
-        if (s.optimizer == 1) {
-            float a = __fmul_rn(g.x, g.x);
-            a = __fmaf_rn(g.y, g.y, a); a = __fmaf_rn(g.z, g.z, a); a = __fmaf_rn(g.w, g.w, a);
-            for (int o = lanes >> 1; o > 0; o >>= 1) a = __fadd_rn(a, __shfl_xor_sync(gmask, a, o));
-            const float Gold = s.G[grow];
-            __syncwarp(gmask);                               // every lane has read G before lane 0 replaces it
-            const float Gn = __fadd_rn(Gold, __fmul_rn(a, __fdiv_rn(1.0f, (float)dim)));
-            if (sub == 0) s.G[grow] = Gn;
-            mult = __fdiv_rn(lr, __fadd_rn(__fsqrt_rn(Gn), s.eps));
-        }
-        float4 xn;
-        xn.x = __fmaf_rn(-mult, g.x, x.x); xn.y = __fmaf_rn(-mult, g.y, x.y);
-        xn.z = __fmaf_rn(-mult, g.z, x.z); xn.w = __fmaf_rn(-mult, g.w, x.w);
-        if (floc >= 0) {
-            float4* dst = reinterpret_cast<float4*>(s.slab + (int64_t)floc * dim) + sub;
-            if (phase == 2) {
-                const int32_t v = w.victim[k];
-                if (v >= 0)   // the displaced row is down-converted and placed back in T
-                    quantize_store<BITS, true>(*dst, s.codes, s.sb, tb.row_base + v, dim, sub, lanes,
-                                               rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)v, step));
-            }
-            *dst = xn;       // cached rows keep full precision, a newcomer enters verbatim
-        } else {
-            quantize_store<BITS, true>(xn, s.codes, s.sb, grow, dim, sub, lanes,
-                                       rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)row, step));
-        }
+        apply_update<BITS, LANES>(s, tb, t, row, loc, floc, victim, g, x, lr, step, sub, gmask);
     }
 }
 
