@@ -354,6 +354,7 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
     if (!h || (!d_grad_out && h->B > 0)) return MPE_ERR_ARG;
     if (!h->have_forward) return MPE_ERR_SEQUENCE;
     if (step < 1 || step > 0xffffffffLL) return MPE_ERR_ARG;
+    if (reinterpret_cast<uintptr_t>(d_grad_out) & 15) return MPE_ERR_ARG;   // rows are moved 16 bytes at a time
     if (step <= h->last_step) return MPE_ERR_SEQUENCE;
     DeviceGuard guard(h->device);
     const State& s = h->st;
@@ -370,7 +371,7 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
         const uint32_t* cv = which ? h->cvalB : h->cvalA;
         LAUNCH(h, "policy", k_policy, grid_for(h, L, 256 / s.ways, 8), 256, 0, s, w, ck, cv, (uint32_t)step, h->epoch);
     }
-    const int gu = grid_for(h, (L + 31) / 32, 8, 3);
+    const int gu = grid_for(h, (L + 31) / 32, UPD_WARPS, 5);
     const int gh = grid_for(h, L / HOT_SPAN + 1, 256 / s.lanes, 4);
     dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
         constexpr int BITS = decltype(bc)::value, LANES = decltype(lc)::value;
@@ -378,7 +379,9 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
         auto upd = k_update<BITS, LANES>;
         auto lst = k_update_list<BITS, LANES>;
         LAUNCH(h, "hot_partial", hot, grid_for(h, L / HOT_SPAN + 1, 1, 4), 256, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
-        LAUNCH(h, "update", upd, gu, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step);
+        static bool smem_set = false;     // one flag per instantiation of this lambda
+        if (!smem_set) { cudaFuncSetAttribute(upd, cudaFuncAttributeMaxDynamicSharedMemorySize, UPD_SMEM); smem_set = true; }
+        LAUNCH(h, "update", upd, gu, UPD_WARPS * 32, UPD_SMEM, s, w, d_grad_out, B, lr, (uint64_t)step);
         LAUNCH(h, "update_hot", lst, gh, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step, (const int32_t*)w.hot_k,
                (const uint32_t*)&w.ctr->hot_rows, 0);
         if (h->max_sets > 0)

@@ -47,6 +47,24 @@ __device__ __forceinline__ uint32_t group_mask(int lanes_per_row) {
     return lanes_per_row == 32 ? 0xffffffffU : (((1U << lanes_per_row) - 1U) << (lane & ~(lanes_per_row - 1)));
 }
 
+// four codes (packed in q, lowest column in the lowest bits) -> q*scale + bias (Algorithm 1, up-conversion)
+template <int BITS>
+__device__ __forceinline__ float4 decode4(uint32_t q, float2 p) {
+    float4 x;
+    if (BITS == 8) {
+        x.x = __fmaf_rn(__uint2float_rn(q & 255u), p.x, p.y);
+        x.y = __fmaf_rn(__uint2float_rn((q >> 8) & 255u), p.x, p.y);
+        x.z = __fmaf_rn(__uint2float_rn((q >> 16) & 255u), p.x, p.y);
+        x.w = __fmaf_rn(__uint2float_rn(q >> 24), p.x, p.y);
+    } else {
+        x.x = __fmaf_rn(__uint2float_rn(q & 15u), p.x, p.y);
+        x.y = __fmaf_rn(__uint2float_rn((q >> 4) & 15u), p.x, p.y);
+        x.z = __fmaf_rn(__uint2float_rn((q >> 8) & 15u), p.x, p.y);
+        x.w = __fmaf_rn(__uint2float_rn((q >> 12) & 15u), p.x, p.y);
+    }
+    return x;
+}
+
 // RO = the table is not written by the running kernel, so the read-only data path may serve the loads
 template <int BITS, bool RO>
 __device__ __forceinline__ float4 dequant4(const uint8_t* codes, const float2* sb, int64_t grow, int dim, int sub) {
@@ -62,19 +80,7 @@ __device__ __forceinline__ float4 dequant4(const uint8_t* codes, const float2* s
         if (BITS == 8) q = reinterpret_cast<const uint32_t*>(codes + grow * dim)[sub];
         else           q = reinterpret_cast<const uint16_t*>(codes + grow * (dim >> 1))[sub];
     }
-    float4 x;
-    if (BITS == 8) {
-        x.x = __fmaf_rn(__uint2float_rn(q & 255u), p.x, p.y);
-        x.y = __fmaf_rn(__uint2float_rn((q >> 8) & 255u), p.x, p.y);
-        x.z = __fmaf_rn(__uint2float_rn((q >> 16) & 255u), p.x, p.y);
-        x.w = __fmaf_rn(__uint2float_rn(q >> 24), p.x, p.y);
-    } else {
-        x.x = __fmaf_rn(__uint2float_rn(q & 15u), p.x, p.y);
-        x.y = __fmaf_rn(__uint2float_rn((q >> 4) & 15u), p.x, p.y);
-        x.z = __fmaf_rn(__uint2float_rn((q >> 8) & 15u), p.x, p.y);
-        x.w = __fmaf_rn(__uint2float_rn((q >> 12) & 15u), p.x, p.y);
-    }
-    return x;
+    return decode4<BITS>(q, p);
 }
 
 __device__ __forceinline__ float4 add4(float4 a, float4 b) {

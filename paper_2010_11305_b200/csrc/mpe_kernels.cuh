@@ -531,47 +531,183 @@ __device__ __forceinline__ void apply_update(const State& s, const TableDev& tb,
     }
 }
 
+// ---- asynchronous 16-byte copies global -> shared (per thread; completion is waited for by group count) ----
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+struct RawRow { float4 f; uint32_t q; float2 sb; };
+
+constexpr int UPD_WARPS = 4;     // warps per block of k_update
+constexpr int UPD_RING = 16;     // gradient rows a group can have in shared memory
+constexpr int UPD_GROUPS = 4;    // copy groups a group keeps in flight (each up to 4 rows)
+constexpr int UPD_NB = 4;        // rows per copy group
+constexpr int UPD_META = 16;     // ints of bookkeeping per staged row
+constexpr int UPD_SMEM = UPD_WARPS * (UPD_RING * 32 * 16 + 32 * UPD_META * 4);
+
 // Every distinct row with at most HOT_SPAN occurrences, except newcomers that wait for a write-back.
-// A warp stages the bookkeeping of 32 consecutive rows in shared memory with coalesced loads, then
-// its groups of LANES lanes take the rows one by one.
+// A warp stages the bookkeeping of 32 consecutive rows in shared memory, one row per lane (coalesced
+// loads; the per-row scalar work -- addresses, the stochastic-rounding key -- is done there once, 32
+// rows at a time).  Each group of LANES lanes then streams through the gradient rows of its rows:
+// asynchronous 16-byte copies bring up to UPD_GROUPS x UPD_NB gradient rows into a shared-memory ring
+// while earlier ones are being added (in index order, radix-32 tree), independent of where one
+// embedding row ends and the next begins.
 template <int BITS, int LANES>
-__global__ void __launch_bounds__(256, 3)
+__global__ void __launch_bounds__(UPD_WARPS * 32)
 k_update(State s, Work w, const float* __restrict__ grad, int B, float lr, uint64_t step) {
-    __shared__ int32_t meta[8][32][8];
+    extern __shared__ __align__(16) unsigned char upd_smem[];
     if (w.ctr->abort) return;
-    constexpr int dim = 4 * LANES, G = 32 / LANES;
+    constexpr int dim = 4 * LANES, G = 32 / LANES, NB = LANES < UPD_NB ? LANES : UPD_NB;
+    enum { M_LOC, M_FLOC, M_COL, M_ROW, M_FIRST, M_CNT, M_SKIP, M_VICTIM, M_KEY, M_VKEY, M_GROW_LO, M_GROW_HI, M_VROW_LO, M_VROW_HI };
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int sub = lane & (LANES - 1), grp = lane / LANES, gbase = lane & ~(LANES - 1);
     const uint32_t gmask = group_mask(LANES);
+    float4* ring = reinterpret_cast<float4*>(upd_smem) + ((warp * G + grp) * UPD_RING) * LANES + sub;   // slot i: ring[i * LANES]
+    int32_t(*meta)[UPD_META] = reinterpret_cast<int32_t(*)[UPD_META]>(upd_smem + UPD_WARPS * UPD_RING * 32 * 16) + warp * 32;
     const int64_t U = w.ctr->U;
-    const int64_t nwarps = (int64_t)gridDim.x * 8;
+    const int64_t nwarps = (int64_t)gridDim.x * UPD_WARPS;
     const int64_t stride = (int64_t)s.T * dim;
-    for (int64_t k0 = ((int64_t)blockIdx.x * 8 + warp) * 32; k0 < U; k0 += nwarps * 32) {
+    const float* gcol = grad + 4 * sub;
+    for (int64_t k0 = ((int64_t)blockIdx.x * UPD_WARPS + warp) * 32; k0 < U; k0 += nwarps * 32) {
         __syncwarp();
         const int64_t k = k0 + lane;
         if (k < U) {
-            const int32_t first = w.seg[k];
-            int32_t* mrow = meta[warp][lane];
-            mrow[0] = w.loc[k]; mrow[1] = w.final_loc[k]; mrow[2] = w.uniq_t[k]; mrow[3] = w.uniq_row[k];
-            mrow[4] = first; mrow[5] = w.seg[k + 1] - first; mrow[6] = w.hot_base[k]; mrow[7] = w.victim[k];
+            const int32_t first = w.seg[k], row = w.uniq_row[k];
+            const int loc = w.loc[k], floc = w.final_loc[k], hb = w.hot_base[k], victim = w.victim[k], t = w.uniq_t[k];
+            int32_t* mrow = meta[lane];
+            mrow[M_LOC] = loc; mrow[M_FLOC] = floc; mrow[M_COL] = t * dim; mrow[M_ROW] = row;
+            mrow[M_FIRST] = first; mrow[M_CNT] = w.seg[k + 1] - first; mrow[M_VICTIM] = victim;
+            // pseudo rows, hot rows (own kernel) and newcomers that wait for a write-back are not ours
+            const bool newcomer = loc < 0 && floc >= 0;
+            const bool skip = loc == LOC_INVALID || hb >= 0 || (newcomer && victim == VICTIM_DEFER);
+            mrow[M_SKIP] = skip ? 1 : 0;
+            if (!skip) {
+                const int64_t rb = s.tables[t].row_base;
+                const int64_t grow = rb + row;
+                mrow[M_GROW_LO] = (int32_t)(uint32_t)grow; mrow[M_GROW_HI] = (int32_t)(grow >> 32);
+                mrow[M_KEY] = (int32_t)rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)row, step);
+                // pull this row's current value towards L2 now; it is needed when its gradient has been summed
+                if (loc >= 0) {
+                    const char* src = reinterpret_cast<const char*>(s.slab + (int64_t)loc * dim);
+#pragma unroll
+                    for (int o = 0; o < dim * 4; o += 128) prefetch_l2(src + o);
+                } else {
+                    prefetch_l2(s.codes + grow * (dim * BITS / 8));
+                    prefetch_l2(s.sb + grow);
+                }
+                if (newcomer && victim >= 0) {
+                    const int64_t vrow = rb + victim;
+                    mrow[M_VROW_LO] = (int32_t)(uint32_t)vrow; mrow[M_VROW_HI] = (int32_t)(vrow >> 32);
+                    mrow[M_VKEY] = (int32_t)rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)victim, step);
+                    const char* src = reinterpret_cast<const char*>(s.slab + (int64_t)floc * dim);
+#pragma unroll
+                    for (int o = 0; o < dim * 4; o += 128) prefetch_l2(src + o);
+                }
+            }
         }
         __syncwarp();
         const int nrow = (int)min((int64_t)32, U - k0);
-        for (int r = grp; r < nrow; r += G) {
-            const int32_t* mrow = meta[warp][r];
-            const int loc = mrow[0], floc = mrow[1];
-            if (loc == LOC_INVALID || mrow[6] >= 0) continue;            // pseudo row; hot rows have their own kernel
-            const int32_t victim = mrow[7];
-            if (loc < 0 && floc >= 0 && victim == VICTIM_DEFER) continue;
-            const int t = mrow[2];
-            const int32_t row = mrow[3], first = mrow[4], m = mrow[5];
-            const TableDev tb = s.tables[t];
-            const float4 x = fetch4<BITS, false>(s, tb, row, loc, sub);  // the value the forward fetched
-            const int64_t col = (int64_t)t * dim + 4 * sub;
-            float4 g = sum_chunk<LANES>(w.occ_b, grad, col, stride, first, min(32, m), gmask, gbase, sub);
-            for (int32_t c = 32; c < m; c += 32)
-                g = add4(g, sum_chunk<LANES>(w.occ_b, grad, col, stride, first + c, min(32, m - c), gmask, gbase, sub));
-            apply_update<BITS, LANES>(s, tb, t, row, loc, floc, victim, g, x, lr, step, sub, gmask);
+        {   // and the sample ids of the warp's occurrences (one contiguous range of the sorted batch)
+            const int32_t o0 = meta[0][M_FIRST], o1 = meta[nrow - 1][M_FIRST] + meta[nrow - 1][M_CNT];
+            for (int32_t o = o0 + 32 * lane; o < o1 && o < o0 + 4096; o += 1024) prefetch_l2(w.occ_b + o);
+        }
+        auto valid_from = [&](int r) { while (r < nrow && meta[r][M_SKIP]) r += G; return r; };
+        int pr = valid_from(grp), po = 0;          // producer: next gradient row to request
+        int cr = pr, co = 0;                        // consumer: next gradient row to add
+        int head = 0, tail = 0, inflight = 0;
+        int ncnt = 0; int32_t nb = 0;               // the next copy group: how many rows, and their sample ids (one per lane)
+        auto describe_next = [&]() {
+            if (pr < nrow) {
+                ncnt = min(NB, meta[pr][M_CNT] - po);
+                nb = sub < ncnt ? w.occ_b[meta[pr][M_FIRST] + po + sub] : 0;
+            }
+        };
+        describe_next();
+        RawRow xr;
+        auto load_x = [&]() {
+            const int loc = meta[cr][M_LOC];
+            if (loc >= 0) {
+                xr.f = reinterpret_cast<const float4*>(s.slab + (int64_t)loc * dim)[sub];
+            } else {
+                const int64_t grow = ((int64_t)meta[cr][M_GROW_HI] << 32) | (uint32_t)meta[cr][M_GROW_LO];
+                xr.sb = s.sb[grow];
+                if (BITS == 8) xr.q = reinterpret_cast<const uint32_t*>(s.codes + grow * dim)[sub];
+                else           xr.q = reinterpret_cast<const uint16_t*>(s.codes + grow * (dim >> 1))[sub];
+            }
+        };
+        if (cr < nrow) load_x();
+        float4 chunkacc = make_float4(0.f, 0.f, 0.f, 0.f), rowacc = chunkacc;
+        while (cr < nrow) {
+            while (inflight < UPD_GROUPS && pr < nrow) {
+                const float* src = gcol + meta[pr][M_COL];
+#pragma unroll
+                for (int u = 0; u < NB; ++u) {
+                    const int32_t b = __shfl_sync(gmask, nb, gbase + u);
+                    if (u < ncnt) cp_async16(ring + ((head + u) & (UPD_RING - 1)) * LANES, src + (int64_t)b * stride);
+                }
+                cp_async_commit();
+                head += ncnt; ++inflight; po += ncnt;
+                if (po == meta[pr][M_CNT]) { pr = valid_from(pr + G); po = 0; }
+                describe_next();
+            }
+            switch (inflight) {                     // the oldest group has landed when at most inflight-1 are pending
+                case 1: cp_async_wait<0>(); break;
+                case 2: cp_async_wait<1>(); break;
+                case 3: cp_async_wait<2>(); break;
+                default: cp_async_wait<3>(); break;
+            }
+            const int m = meta[cr][M_CNT];
+            const int cnt = min(NB, m - co);
+            // a copy group never straddles a chunk of 32 terms: add its rows left to right ...
+            float4 acc = ring[(tail & (UPD_RING - 1)) * LANES];
+            if (co & 31) acc = add4(chunkacc, acc);
+#pragma unroll
+            for (int u = 1; u < NB; ++u)
+                if (u < cnt) acc = add4(acc, ring[((tail + u) & (UPD_RING - 1)) * LANES]);
+            chunkacc = acc;
+            tail += cnt; co += cnt; --inflight;
+            // ... and fold a finished chunk into the sum of chunk sums
+            if ((co & 31) == 0 || co == m) rowacc = co <= 32 ? chunkacc : add4(rowacc, chunkacc);
+            if (co == m) {
+                const int32_t* mc = meta[cr];
+                const int loc = mc[M_LOC], floc = mc[M_FLOC];
+                float4 x = xr.f;
+                if (loc < 0) x = decode4<BITS>(xr.q, xr.sb);
+                const int64_t grow = ((int64_t)mc[M_GROW_HI] << 32) | (uint32_t)mc[M_GROW_LO];
+                float mult = lr;                                         // SGD: x <- x - lr * g
+                if (s.optimizer == 1) {                                  // row-wise Adagrad
+                    float a = __fmul_rn(rowacc.x, rowacc.x);
+                    a = __fmaf_rn(rowacc.y, rowacc.y, a); a = __fmaf_rn(rowacc.z, rowacc.z, a); a = __fmaf_rn(rowacc.w, rowacc.w, a);
+#pragma unroll
+                    for (int o = LANES >> 1; o > 0; o >>= 1) a = __fadd_rn(a, __shfl_xor_sync(gmask, a, o));
+                    const float Gold = s.G[grow];
+                    __syncwarp(gmask);                                   // every lane has read G before lane 0 replaces it
+                    const float Gn = __fadd_rn(Gold, __fmul_rn(a, __fdiv_rn(1.0f, (float)dim)));
+                    if (sub == 0) s.G[grow] = Gn;
+                    mult = __fdiv_rn(lr, __fadd_rn(__fsqrt_rn(Gn), s.eps));
+                }
+                float4 xn;
+                xn.x = __fmaf_rn(-mult, rowacc.x, x.x); xn.y = __fmaf_rn(-mult, rowacc.y, x.y);
+                xn.z = __fmaf_rn(-mult, rowacc.z, x.z); xn.w = __fmaf_rn(-mult, rowacc.w, x.w);
+                if (floc >= 0) {
+                    float4* dst = reinterpret_cast<float4*>(s.slab + (int64_t)floc * dim) + sub;
+                    if (loc < 0 && mc[M_VICTIM] >= 0) {  // the row this newcomer displaces is down-converted and placed back in T
+                        const int64_t vrow = ((int64_t)mc[M_VROW_HI] << 32) | (uint32_t)mc[M_VROW_LO];
+                        quantize_store<BITS, true>(*dst, s.codes, s.sb, vrow, dim, sub, LANES, (uint32_t)mc[M_VKEY]);
+                    }
+                    *dst = xn;                           // cached rows keep full precision, a newcomer enters verbatim
+                } else {
+                    quantize_store<BITS, true>(xn, s.codes, s.sb, grow, dim, sub, LANES, (uint32_t)mc[M_KEY]);
+                }
+                cr = valid_from(cr + G); co = 0;
+                if (cr < nrow) load_x();
+            }
         }
     }
 }
