@@ -267,3 +267,48 @@ def test_memory_accounting_matches_the_appendix_table():
         m = h.memory_bytes().astype(np.float64)
         assert abs((m[0] + m[1] + m[2] + m[3]) / m[5] - float(factor)) < 6e-6
         h.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# Full-size configurations, in the launch configuration the benchmark times.  The oracle follows a
+# sample of the tables (tables are independent); everything observable of those tables is compared.
+# ---------------------------------------------------------------------------------------------
+def _full_size(cfg, tables, steps):
+    from parity_util import make_pair, compare_state
+    h, o = make_pair(cfg, tables)
+    st = wl.Stream(cfg, "cuda")
+    rng = np.random.default_rng(0)
+    cols = np.concatenate([np.arange(t * cfg.dim, (t + 1) * cfg.dim) for t in tables])
+    for step in range(1, steps + 1):
+        idx, off, grad = st.batch(step)
+        out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, device="cuda")
+        h.forward(idx, off, cfg.batch, out)
+        ref = o.forward(idx.cpu().numpy(), off.cpu().numpy(), cfg.batch)
+        assert np.array_equal(out[:, torch.as_tensor(cols, device="cuda")].cpu().numpy(), ref[:, cols]), f"step {step}: pooled outputs"
+        h.backward(grad, cfg.lr, step)
+        o.backward(grad.cpu().numpy(), cfg.lr, step)
+        assert h.last_error() == (0, 0)
+    compare_state(h, o, cfg, tables, rng)
+    h.flush()
+    o.flush()
+    compare_state(h, o, cfg, tables, rng)
+    return h
+
+
+def test_full_size_config4_sampled_tables():
+    cfg = wl.config(4)
+    h = _full_size(cfg, [0, 37, 63], 3)
+    info = h.step_info()
+    assert info[0] > 25_000_000 and info[3] > 500      # ~31M indices, thousands of hot rows
+    h.close()
+
+
+def test_full_size_config3_sampled_tables():
+    cfg = wl.config(3)
+    _full_size(cfg, [0, 5], 4).close()
+
+
+def test_full_size_config5_points():
+    pts = list(wl.sweep5())
+    for i in (5, 30, 58):
+        _full_size(pts[i], [1], 3).close()
