@@ -133,8 +133,8 @@ int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
     A(w.bag_of, n); A(w.kidx, n); A(w.occ_loc, n); A(w.occ_b, n);
     A(w.uniq_row, n); A(w.uniq_t, n); A(w.seg, n + 1); A(w.loc, n); A(w.final_loc, n); A(w.victim, n);
     A(w.hot_base, n); A(w.uset, n);
-    const int64_t max_tasks = L / (HOT_SPAN / 2) + 2;
-    A(w.task_k, max_tasks); A(w.partial, max_tasks * h->dim); A(w.hot_k, L / HOT_SPAN + 2); A(w.defer_k, n);
+    const int64_t max_tasks = L / HOT_MIN + 2;
+    A(w.task_k, max_tasks); A(w.partial, max_tasks * h->dim); A(w.hot_k, L / HOT_MIN + 2); A(w.defer_k, n); A(w.heads, n);
 #undef A
     CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), h->stream));
     h->cap_L = L; h->cap_bags = bags;
@@ -156,7 +156,7 @@ int seg_sort(mpe_handle* h, uint32_t* kA, uint32_t* kB, uint32_t* vA, uint32_t* 
     const int T = h->T;
     LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, seg_start, T, tile_base, hist_len, (const uint32_t*)&h->wk.ctr->abort);
     const int64_t max_tiles = (n_upper + SORT_TILE - 1) / SORT_TILE + T;
-    const int g = grid_for(h, max_tiles, 1, 4);
+    const int g = grid_for(h, max_tiles, 1, 3);
     const int passes = (key_bits + 7) / 8;
     uint32_t *kin = kA, *kout = kB, *vin = nullptr, *vout = vB;
     for (int p = 0; p < passes; ++p) {
@@ -254,7 +254,8 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
         h->max_rows = std::max(h->max_rows, tb.N); h->max_sets = std::max(h->max_sets, tb.n_sets);
     }
     h->total_slots = h->total_sets * ways;
-    if (h->total_slots > 0x7fffffffLL) { delete h; return MPE_ERR_UNSUPPORTED; }
+    // slots are int32; one sample's row of the pooled output must stay below 4 GiB (32-bit byte strides in the kernels)
+    if (h->total_slots > 0x7fffffffLL || (int64_t)num_tables * dim > 0x0fffffffLL) { delete h; return MPE_ERR_UNSUPPORTED; }
 
     State& s = h->st;
     s.T = num_tables; s.dim = dim; s.lanes = dim / 4; s.ways = ways; s.policy = policy; s.optimizer = optimizer;
@@ -337,7 +338,7 @@ int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offset
     LAUNCH(h, "unique_write", k_unique<true>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
     LAUNCH(h, "ustart", k_ustart, 1, 256, 0, w, T);
     // tag lookup, then fetch + pool
-    LAUNCH(h, "probe", k_probe, grid_for(h, total_indices, 256 / s.ways, 8), 256, 0, s, w, h->epoch);
+    LAUNCH(h, "probe", k_probe, grid_for(h, total_indices, 256, 8), 256, 0, s, w, h->epoch);
     LAUNCH(h, "broadcast", k_broadcast, grid_for(h, total_indices, 256, 8), 256, 0, s, w, h->spos, batch);
     const int gp = grid_for(h, bags, 256 / s.lanes, 8);
     dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
@@ -369,16 +370,18 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
                                    bits_for((uint32_t)h->max_sets), L);
         const uint32_t* ck = which ? h->ckeyB : h->ckeyA;
         const uint32_t* cv = which ? h->cvalB : h->cvalA;
-        LAUNCH(h, "policy", k_policy, grid_for(h, L, 256 / s.ways, 8), 256, 0, s, w, ck, cv, (uint32_t)step, h->epoch);
+        LAUNCH(h, "policy_heads", k_policy_heads, grid_for(h, L, 256, 8), 256, 0, s, w, ck);
+        LAUNCH(h, "policy", k_policy, grid_for(h, std::min<int64_t>(L, h->total_sets), 256 / s.ways, 8), 256, 0, s, w, ck, cv,
+               (uint32_t)step, h->epoch);
     }
     const int gu = grid_for(h, (L + 31) / 32, UPD_WARPS, 5);
-    const int gh = grid_for(h, L / HOT_SPAN + 1, 256 / s.lanes, 4);
+    const int gh = grid_for(h, L / HOT_MIN + 1, 256 / s.lanes, 4);
     dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
         constexpr int BITS = decltype(bc)::value, LANES = decltype(lc)::value;
         auto hot = k_hot_partial<LANES>;
         auto upd = k_update<BITS, LANES>;
         auto lst = k_update_list<BITS, LANES>;
-        LAUNCH(h, "hot_partial", hot, grid_for(h, L / HOT_SPAN + 1, 1, 4), 256, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
+        LAUNCH(h, "hot_partial", hot, grid_for(h, L / HOT_MIN + 1, 1, 1024 / (8 * LANES)), 8 * LANES, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
         static bool smem_set = false;     // one flag per instantiation of this lambda
         if (!smem_set) { cudaFuncSetAttribute(upd, cudaFuncAttributeMaxDynamicSharedMemorySize, UPD_SMEM); smem_set = true; }
         LAUNCH(h, "update", upd, gu, UPD_WARPS * 32, UPD_SMEM, s, w, d_grad_out, B, lr, (uint64_t)step);

@@ -8,6 +8,7 @@
 namespace mpe {
 
 constexpr int HOT_SPAN = 1024;        // occurrences covered by one multi-block gradient task (two tree levels)
+constexpr int HOT_MIN = 256;          // rows with more occurrences than this take the multi-block path
 constexpr int ERR_INDEX = 0, ERR_OFFSETS = 1;
 
 struct TableDev {
@@ -28,6 +29,8 @@ struct Counters {
     uint32_t hot_tasks;
     uint32_t abort;        // offsets were inconsistent: every later kernel of the step returns at once
     uint32_t deferred;     // newcomers that wait for the write-back of an updated row
+    uint32_t n_heads;      // cache sets that have miss candidates in this step
+    uint32_t upd_next;     // next block of 32 distinct rows to hand to a warp of k_update
     unsigned long long dropped;      // out-of-range indices in this batch
     unsigned long long err[2];       // sticky: ERR_INDEX, ERR_OFFSETS
 };
@@ -60,6 +63,7 @@ struct Work {
     int32_t* task_k;       // [hot tasks]
     int32_t* hot_k;        // [hot rows]
     int32_t* defer_k;      // [deferred newcomers]
+    int32_t* heads;        // [sets with candidates] position of the set's first candidate in the set-sorted list
     float* partial;        // [hot tasks][dim]
 };
 
@@ -69,7 +73,7 @@ struct Work {
 __global__ void k_prelude(Work w, const int32_t* __restrict__ offsets, int T, int B, uint32_t L) {
     if (threadIdx.x == 0 && blockIdx.x == 0) {
         Counters* c = w.ctr;
-        c->L = L; c->U = 0; c->hot_rows = 0; c->hot_tasks = 0; c->abort = 0; c->dropped = 0; c->deferred = 0;
+        c->L = L; c->U = 0; c->hot_rows = 0; c->hot_tasks = 0; c->abort = 0; c->dropped = 0; c->deferred = 0; c->n_heads = 0; c->upd_next = 0;
         bool bad = offsets[0] != 0 || offsets[(int64_t)T * B] != (int32_t)L;
         int32_t prev = 0;
         w.table_start[0] = 0;
@@ -180,30 +184,44 @@ __global__ void k_ustart(Work w, int T) {
 // ---------------------------------------------------------------------------------------------
 // cache tag lookup: one group of `ways` lanes per distinct row (Section 3 "Cache Structure")
 // ---------------------------------------------------------------------------------------------
-__global__ void k_probe(State s, Work w, uint32_t epoch) {
+__global__ void __launch_bounds__(256)
+k_probe(State s, Work w, uint32_t epoch) {
+    // A warp takes 32 consecutive distinct rows: lane l works out row l's set (32 rows at a time), then the
+    // warp compares the tags of 32/ways rows per round, `ways` lanes per row.
     if (w.ctr->abort) return;
-    const int ways = s.ways;
-    const int lane = threadIdx.x & 31, way = lane & (ways - 1);
+    const int ways = s.ways, G = 32 / ways;
+    const int lane = threadIdx.x & 31, way = lane & (ways - 1), grp = lane / ways;
     const uint32_t gmask = group_mask(ways);
     const int64_t U = w.ctr->U;
-    const int64_t gpb = blockDim.x / ways, ng = gpb * gridDim.x;
-    for (int64_t k = blockIdx.x * gpb + threadIdx.x / ways; k < U; k += ng) {
-        const int t = w.uniq_t[k];
-        const int32_t row = w.uniq_row[k];
-        const TableDev tb = s.tables[t];
-        int loc = LOC_MISS, set = 0;
-        if (row >= tb.N) loc = LOC_INVALID;
-        else if (tb.n_sets > 0) {
-            set = set_of((uint32_t)row, tb.salt, tb.n_sets);
-            const int64_t slot = (tb.set_base + set) * ways + way;
-            const bool match = s.tags[slot] == row;
-            const uint32_t hit = __ballot_sync(gmask, match) & gmask;
-            if (hit) {
-                loc = (int)((tb.set_base + set) * ways + (__ffs(hit) - 1 - (lane & ~(ways - 1))));
-                if (match) { s.hit_epoch[slot] = epoch; s.hit_k[slot] = (int32_t)k; }
-            }
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t k0 = ((int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 32; k0 < U; k0 += nwarps * 32) {
+        const int64_t k = k0 + lane;
+        int32_t row = 0, set = 0, gset = -1;         // gset: index of the row's set in the concatenated cache, -1 = no probe
+        int myloc = LOC_MISS;
+        if (k < U) {
+            const TableDev tb = s.tables[w.uniq_t[k]];
+            row = w.uniq_row[k];
+            if (row >= tb.N) myloc = LOC_INVALID;
+            else if (tb.n_sets > 0) { set = set_of((uint32_t)row, tb.salt, tb.n_sets); gset = (int32_t)(tb.set_base + set); }
         }
-        if (way == 0) { w.loc[k] = loc; w.final_loc[k] = loc; w.uset[k] = set; }
+#pragma unroll 4
+        for (int it = 0; it < ways; ++it) {            // 32 / G rounds
+            const int r = it * G + grp;               // the row this group looks at
+            const int32_t rgset = __shfl_sync(0xffffffffU, gset, r);
+            const int32_t rrow = __shfl_sync(0xffffffffU, row, r);
+            bool match = false;
+            int64_t slot = 0;
+            if (rgset >= 0) { slot = (int64_t)rgset * ways + way; match = s.tags[slot] == rrow; }
+            const uint32_t hit = __ballot_sync(0xffffffffU, match) & gmask;
+            int rloc = LOC_MISS;
+            if (hit) {
+                rloc = (int)((int64_t)rgset * ways + (__ffs(hit) - 1 - (lane & ~(ways - 1))));
+                if (match) { s.hit_epoch[slot] = epoch; s.hit_k[slot] = (int32_t)(k0 + r); }
+            }
+            const int got = __shfl_sync(0xffffffffU, rloc, (lane % G) * ways);   // result of the group that handled my row
+            if (lane / G == it && gset >= 0) myloc = got;
+        }
+        if (k < U) { w.loc[k] = myloc; w.final_loc[k] = myloc; w.uset[k] = set; }
     }
 }
 
@@ -238,37 +256,45 @@ __global__ void __launch_bounds__(256)
 k_pool(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int B,
        float* __restrict__ out) {
     constexpr int NB = LANES < 8 ? LANES : 8;
+    constexpr int dim = 4 * LANES;
     const int sub = threadIdx.x & (LANES - 1);
     const int gbase = (threadIdx.x & 31) & ~(LANES - 1);
     const uint32_t gmask = group_mask(LANES);
     const int64_t nbags = (int64_t)s.T * B;
     const int64_t gpb = blockDim.x / LANES, ng = gpb * gridDim.x;
     const bool abort = w.ctr->abort != 0;
+    const char* slab_col = reinterpret_cast<const char*>(s.slab) + 16 * sub;
     for (int64_t bag = blockIdx.x * gpb + threadIdx.x / LANES; bag < nbags; bag += ng) {
         const int t = (int)(bag / B);
         const int b = (int)(bag - (int64_t)t * B);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (!abort) {
-            const TableDev tb = s.tables[t];
+            const int64_t row_base = s.tables[t].row_base;
             const int32_t lo = offsets[bag], hi = offsets[bag + 1];
             for (int32_t p0 = lo; p0 < hi; p0 += LANES) {
                 const int n = min(LANES, hi - p0);
                 int myloc = LOC_INVALID; int32_t myrow = 0;
                 if (sub < n) { myloc = w.occ_loc[p0 + sub]; myrow = indices[p0 + sub]; }
                 for (int u0 = 0; u0 < n; u0 += NB) {
-                    float4 x[NB]; int lc[NB];
+                    float4 x[NB];
 #pragma unroll
                     for (int u = 0; u < NB; ++u) {
-                        lc[u] = __shfl_sync(gmask, myloc, gbase + u0 + u);
-                        const int32_t rw = __shfl_sync(gmask, myrow, gbase + u0 + u);
-                        if (u0 + u < n && lc[u] != LOC_INVALID) x[u] = fetch4<BITS, true>(s, tb, rw, lc[u], sub);
+                        const int lc = __shfl_sync(gmask, myloc, gbase + u0 + u);   // LOC_INVALID beyond the bag's end
+                        x[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (lc >= 0) {          // cache resident: the FP32 row
+                            x[u] = __ldg(reinterpret_cast<const float4*>(slab_col + (size_t)(uint32_t)lc * (size_t)(dim * 4)));
+                        } else if (lc == LOC_MISS) {   // up-convert the low-precision row
+                            const int32_t rw = __shfl_sync(gmask, myrow, gbase + u0 + u);
+                            x[u] = dequant4<BITS, true>(s.codes, s.sb, row_base + rw, dim, sub);
+                        }
                     }
+                    // rows are added in index order; an out-of-range index adds +0, which never changes the sum
 #pragma unroll
-                    for (int u = 0; u < NB; ++u) if (u0 + u < n && lc[u] != LOC_INVALID) acc = add4(acc, x[u]);
+                    for (int u = 0; u < NB; ++u) acc = add4(acc, x[u]);
                 }
             }
         }
-        reinterpret_cast<float4*>(out + ((int64_t)b * s.T + t) * s.dim)[sub] = acc;
+        reinterpret_cast<float4*>(out + ((int64_t)b * s.T + t) * dim)[sub] = acc;
     }
 }
 
@@ -300,7 +326,7 @@ __global__ void k_priority(State s, Work w, uint32_t step, uint32_t* __restrict_
                 }
                 if (loc >= 0) { hitm = mult; uh = 1; }
                 else if (tb.n_sets > 0) key = (uint32_t)w.uset[k];
-                if (mult > (uint32_t)HOT_SPAN) {
+                if (mult > (uint32_t)HOT_MIN) {
                     const uint32_t nt = (mult + HOT_SPAN - 1) / HOT_SPAN;
                     hb = (int)atomicAdd(&w.ctr->hot_tasks, nt);
                     w.hot_k[atomicAdd(&w.ctr->hot_rows, 1u)] = (int32_t)k;
@@ -338,6 +364,27 @@ __global__ void k_priority(State s, Work w, uint32_t step, uint32_t* __restrict_
 constexpr int VICTIM_NONE = -1;       // the way was empty, or the displaced row writes itself back
 constexpr int VICTIM_DEFER = -2;      // the displaced row was hit in this step: the newcomer waits for its write-back
 
+// the first candidate of every set that has any (the set-sorted list is grouped by table, then set)
+__global__ void k_policy_heads(State s, Work w, const uint32_t* __restrict__ ckey) {
+    if (w.ctr->abort) return;
+    const int64_t U = w.ctr->U;
+    const int64_t U32 = (U + 31) & ~31LL;
+    const int lane = threadIdx.x & 31;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < U32; j += (int64_t)gridDim.x * blockDim.x) {
+        bool head = false;
+        if (j < U) {
+            const uint32_t key = ckey[j];
+            const int t = find_segment(w.ustart, s.T, (int32_t)j);
+            head = key < (uint32_t)s.tables[t].n_sets && (j == w.ustart[t] || ckey[j - 1] != key);
+        }
+        const uint32_t m = __ballot_sync(0xffffffffU, head);
+        uint32_t base = 0;
+        if (lane == 0 && m) base = atomicAdd(&w.ctr->n_heads, (uint32_t)__popc(m));
+        base = __shfl_sync(0xffffffffU, base, 0);
+        if (head) w.heads[base + __popc(m & ((1u << lane) - 1u))] = (int32_t)j;
+    }
+}
+
 __global__ void __launch_bounds__(256)
 k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __restrict__ cval,
          uint32_t step, uint32_t epoch) {
@@ -345,14 +392,13 @@ k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __r
     const int ways = s.ways;
     const int lane = threadIdx.x & 31, way = lane & (ways - 1), gbase = lane & ~(ways - 1);
     const uint32_t gmask = group_mask(ways);
-    const int64_t U = w.ctr->U;
+    const int64_t nheads = w.ctr->n_heads;
     const int64_t gpb = blockDim.x / ways, ng = gpb * gridDim.x;
-    for (int64_t j = blockIdx.x * gpb + threadIdx.x / ways; j < U; j += ng) {
+    for (int64_t hi = blockIdx.x * gpb + threadIdx.x / ways; hi < nheads; hi += ng) {
+        const int64_t j = w.heads[hi];
         const uint32_t key = ckey[j];
-        const int t = w.uniq_t[cval[j]];
+        const int t = find_segment(w.ustart, s.T, (int32_t)j);
         const TableDev tb = s.tables[t];
-        if (key >= (uint32_t)tb.n_sets) continue;                       // not a candidate
-        if (j != w.ustart[t] && ckey[j - 1] == key) continue;           // not the first candidate of its set
         const int64_t slot = (tb.set_base + key) * ways + way;
         int32_t tag = s.tags[slot];
         uint32_t pri = 0;
@@ -375,20 +421,19 @@ k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __r
                 const int32_t row = __shfl_sync(gmask, crow, gbase + u);
                 const uint32_t pv = __shfl_sync(gmask, cpv, gbase + u);
                 // empty ways rank below every priority; ties go to the lowest way
-                const unsigned long long mine = tag < 0 ? (unsigned long long)way
-                                                        : ((((unsigned long long)pri + 1ULL) << 8) | (unsigned long long)way);
-                unsigned long long best = mine;
-                for (int o = ways >> 1; o > 0; o >>= 1) {
-                    const unsigned long long other = __shfl_xor_sync(gmask, best, o);
-                    best = other < best ? other : best;
+                const uint32_t empties = __ballot_sync(gmask, tag < 0) & gmask;
+                int jw; bool jempty; uint32_t jpri = 0;
+                if (empties) { jw = __ffs(empties) - 1 - gbase; jempty = true; }
+                else {
+                    jpri = __reduce_min_sync(gmask, pri);
+                    jw = __ffs(__ballot_sync(gmask, pri == jpri) & gmask) - 1 - gbase;
+                    jempty = false;
                 }
-                const int jw = (int)(best & 255ULL);
-                const unsigned long long jp = best >> 8;                   // 0 = empty, else PV[j] + 1
-                bool replace = jp == 0 || (unsigned long long)pv + 1ULL > jp;
+                bool replace = jempty || pv > jpri;
                 if (ways == 1 && s.policy == 0) replace = true;              // direct-mapped LRU never compares
                 if (replace) {
                     ++n_admit;
-                    if (jp != 0) ++n_evict;
+                    if (!jempty) ++n_evict;
                     if (way == jw) {
                         if (tag >= 0 && cand < 0) {
                             // a row that was resident when the step began leaves the cache
@@ -422,21 +467,42 @@ k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __r
 // ---------------------------------------------------------------------------------------------
 // backward 3: merged gradient of one distinct row (Section 5.1), radix-32 tree over index positions
 // ---------------------------------------------------------------------------------------------
-// up to 32 consecutive occurrences, added left to right; the group reads LANES sample ids at a time
+// up to 32 consecutive occurrences, added left to right; the group reads LANES sample ids at a time.
+// gcol points at the group's lane-th float4 of column block t; stride_bytes is the size of one sample's row of grad_out.
 template <int LANES>
-__device__ __forceinline__ float4 sum_chunk(const int32_t* __restrict__ occ_b, const float* __restrict__ grad, int64_t col,
-                                            int64_t stride, int32_t first, int len, uint32_t gmask, int gbase, int sub) {
+__device__ __forceinline__ float4 sum_chunk(const int32_t* __restrict__ occ_b, const char* __restrict__ gcol, uint32_t stride_bytes,
+                                            int32_t first, int len, uint32_t gmask, int gbase, int sub) {
     constexpr int NB = LANES < 8 ? LANES : 8;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 acc;
+    if (LANES == 32 && len == 32) {       // a full chunk handled by a whole warp: no bounds to check
+        const uint32_t myb = (uint32_t)occ_b[first + sub];
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            v[u] = __ldg(reinterpret_cast<const float4*>(gcol + (size_t)__shfl_sync(0xffffffffU, myb, u) * stride_bytes));
+        acc = v[0];
+#pragma unroll
+        for (int u = 1; u < 8; ++u) acc = add4(acc, v[u]);
+#pragma unroll
+        for (int u0 = 8; u0 < 32; u0 += 8) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                v[u] = __ldg(reinterpret_cast<const float4*>(gcol + (size_t)__shfl_sync(0xffffffffU, myb, u0 + u) * stride_bytes));
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc = add4(acc, v[u]);
+        }
+        return acc;
+    }
+    acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int j0 = 0; j0 < len; j0 += LANES) {
         const int n = min(LANES, len - j0);
-        const int32_t myb = sub < n ? occ_b[first + j0 + sub] : 0;
+        const uint32_t myb = sub < n ? (uint32_t)occ_b[first + j0 + sub] : 0u;
         for (int u0 = 0; u0 < n; u0 += NB) {
             float4 v[NB];
 #pragma unroll
             for (int u = 0; u < NB; ++u) {
-                const int32_t b = __shfl_sync(gmask, myb, gbase + u0 + u);
-                if (u0 + u < n) v[u] = __ldg(reinterpret_cast<const float4*>(grad + (int64_t)b * stride + col));
+                const uint32_t b = __shfl_sync(gmask, myb, gbase + u0 + u);
+                if (u0 + u < n) v[u] = __ldg(reinterpret_cast<const float4*>(gcol + (size_t)b * stride_bytes));
             }
 #pragma unroll
             for (int u = 0; u < NB; ++u)
@@ -464,8 +530,9 @@ __device__ __forceinline__ float4 tree_reduce(const Term& term, int64_t first, i
 }
 
 // rows with more than HOT_SPAN occurrences: one block per HOT_SPAN occurrences computes two tree levels
+// (8 groups of LANES lanes share the 32 chunks of a task)
 template <int LANES>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(8 * LANES)
 k_hot_partial(State s, Work w, const float* __restrict__ grad, int B) {
     extern __shared__ float chunk_sums[];     // [32][dim]
     if (w.ctr->abort) return;
@@ -474,16 +541,16 @@ k_hot_partial(State s, Work w, const float* __restrict__ grad, int B) {
     const int gbase = (threadIdx.x & 31) & ~(LANES - 1);
     const uint32_t gmask = group_mask(LANES);
     const uint32_t ntask = w.ctr->hot_tasks;
-    const int64_t stride = (int64_t)s.T * dim;
+    const uint32_t stride_bytes = (uint32_t)s.T * (uint32_t)dim * 4u;
     for (uint32_t task = blockIdx.x; task < ntask; task += gridDim.x) {
         const int32_t k = w.task_k[task];
         const int32_t j = (int32_t)task - w.hot_base[k];
         const int32_t first = w.seg[k] + j * HOT_SPAN;
         const int32_t n = min(HOT_SPAN, w.seg[k + 1] - first);
         const int nchunk = (n + 31) >> 5;
-        const int64_t col = (int64_t)w.uniq_t[k] * dim + 4 * sub;
+        const char* gcol = reinterpret_cast<const char*>(grad + (int64_t)w.uniq_t[k] * dim + 4 * sub);
         for (int c = grp; c < nchunk; c += ngrp) {
-            const float4 v = sum_chunk<LANES>(w.occ_b, grad, col, stride, first + 32 * c, min(32, n - 32 * c), gmask, gbase, sub);
+            const float4 v = sum_chunk<LANES>(w.occ_b, gcol, stride_bytes, first + 32 * c, min(32, n - 32 * c), gmask, gbase, sub);
             reinterpret_cast<float4*>(chunk_sums + c * dim)[sub] = v;
         }
         __syncthreads();
@@ -571,11 +638,14 @@ k_update(State s, Work w, const float* __restrict__ grad, int B, float lr, uint6
     float4* ring = reinterpret_cast<float4*>(upd_smem) + ((warp * G + grp) * UPD_RING) * LANES + sub;   // slot i: ring[i * LANES]
     int32_t(*meta)[UPD_META] = reinterpret_cast<int32_t(*)[UPD_META]>(upd_smem + UPD_WARPS * UPD_RING * 32 * 16) + warp * 32;
     const int64_t U = w.ctr->U;
-    const int64_t nwarps = (int64_t)gridDim.x * UPD_WARPS;
-    const int64_t stride = (int64_t)s.T * dim;
-    const float* gcol = grad + 4 * sub;
-    for (int64_t k0 = ((int64_t)blockIdx.x * UPD_WARPS + warp) * 32; k0 < U; k0 += nwarps * 32) {
-        __syncwarp();
+    const uint32_t stride_bytes = (uint32_t)s.T * (uint32_t)dim * 4u;
+    const char* gcol = reinterpret_cast<const char*>(grad + 4 * sub);
+    for (;;) {
+        // blocks of 32 rows are handed out on demand: their cost varies with the rows' multiplicities
+        uint32_t blk = 0;
+        if (lane == 0) blk = atomicAdd(&w.ctr->upd_next, 1u);
+        const int64_t k0 = (int64_t)__shfl_sync(0xffffffffU, blk, 0) * 32;
+        if (k0 >= U) break;
         const int64_t k = k0 + lane;
         if (k < U) {
             const int32_t first = w.seg[k], row = w.uniq_row[k];
@@ -645,11 +715,11 @@ k_update(State s, Work w, const float* __restrict__ grad, int B, float lr, uint6
         float4 chunkacc = make_float4(0.f, 0.f, 0.f, 0.f), rowacc = chunkacc;
         while (cr < nrow) {
             while (inflight < UPD_GROUPS && pr < nrow) {
-                const float* src = gcol + meta[pr][M_COL];
+                const char* src = gcol + (size_t)(uint32_t)meta[pr][M_COL] * 4u;
 #pragma unroll
                 for (int u = 0; u < NB; ++u) {
-                    const int32_t b = __shfl_sync(gmask, nb, gbase + u);
-                    if (u < ncnt) cp_async16(ring + ((head + u) & (UPD_RING - 1)) * LANES, src + (int64_t)b * stride);
+                    const uint32_t b = (uint32_t)__shfl_sync(gmask, nb, gbase + u);
+                    if (u < ncnt) cp_async16(ring + ((head + u) & (UPD_RING - 1)) * LANES, src + (size_t)b * stride_bytes);
                 }
                 cp_async_commit();
                 head += ncnt; ++inflight; po += ncnt;
@@ -725,7 +795,7 @@ k_update_list(State s, Work w, const float* __restrict__ grad, int B, float lr, 
     const uint32_t gmask = group_mask(LANES);
     const int64_t n = *count;
     const int64_t gpb = blockDim.x / LANES, ng = gpb * gridDim.x;
-    const int64_t stride = (int64_t)s.T * dim;
+    const uint32_t stride_bytes = (uint32_t)s.T * (uint32_t)dim * 4u;
     for (int64_t i = blockIdx.x * gpb + threadIdx.x / LANES; i < n; i += ng) {
         const int32_t k = list[i];
         const int loc = w.loc[k], floc = w.final_loc[k];
@@ -736,14 +806,14 @@ k_update_list(State s, Work w, const float* __restrict__ grad, int B, float lr, 
         const int32_t row = w.uniq_row[k];
         const TableDev tb = s.tables[t];
         const int32_t first = w.seg[k], m = w.seg[k + 1] - first;
-        const int64_t col = (int64_t)t * dim + 4 * sub;
+        const char* gcol = reinterpret_cast<const char*>(grad + (int64_t)t * dim + 4 * sub);
         const float4 x = fetch4<BITS, false>(s, tb, row, loc, sub);
         float4 g;
         const int hb = w.hot_base[k];
         if (hb < 0) {
-            g = sum_chunk<LANES>(w.occ_b, grad, col, stride, first, min(32, m), gmask, gbase, sub);
+            g = sum_chunk<LANES>(w.occ_b, gcol, stride_bytes, first, min(32, m), gmask, gbase, sub);
             for (int32_t c = 32; c < m; c += 32)
-                g = add4(g, sum_chunk<LANES>(w.occ_b, grad, col, stride, first + c, min(32, m - c), gmask, gbase, sub));
+                g = add4(g, sum_chunk<LANES>(w.occ_b, gcol, stride_bytes, first + c, min(32, m - c), gmask, gbase, sub));
         } else {
             const float* part = w.partial + (int64_t)hb * dim + 4 * sub;
             auto term = [&](int64_t j) { return *reinterpret_cast<const float4*>(part + j * dim); };

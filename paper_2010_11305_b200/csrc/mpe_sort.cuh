@@ -102,7 +102,7 @@ k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_s
 
 // ---- pass 3 of 3: stable scatter ------------------------------------------------
 // vals_in == nullptr means "the payload is the element's position" (first pass).
-__global__ void __launch_bounds__(SORT_THREADS)
+__global__ void __launch_bounds__(SORT_THREADS, 3)
 k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
                uint32_t* __restrict__ keys_out, uint32_t* __restrict__ vals_out,
                const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base, int T, int shift,
@@ -127,19 +127,20 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict_
         __syncthreads();
         // warp w owns elements [w*512, w*512+512) of the tile, item i of lane l is w*512 + i*32 + l,
         // so "item order, then lane order" is the original order
-        uint32_t key[SORT_ITEMS], val[SORT_ITEMS], rank[SORT_ITEMS];
+        uint32_t key[SORT_ITEMS], rank[SORT_ITEMS];
 #pragma unroll
         for (int i = 0; i < SORT_ITEMS; ++i) {
             const int e = warp * (32 * SORT_ITEMS) + i * 32 + lane;
-            const bool ok = e < count;
-            key[i] = ok ? keys_in[start + e] : 0xffffffffU;
-            val[i] = ok ? (vals_in ? vals_in[start + e] : (uint32_t)(start + e)) : 0u;
+            key[i] = e < count ? keys_in[start + e] : 0xffffffffU;
+        }
+#pragma unroll
+        for (int i = 0; i < SORT_ITEMS; ++i) {
             const uint32_t dg = (key[i] >> shift) & 255u;
             const uint32_t peers = __match_any_sync(0xffffffffU, dg);
-            const uint32_t before = wcnt[warp][dg];
-            __syncwarp();
-            if ((peers & ((1u << lane) - 1u)) == 0) wcnt[warp][dg] = before + __popc(peers);
-            __syncwarp();
+            const int leader = __ffs(peers) - 1;
+            uint32_t before = 0;
+            if (lane == leader) before = atomicAdd(&wcnt[warp][dg], (uint32_t)__popc(peers));   // one lane per digit value
+            before = __shfl_sync(0xffffffffU, before, leader);
             rank[i] = before + __popc(peers & ((1u << lane) - 1u));
         }
         __syncthreads();
@@ -153,10 +154,11 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict_
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < SORT_ITEMS; ++i) {
+            const int e = warp * (32 * SORT_ITEMS) + i * 32 + lane;
             const uint32_t dg = (key[i] >> shift) & 255u;
             const uint32_t pos = dstart[dg] + wcnt[warp][dg] + rank[i];
             skey[pos] = key[i];
-            sval[pos] = val[i];
+            sval[pos] = e < count ? (vals_in ? vals_in[start + e] : (uint32_t)(start + e)) : 0u;
         }
         __syncthreads();
         // padding keys (0xffffffff, digit 255) follow every real key of the tile, so positions [0,count) are real
