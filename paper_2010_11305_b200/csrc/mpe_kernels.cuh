@@ -255,7 +255,7 @@ template <int BITS, int LANES>
 __global__ void __launch_bounds__(256)
 k_pool(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int B,
        float* __restrict__ out) {
-    constexpr int NB = LANES < 8 ? LANES : 8;
+    constexpr int NB = LANES < 4 ? LANES : 4;        // rows per batch; two batches are in flight
     constexpr int dim = 4 * LANES;
     const int sub = threadIdx.x & (LANES - 1);
     const int gbase = (threadIdx.x & 31) & ~(LANES - 1);
@@ -264,33 +264,60 @@ k_pool(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __re
     const int64_t gpb = blockDim.x / LANES, ng = gpb * gridDim.x;
     const bool abort = w.ctr->abort != 0;
     const char* slab_col = reinterpret_cast<const char*>(s.slab) + 16 * sub;
-    for (int64_t bag = blockIdx.x * gpb + threadIdx.x / LANES; bag < nbags; bag += ng) {
+    int64_t bag = blockIdx.x * gpb + threadIdx.x / LANES;
+    // (slot, row id) of the first LANES indices of a bag, one per lane; fetched one bag ahead
+    int32_t lo = 0, hi = 0; int wloc = LOC_INVALID; int32_t wrow = 0;
+    auto open_bag = [&](int64_t bg) {
+        wloc = LOC_INVALID;
+        if (bg < nbags && !abort) {
+            lo = offsets[bg]; hi = offsets[bg + 1];
+            if (lo + sub < hi) { wloc = w.occ_loc[lo + sub]; wrow = indices[lo + sub]; }
+        } else { lo = hi = 0; }
+    };
+    open_bag(bag);
+    for (; bag < nbags; bag += ng) {
         const int t = (int)(bag / B);
         const int b = (int)(bag - (int64_t)t * B);
+        const int64_t row_base = s.tables[t].row_base;
+        const int32_t clo = lo, chi = hi;
+        int myloc = wloc; int32_t myrow = wrow;
+        open_bag(bag + ng);                           // the next bag's first window is on its way while this one is pooled
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (!abort) {
-            const int64_t row_base = s.tables[t].row_base;
-            const int32_t lo = offsets[bag], hi = offsets[bag + 1];
-            for (int32_t p0 = lo; p0 < hi; p0 += LANES) {
-                const int n = min(LANES, hi - p0);
-                int myloc = LOC_INVALID; int32_t myrow = 0;
-                if (sub < n) { myloc = w.occ_loc[p0 + sub]; myrow = indices[p0 + sub]; }
-                for (int u0 = 0; u0 < n; u0 += NB) {
-                    float4 x[NB];
+        // one row: cache resident -> the FP32 row; uncached -> up-convert the codes; out of range -> +0 (never changes the sum)
+        auto fetch = [&](int src_lane) {
+            const int lc = __shfl_sync(gmask, myloc, gbase + src_lane);
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (lc >= 0) {
+                x = __ldg(reinterpret_cast<const float4*>(slab_col + (size_t)(uint32_t)lc * (size_t)(dim * 4)));
+            } else if (lc == LOC_MISS) {
+                const int32_t rw = __shfl_sync(gmask, myrow, gbase + src_lane);
+                x = dequant4<BITS, true>(s.codes, s.sb, row_base + rw, dim, sub);
+            }
+            return x;
+        };
+        for (int32_t p0 = clo; p0 < chi; p0 += LANES) {
+            if (p0 > clo) {                           // later windows of a long bag
+                myloc = LOC_INVALID;
+                if (p0 + sub < chi) { myloc = w.occ_loc[p0 + sub]; myrow = indices[p0 + sub]; }
+            }
+            const int n = min(LANES, chi - p0);
+            float4 xa[NB], xb[NB];
 #pragma unroll
-                    for (int u = 0; u < NB; ++u) {
-                        const int lc = __shfl_sync(gmask, myloc, gbase + u0 + u);   // LOC_INVALID beyond the bag's end
-                        x[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (lc >= 0) {          // cache resident: the FP32 row
-                            x[u] = __ldg(reinterpret_cast<const float4*>(slab_col + (size_t)(uint32_t)lc * (size_t)(dim * 4)));
-                        } else if (lc == LOC_MISS) {   // up-convert the low-precision row
-                            const int32_t rw = __shfl_sync(gmask, myrow, gbase + u0 + u);
-                            x[u] = dequant4<BITS, true>(s.codes, s.sb, row_base + rw, dim, sub);
-                        }
+            for (int u = 0; u < NB; ++u) xa[u] = fetch(u);
+            for (int u0 = 0; u0 < n; u0 += 2 * NB) {  // rows are added in index order
+                if (u0 + NB < n) {
+#pragma unroll
+                    for (int u = 0; u < NB; ++u) xb[u] = fetch((u0 + NB + u) & (LANES - 1));
+                }
+#pragma unroll
+                for (int u = 0; u < NB; ++u) acc = add4(acc, xa[u]);
+                if (u0 + NB < n) {
+                    if (u0 + 2 * NB < n) {
+#pragma unroll
+                        for (int u = 0; u < NB; ++u) xa[u] = fetch((u0 + 2 * NB + u) & (LANES - 1));
                     }
-                    // rows are added in index order; an out-of-range index adds +0, which never changes the sum
 #pragma unroll
-                    for (int u = 0; u < NB; ++u) acc = add4(acc, x[u]);
+                    for (int u = 0; u < NB; ++u) acc = add4(acc, xb[u]);
                 }
             }
         }
@@ -597,15 +624,6 @@ __device__ __forceinline__ void apply_update(const State& s, const TableDev& tb,
                                    rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)row, step));
     }
 }
-
-// ---- asynchronous 16-byte copies global -> shared (per thread; completion is waited for by group count) ----
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
-    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
