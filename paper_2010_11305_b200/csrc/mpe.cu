@@ -43,6 +43,8 @@ struct mpe_handle {
     int64_t sh_cap_L = 0, sh_cap_off = 0, sh_cap_out = 0;
     // step state
     cudaStream_t stream = nullptr;
+    cudaStream_t side = nullptr;            // runs the hot rows' partial sums next to the policy kernels
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     bool have_forward = false;
     int64_t last_step = 0;
     uint64_t steps = 0;
@@ -80,16 +82,17 @@ int prof_name(mpe_handle* h, const char* name) {
 }
 
 struct LaunchScope {
-    mpe_handle* h; ProfRec rec{};
-    LaunchScope(mpe_handle* h_, const char* name) : h(h_) {
+    mpe_handle* h; cudaStream_t st; ProfRec rec{};
+    LaunchScope(mpe_handle* h_, const char* name, cudaStream_t st_) : h(h_), st(st_) {
         ++h->launches;
-        if (h->profiling) { rec.name = prof_name(h, name); rec.a = get_event(h); rec.b = get_event(h); cudaEventRecord(rec.a, h->stream); }
+        if (h->profiling) { rec.name = prof_name(h, name); rec.a = get_event(h); rec.b = get_event(h); cudaEventRecord(rec.a, st); }
     }
-    ~LaunchScope() { if (h->profiling) { cudaEventRecord(rec.b, h->stream); h->prof_recs.push_back(rec); } }
+    ~LaunchScope() { if (h->profiling) { cudaEventRecord(rec.b, st); h->prof_recs.push_back(rec); } }
 };
 
-#define LAUNCH(h, name, kern, grid, block, smem, ...) \
-    do { LaunchScope ls_(h, name); kern<<<(grid), (block), (smem), (h)->stream>>>(__VA_ARGS__); } while (0)
+#define LAUNCH_ON(h, st, name, kern, grid, block, smem, ...) \
+    do { LaunchScope ls_(h, name, st); kern<<<(grid), (block), (smem), (st)>>>(__VA_ARGS__); } while (0)
+#define LAUNCH(h, name, kern, grid, block, smem, ...) LAUNCH_ON(h, (h)->stream, name, kern, grid, block, smem, __VA_ARGS__)
 
 int grid_for(const mpe_handle* h, int64_t work_items, int64_t items_per_block, int blocks_per_sm) {
     int64_t need = (work_items + items_per_block - 1) / items_per_block;
@@ -145,7 +148,7 @@ int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
 void scan_u32(mpe_handle* h, uint32_t* data, const uint32_t* n_ptr, int64_t n_upper) {
     const int g = grid_for(h, n_upper, SCAN_TILE, 8);
     LAUNCH(h, "scan_reduce", k_scan_reduce, g, SCAN_THREADS, 0, data, n_ptr, h->block_sums);
-    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, 1024, 0, h->block_sums, n_ptr, (uint32_t)SCAN_TILE, (uint32_t*)nullptr);
+    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, n_ptr, (uint32_t)SCAN_TILE, (uint32_t*)nullptr);
     LAUNCH(h, "scan_apply", k_scan_apply, g, SCAN_THREADS, 0, data, n_ptr, (const uint32_t*)h->block_sums);
 }
 
@@ -235,6 +238,9 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
     h->device = device;
     DeviceGuard guard(device);
     cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, device);
+    if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess) { delete h; return MPE_ERR_CUDA; }
     h->T = num_tables; h->dim = dim; h->bits = bits; h->ways = ways; h->policy = policy; h->optimizer = optimizer;
     h->code_bytes = dim * bits / 8; h->eps = eps; h->lo = init_lo; h->hi = init_hi; h->seed = seed;
     h->tables.resize(num_tables);
@@ -334,7 +340,7 @@ int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offset
     // distinct rows
     const int gs = grid_for(h, total_indices, SCAN_TILE, 8);
     LAUNCH(h, "unique_count", k_unique<false>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
-    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, 1024, 0, h->block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);
+    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);
     LAUNCH(h, "unique_write", k_unique<true>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
     LAUNCH(h, "ustart", k_ustart, 1, 256, 0, w, T);
     // tag lookup, then fetch + pool
@@ -363,6 +369,16 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
     const int64_t L = h->L;
     const int B = h->B;
 
+    // the hot rows' partial gradient sums only need the sorted batch: they run on a second stream next to the
+    // priority / candidate-sort / policy kernels, which leave most of the machine idle
+    CK(h, cudaEventRecord(h->ev_fork, h->stream));
+    CK(h, cudaStreamWaitEvent(h->side, h->ev_fork, 0));
+    dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
+        constexpr int LANES = decltype(lc)::value;
+        auto hot = k_hot_partial<LANES>;
+        LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, L / HOT_MIN + 1, 1, 2), 8 * LANES, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
+    });
+    CK(h, cudaEventRecord(h->ev_join, h->side));
     LAUNCH(h, "priority", k_priority, grid_for(h, L, 256, 8), 256, 0, s, w, (uint32_t)step, h->ckeyA);
     if (h->max_sets > 0) {
         // group the rows that missed by cache set, keeping ascending row id inside a set
@@ -378,13 +394,12 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
     const int gh = grid_for(h, L / HOT_MIN + 1, 256 / s.lanes, 4);
     dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
         constexpr int BITS = decltype(bc)::value, LANES = decltype(lc)::value;
-        auto hot = k_hot_partial<LANES>;
         auto upd = k_update<BITS, LANES>;
         auto lst = k_update_list<BITS, LANES>;
-        LAUNCH(h, "hot_partial", hot, grid_for(h, L / HOT_MIN + 1, 1, 1024 / (8 * LANES)), 8 * LANES, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
         static bool smem_set = false;     // one flag per instantiation of this lambda
         if (!smem_set) { cudaFuncSetAttribute(upd, cudaFuncAttributeMaxDynamicSharedMemorySize, UPD_SMEM); smem_set = true; }
         LAUNCH(h, "update", upd, gu, UPD_WARPS * 32, UPD_SMEM, s, w, d_grad_out, B, lr, (uint64_t)step);
+        cudaStreamWaitEvent(h->stream, h->ev_join, 0);
         LAUNCH(h, "update_hot", lst, gh, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step, (const int32_t*)w.hot_k,
                (const uint32_t*)&w.ctr->hot_rows, 0);
         if (h->max_sets > 0)
@@ -448,6 +463,9 @@ int mpe_destroy(mpe_handle* h) {
     if (!h) return MPE_ERR_ARG;
     DeviceGuard guard(h->device);
     cudaStreamSynchronize(h->stream);
+    if (h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); }
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
     free_workspace(h);
     State& s = h->st;
     cudaFree(h->d_tables); cudaFree(s.codes); cudaFree(s.sb); cudaFree(s.cnt); cudaFree(s.G); cudaFree(s.slab);

@@ -221,7 +221,19 @@ k_probe(State s, Work w, uint32_t epoch) {
             const int got = __shfl_sync(0xffffffffU, rloc, (lane % G) * ways);   // result of the group that handled my row
             if (lane / G == it && gset >= 0) myloc = got;
         }
-        if (k < U) { w.loc[k] = myloc; w.final_loc[k] = myloc; w.uset[k] = set; }
+        if (k < U) {
+            w.loc[k] = myloc; w.final_loc[k] = myloc; w.uset[k] = set;
+            // rows with very many occurrences get their gradient summed by whole blocks, HOT_SPAN occurrences per task
+            int hb = -1;
+            const uint32_t mult = (uint32_t)(w.seg[k + 1] - w.seg[k]);
+            if (myloc != LOC_INVALID && mult > (uint32_t)HOT_MIN) {
+                const uint32_t nt = (mult + HOT_SPAN - 1) / HOT_SPAN;
+                hb = (int)atomicAdd(&w.ctr->hot_tasks, nt);
+                w.hot_k[atomicAdd(&w.ctr->hot_rows, 1u)] = (int32_t)k;
+                for (uint32_t j = 0; j < nt; ++j) w.task_k[hb + j] = (int32_t)k;
+            }
+            w.hot_base[k] = hb;
+        }
     }
 }
 
@@ -341,7 +353,6 @@ __global__ void k_priority(State s, Work w, uint32_t step, uint32_t* __restrict_
             const int loc = w.loc[k];
             const uint32_t mult = (uint32_t)(w.seg[k + 1] - w.seg[k]);
             uint32_t key = (uint32_t)tb.n_sets;              // sorts behind every real set: not a candidate
-            int hb = -1;
             if (loc != LOC_INVALID) {
                 m = mult; un = 1;
                 if (s.policy == 1) {                         // LFU: access count of the row, saturating
@@ -353,15 +364,8 @@ __global__ void k_priority(State s, Work w, uint32_t step, uint32_t* __restrict_
                 }
                 if (loc >= 0) { hitm = mult; uh = 1; }
                 else if (tb.n_sets > 0) key = (uint32_t)w.uset[k];
-                if (mult > (uint32_t)HOT_MIN) {
-                    const uint32_t nt = (mult + HOT_SPAN - 1) / HOT_SPAN;
-                    hb = (int)atomicAdd(&w.ctr->hot_tasks, nt);
-                    w.hot_k[atomicAdd(&w.ctr->hot_rows, 1u)] = (int32_t)k;
-                    for (uint32_t j = 0; j < nt; ++j) w.task_k[hb + j] = (int32_t)k;
-                }
             }
             ckey[k] = key;
-            w.hot_base[k] = hb;
         }
         // counters: one atomic per warp when the warp sits inside one table
         const int t0 = __shfl_sync(0xffffffffU, t, 0);

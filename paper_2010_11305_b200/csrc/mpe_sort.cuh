@@ -190,20 +190,25 @@ k_scan_reduce(const uint32_t* __restrict__ in, const uint32_t* __restrict__ n_pt
     }
 }
 
-// one block: exclusive scan of block_sums[0..nblk) in place; the grand total goes to *total_out
-__global__ void __launch_bounds__(1024)
+// one small block (it has to fit next to whatever else is resident): exclusive scan of block_sums[0..nblk) in place;
+// the grand total goes to *total_out
+constexpr int BSUM_THREADS = 256;
+__global__ void __launch_bounds__(BSUM_THREADS)
 k_scan_block_sums(uint32_t* __restrict__ block_sums, const uint32_t* __restrict__ n_ptr, uint32_t tile,
                   uint32_t* __restrict__ total_out) {
-    __shared__ uint32_t tmp[1024 / 32 + 1];
+    __shared__ uint32_t tmp[BSUM_THREADS / 32 + 1];
     const uint32_t n = *n_ptr;
     const uint32_t nblk = (n + tile - 1) / tile;
     uint32_t carry = 0;
-    for (uint32_t base = 0; base < nblk; base += 1024) {
-        const uint32_t i = base + threadIdx.x;
-        const uint32_t v = i < nblk ? block_sums[i] : 0;
+    for (uint32_t base = 0; base < nblk; base += BSUM_THREADS * 4) {
+        const uint32_t i = base + threadIdx.x * 4;
+        uint32_t v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) v[q] = i + q < nblk ? block_sums[i + q] : 0;
         uint32_t total;
-        const uint32_t ex = block_exclusive_scan<1024>(v, &total, tmp);
-        if (i < nblk) block_sums[i] = carry + ex;
+        uint32_t ex = carry + block_exclusive_scan<BSUM_THREADS>(v[0] + v[1] + v[2] + v[3], &total, tmp);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { if (i + q < nblk) block_sums[i + q] = ex; ex += v[q]; }
         carry += total;
     }
     if (threadIdx.x == 0 && total_out) *total_out = carry;
