@@ -31,6 +31,9 @@ from paper_2010_11305_b200 import workloads as wl  # noqa: E402
 
 METRIC = "embedding rows/sec per training step (fwd+bwd+cache) and % of 8 TB/s HBM"
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum per index of the batch, from the ncu capture summarised in
+# profiles/k_update_cfg4_8tables.md (8 of the 64 tables; traffic grows in proportion to the indices processed)
+NCU_DRAM_BYTES_PER_INDEX = {"update": 99.6}
 
 
 def measured_peaks():
@@ -92,29 +95,43 @@ def describe(cfg):
             f"cache {cfg.cache_fraction:g} x rows, {cfg.ways or 32}-way {pol}, batch {cfg.batch}, bags {cfg.bag}, {opt}")
 
 
-def byte_model(cfg, L, U, U_hit, occ_hit, admissions, evictions, passes_main, passes_cand):
-    """Algorithmic bytes of one step, per kernel (what the method itself has to move, counted per access)."""
+def byte_model(cfg, L, U, U_hit, occ_hit, admissions, evictions, hot_occ, passes_main, passes_cand):
+    """Algorithmic bytes of one step, counted per access (the paper's effective-bandwidth numerator).
+
+    Returns (step_bytes, per_kernel).  step_bytes is what the METHOD has to move: per index 4 B of id plus the
+    fetched row (FP32 row on a hit, codes + scale + bias on a miss), the pooled output, one gradient row per
+    index, per distinct row a read and a write of its home (FP32 row or quantized row), the priority update,
+    the optimizer state, evictions (FP32 read + quantized write) and admissions (FP32 write), and the
+    de-duplication minimum 8 L + 4 U.  per_kernel adds the bookkeeping arrays each kernel of this
+    implementation touches; it is the numerator of the per-kernel roofline figure.
+    """
     d, T, B = cfg.dim, cfg.num_tables, cfg.batch
     rb = d * cfg.bits // 8 + 8      # codes + FP32 scale + FP32 bias
     fb = 4 * d
     occ_miss, U_miss = L - occ_hit, U - U_hit
     out_bytes = 4 * B * T * d
+    pv = (8 * U) if cfg.policy == wl.LFU else (4 * U_hit)
+    opt = (8 * U) if cfg.optimizer == wl.ROWWISE_ADAGRAD else 0
+    fwd = 4 * L + occ_hit * fb + occ_miss * rb + out_bytes
+    bwd = L * fb + U_hit * 2 * fb + U_miss * 2 * rb + pv + opt + evictions * (fb + rb) + admissions * fb
+    dedup = 8 * L + 4 * U
+    step = fwd + bwd + dedup
     m = {}
     m["make_keys"] = 4 * L + 4 * T * B + 8 * L
     m["sort_hist"] = passes_main * 4 * L + passes_cand * 4 * U
     m["sort_scatter"] = passes_main * 16 * L + passes_cand * 16 * U
     m["unique_count"] = 4 * L
     m["unique_write"] = 8 * L + 12 * U
-    m["probe"] = 8 * U + 4 * cfg.ways * U + 12 * U
+    m["probe"] = 8 * U + 4 * cfg.ways * U + 16 * U
     m["broadcast"] = 20 * L
     m["pool"] = 8 * L + occ_hit * fb + occ_miss * rb + out_bytes
-    m["priority"] = 16 * U + (8 * U if cfg.policy == wl.LFU else 4 * U_hit) + 8 * U
+    m["priority"] = 16 * U + pv + 4 * U
+    m["policy_heads"] = 4 * U
     m["policy"] = U_miss * (8 + 4 + (4 if cfg.policy == wl.LFU else 0) + 8) + admissions * 8 * cfg.ways
-    grad_bytes = L * (fb + 4)
-    m["update"] = grad_bytes + 32 * U + U_hit * 2 * fb + (U_miss - admissions) * 2 * rb + admissions * (rb + fb) + evictions * (fb + rb)
-    if cfg.optimizer == wl.ROWWISE_ADAGRAD:
-        m["update"] += 8 * U
-    return m
+    m["hot_partial"] = hot_occ * (fb + 4)
+    m["update"] = (L - hot_occ) * (fb + 4) + 32 * U + U_hit * 2 * fb + (U_miss - admissions) * 2 * rb + admissions * (rb + fb) \
+        + evictions * (fb + rb) + opt
+    return step, m
 
 
 def run_ours(args, cfg, rank, world, local_rank):
@@ -172,6 +189,7 @@ def run_ours(args, cfg, rank, world, local_rank):
     ds = stats1 - stats0
     K = args.steps
     L, occ_hit, U, U_hit, adm, evi = (ds[i] / K for i in (0, 1, 2, 3, 4, 5))
+    hot_rows, hot_occ = float(h.step_info()[3]), float(h.step_info()[4])      # of the last timed step
 
     # end to end through the host-buffer entry point: pinned host inputs, H2D + step + D2H inside the timed region
     h_batches = []
@@ -205,8 +223,8 @@ def run_ours(args, cfg, rank, world, local_rank):
     passes_main = (max(cfg.num_rows).bit_length() + 7) // 8
     max_sets = max(h.cache_geometry(t)[0] for t in range(cfg.num_tables))
     passes_cand = (max(max_sets, 1).bit_length() + 7) // 8 if max_sets else 0
-    model = byte_model(cfg, L, U, U_hit, occ_hit, adm, evi, passes_main, passes_cand)
-    step_bytes = float(sum(model.values()))
+    step_bytes, model = byte_model(cfg, L, U, U_hit, occ_hit, adm, evi, hot_occ, passes_main, passes_cand)
+    step_bytes = float(step_bytes)
     ms_step = ms / K
     top = max(prof.items(), key=lambda kv: kv[1][0]) if prof else (None, (0.0, 0))
     peak, peak_kind = measured_peaks()
@@ -218,7 +236,9 @@ def run_ours(args, cfg, rank, world, local_rank):
         bytes_per_launch = model.get(name, 0.0) / max(launches_per_step, 1e-9)
         achieved = bytes_per_launch / (per_launch_ms * 1e-3) / 1e9 if per_launch_ms > 0 else 0.0
         roof = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None, "bytes_per_launch": bytes_per_launch, "ms_per_launch": per_launch_ms,
+                "frac": achieved / peak,
+                "traffic": NCU_DRAM_BYTES_PER_INDEX[name] * L / max(launches_per_step, 1e-9) if name in NCU_DRAM_BYTES_PER_INDEX and args.config == 4 else None,
+                "bytes_per_launch": bytes_per_launch, "ms_per_launch": per_launch_ms,
                 "share_of_step": tms / ms}
     result = {
         "metric": METRIC, "value": rows_timed / (ms * 1e-3), "unit": "rows/s", "n_gpus": world, "steps": K,
@@ -235,7 +255,7 @@ def run_ours(args, cfg, rank, world, local_rank):
                       "frac_of_8TBs": step_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
                       "frac_of_measured_copy": step_bytes / (ms_step * 1e-3) / 1e9 / peak},
         "per_step": {"indices": L, "distinct_rows": U, "distinct_hits": U_hit, "index_hit_rate": occ_hit / max(L, 1),
-                     "admissions": adm, "evictions": evi},
+                     "admissions": adm, "evictions": evi, "hot_rows": hot_rows, "hot_row_indices": hot_occ},
         "kernels_ms_per_step": {k: v[0] / K for k, v in sorted(prof.items(), key=lambda kv: -kv[1][0])},
     }
     return result
@@ -322,7 +342,7 @@ def main():
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             cfg0 = make_cfg()
-            r = run_oracle(cfg0, 1, 0, torch.device("cuda", local_rank))
+            r = run_oracle(cfg0, 1, 0, torch.device("cuda", local_rank), budget_rows=12_000_000)
             result["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
         print(json.dumps(result))
     if world > 1:

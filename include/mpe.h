@@ -127,9 +127,11 @@ int mpe_stats(mpe_handle* h, int32_t table, uint64_t* out8);
 int mpe_memory_bytes(mpe_handle* h, uint64_t* out6);
 /* Geometry of table `table`'s cache. */
 int mpe_cache_geometry(mpe_handle* h, int32_t table, int32_t* n_sets, int32_t* ways);
-/* Figures of the last mpe_forward: out4 = {valid indices, distinct rows, dropped indices, rows whose
- * multiplicity needs the multi-block gradient tree}. */
-int mpe_step_info(mpe_handle* h, int64_t* out4);
+/* Figures of the last step: out6 = {valid indices, distinct rows, dropped indices, rows whose gradient
+ * is summed by the multi-block tree (more than 256 occurrences), indices that belong to such rows,
+ * newcomers that had to wait for the write-back of a row updated in the same step (known after
+ * mpe_backward)}. */
+int mpe_step_info(mpe_handle* h, int64_t* out6);
 /* Low-precision entries of n rows: h_codes[n][dim*bits/8] (INT4: column 2k in the low nibble of
  * byte k), h_scale[n], h_bias[n].  The entry of a cache-resident row is stale until it is evicted
  * or flushed. */

@@ -148,7 +148,7 @@ class Mpe:
         return n.value, w.value
 
     def step_info(self):
-        out = np.zeros(4, np.int64)
+        out = np.zeros(6, np.int64)
         _check(_lib.mpe_step_info(self._h, out.ctypes.data), "mpe_step_info")
         return out
 

@@ -521,9 +521,10 @@ int mpe_cache_geometry(mpe_handle* h, int32_t table, int32_t* n_sets, int32_t* w
     return MPE_OK;
 }
 
-int mpe_step_info(mpe_handle* h, int64_t* out4) {
-    if (!h || !out4) return MPE_ERR_ARG;
-    out4[0] = out4[1] = out4[2] = out4[3] = 0;
+int mpe_step_info(mpe_handle* h, int64_t* out6) {
+    if (!h || !out6) return MPE_ERR_ARG;
+    int64_t* out4 = out6;
+    for (int i = 0; i < 6; ++i) out6[i] = 0;
     if (!h->wk.ctr) return MPE_OK;
     DeviceGuard guard(h->device);
     CK(h, cudaStreamSynchronize(h->stream));
@@ -545,6 +546,8 @@ int mpe_step_info(mpe_handle* h, int64_t* out4) {
     out4[1] = (int64_t)c.U - pseudo;
     out4[2] = (int64_t)c.dropped;
     out4[3] = (int64_t)c.hot_rows;
+    out6[4] = (int64_t)c.hot_occ;
+    out6[5] = (int64_t)c.deferred;
     return MPE_OK;
 }
 

@@ -32,6 +32,7 @@ struct Counters {
     uint32_t n_heads;      // cache sets that have miss candidates in this step
     uint32_t upd_next;     // next block of 32 distinct rows to hand to a warp of k_update
     unsigned long long dropped;      // out-of-range indices in this batch
+    unsigned long long hot_occ;      // indices that belong to hot rows
     unsigned long long err[2];       // sticky: ERR_INDEX, ERR_OFFSETS
 };
 
@@ -73,7 +74,7 @@ struct Work {
 __global__ void k_prelude(Work w, const int32_t* __restrict__ offsets, int T, int B, uint32_t L) {
     if (threadIdx.x == 0 && blockIdx.x == 0) {
         Counters* c = w.ctr;
-        c->L = L; c->U = 0; c->hot_rows = 0; c->hot_tasks = 0; c->abort = 0; c->dropped = 0; c->deferred = 0; c->n_heads = 0; c->upd_next = 0;
+        c->L = L; c->U = 0; c->hot_rows = 0; c->hot_tasks = 0; c->abort = 0; c->dropped = 0; c->hot_occ = 0; c->deferred = 0; c->n_heads = 0; c->upd_next = 0;
         bool bad = offsets[0] != 0 || offsets[(int64_t)T * B] != (int32_t)L;
         int32_t prev = 0;
         w.table_start[0] = 0;
@@ -230,6 +231,7 @@ k_probe(State s, Work w, uint32_t epoch) {
                 const uint32_t nt = (mult + HOT_SPAN - 1) / HOT_SPAN;
                 hb = (int)atomicAdd(&w.ctr->hot_tasks, nt);
                 w.hot_k[atomicAdd(&w.ctr->hot_rows, 1u)] = (int32_t)k;
+                atomicAdd(&w.ctr->hot_occ, (unsigned long long)mult);
                 for (uint32_t j = 0; j < nt; ++j) w.task_k[hb + j] = (int32_t)k;
             }
             w.hot_base[k] = hb;
