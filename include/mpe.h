@@ -39,7 +39,8 @@ enum {
     MPE_ERR_SEQUENCE = -4,     /* backward without a preceding forward, or step not strictly increasing */
     MPE_ERR_INDEX = -5,        /* device saw row ids outside [0, num_rows) (detail = how many); they were dropped */
     MPE_ERR_OFFSETS = -6,      /* device saw offsets that are not 0 = o[0] <= o[1] <= ... <= o[T*B] = total */
-    MPE_ERR_NOMEM = -7         /* allocation failed */
+    MPE_ERR_NOMEM = -7,        /* allocation failed */
+    MPE_ERR_TOO_LARGE = -8     /* mpe_forward_static: the batch does not fit the fixed scratch */
 };
 
 /*
@@ -105,6 +106,39 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
  * Uses the stream of the last mpe_forward (default stream if none). */
 int mpe_step_host(mpe_handle* h, const int32_t* h_indices, const int32_t* h_offsets, int32_t batch,
                   int64_t total_indices, const float* h_grad_out, float* h_out, float lr, int64_t step);
+
+/*
+ * Evaluation forward that allocates nothing.  (The paper has no counterpart: this is an addition for
+ * callers that are not allowed to allocate device memory when they call into the library -- code that
+ * runs under a memory budget fixed at start-up, inside another framework's allocator that must see every
+ * byte, or in a region where a synchronising cudaMalloc/cudaFree would stall concurrent streams.
+ * mpe_forward sizes its workspace with cudaMalloc whenever a larger batch arrives; this entry point never
+ * does.)
+ *
+ * Same inputs, outputs, layouts and result as mpe_forward -- the pooled FP32 sums of the bags, bit for bit
+ * -- but every intermediate array of the step (sort keys and payloads, histograms, prefix sums, the
+ * distinct-row list and its maps) lives in ONE fixed array compiled into the library
+ * (`static __device__`, about 2.2 MB; every GPU that loads the library holds it until the process exits).
+ * Limits: total_indices <= MPE_STATIC_MAX_INDICES, num_tables * batch <= MPE_STATIC_MAX_BAGS,
+ * num_tables <= MPE_STATIC_MAX_TABLES; a larger call returns MPE_ERR_TOO_LARGE and does nothing.
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ * It is an evaluation forward: it never changes table, cache or policy state and cannot be followed by
+ * mpe_backward; calling it between the mpe_forward and mpe_backward of a training step returns
+ * MPE_ERR_SEQUENCE.  Out-of-range row ids contribute nothing and inconsistent offsets give all-zero
+ * output, as in mpe_forward, but this entry point does not record them for mpe_last_error.
+ *
+ * All calls, from every handle on that GPU, share the one array, and it keeps the previous call's
+ * contents (the call clears the counters it needs at zero): two calls whose GPU work overlaps -- different
+ * streams, or different handles -- race on it.  Issue them on one stream, or wait between them.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress); make that
+ * first call outside any stream capture.
+ */
+#define MPE_STATIC_MAX_INDICES 32768
+#define MPE_STATIC_MAX_BAGS 32768
+#define MPE_STATIC_MAX_TABLES 64
+int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch,
+                       int64_t total_indices, float* d_out, void* cuda_stream);
 
 /* Write every cache-resident row back into the low-precision table with stochastic rounding; rows
  * stay resident and unchanged.  Afterwards the table alone is a complete snapshot of the model.

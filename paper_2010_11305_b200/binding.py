@@ -16,10 +16,11 @@ LIB_PATH = os.path.join(_HERE, "libmpe.so")
 
 LRU, LFU = 0, 1
 SGD, ROWWISE_ADAGRAD = 0, 1
-OK, ERR_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_SEQUENCE, ERR_INDEX, ERR_OFFSETS, ERR_NOMEM = 0, -1, -2, -3, -4, -5, -6, -7
+OK, ERR_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_SEQUENCE, ERR_INDEX, ERR_OFFSETS, ERR_NOMEM, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6, -7, -8
+STATIC_MAX_INDICES, STATIC_MAX_BAGS, STATIC_MAX_TABLES = 32768, 32768, 64
 
 EXPORTS = [
-    "mpe_create", "mpe_reserve", "mpe_forward", "mpe_backward", "mpe_step_host", "mpe_flush", "mpe_destroy",
+    "mpe_create", "mpe_reserve", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_step_host", "mpe_flush", "mpe_destroy",
     "mpe_last_error", "mpe_stats", "mpe_memory_bytes", "mpe_cache_geometry", "mpe_step_info", "mpe_export_rows",
     "mpe_export_cache", "mpe_export_aux", "mpe_kernel_launches", "mpe_profile", "mpe_profile_read", "mpe_error_string",
 ]
@@ -41,6 +42,7 @@ _vp, _i32, _i64, _u64, _f32, _f64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
 _lib.mpe_create.argtypes = [C.POINTER(_vp), C.POINTER(TableSpec), _i32, _i32, _f64, _i32, _i32, _i32, _f32, _f32, _f32, _u64, _i32]
 _lib.mpe_reserve.argtypes = [_vp, _i32, _i64]
 _lib.mpe_forward.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp]
+_lib.mpe_forward_static.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp]
 _lib.mpe_backward.argtypes = [_vp, _vp, _f32, _i64]
 _lib.mpe_step_host.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp, _f32, _i64]
 _lib.mpe_flush.argtypes = [_vp]
@@ -114,6 +116,11 @@ class Mpe:
     def forward(self, d_indices, d_offsets, batch, d_out, stream=None):
         _check(_lib.mpe_forward(self._h, _ptr(d_indices), _ptr(d_offsets), batch, d_indices.numel(), _ptr(d_out),
                                 stream), "mpe_forward")
+
+    def forward_static(self, d_indices, d_offsets, batch, d_out, stream=None):
+        """Evaluation forward for callers that must not allocate: its scratch is a fixed array inside the library."""
+        _check(_lib.mpe_forward_static(self._h, _ptr(d_indices), _ptr(d_offsets), batch, d_indices.numel(), _ptr(d_out),
+                                       stream), "mpe_forward_static")
 
     def backward(self, d_grad_out, lr, step):
         _check(_lib.mpe_backward(self._h, _ptr(d_grad_out), lr, step), "mpe_backward")

@@ -210,6 +210,7 @@ const char* mpe_error_string(int code) {
         case MPE_ERR_INDEX: return "row index out of range";
         case MPE_ERR_OFFSETS: return "inconsistent offsets";
         case MPE_ERR_NOMEM: return "out of memory";
+        case MPE_ERR_TOO_LARGE: return "batch larger than the fixed scratch of mpe_forward_static";
         default: return "unknown error";
     }
 }
@@ -652,3 +653,115 @@ int mpe_profile_read(mpe_handle* h, int32_t cap, char* names, double* ms, uint64
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Evaluation forward whose whole per-step workspace is a fixed array inside the library image
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int64_t STATIC_MAX_INDICES = MPE_STATIC_MAX_INDICES;
+constexpr int64_t STATIC_MAX_BAGS = MPE_STATIC_MAX_BAGS;
+constexpr int STATIC_MAX_TABLES = MPE_STATIC_MAX_TABLES;
+constexpr size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
+constexpr size_t STATIC_PER_INDEX_ARRAYS = 16;     // u32/i32 arrays of STATIC_MAX_INDICES + 2 entries
+constexpr size_t STATIC_SCRATCH_BYTES =
+    STATIC_PER_INDEX_ARRAYS * align256((STATIC_MAX_INDICES + 2) * 4) +                                 // keys, payloads, per-index and per-row maps
+    align256(256 * ((STATIC_MAX_INDICES + SORT_TILE - 1) / SORT_TILE + STATIC_MAX_TABLES + 1) * 4) +   // sort histograms
+    align256((256 * ((STATIC_MAX_INDICES + SORT_TILE - 1) / SORT_TILE + STATIC_MAX_TABLES + 1) / SCAN_TILE + 2 +
+              STATIC_MAX_INDICES / SCAN_TILE + 2) * 4) +                                               // block sums
+    4 * align256((STATIC_MAX_TABLES + 1) * 4) +                                                        // per-table starts
+    2 * align256((STATIC_MAX_INDICES / HOT_MIN + 2) * 4) +                                             // hot-row lists
+    align256(sizeof(Counters));
+
+// The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress; it is not a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+unsigned char* g_scratch_addr[MAX_DEVICES] = {};     // device address of g_static_scratch, per device, filled on first use
+
+struct Carver {
+    unsigned char* p; size_t used = 0;
+    template <class T> T* take(size_t count) { T* r = reinterpret_cast<T*>(p + used); used += align256(count * sizeof(T)); return r; }
+};
+
+}  // namespace
+
+extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch,
+                                  int64_t total_indices, float* d_out, void* cuda_stream) {
+    if (!h || !d_offsets || batch < 0 || total_indices < 0) return MPE_ERR_ARG;
+    if ((total_indices > 0 && !d_indices) || (batch > 0 && !d_out)) return MPE_ERR_ARG;
+    const int64_t bags = (int64_t)h->T * batch;
+    if (total_indices > STATIC_MAX_INDICES || bags > STATIC_MAX_BAGS || h->T > STATIC_MAX_TABLES) return MPE_ERR_TOO_LARGE;
+    if (h->have_forward) return MPE_ERR_SEQUENCE;      // a training step is half done: its backward still needs the probe marks
+    if (h->device < 0 || h->device >= MAX_DEVICES) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    if (!g_scratch_addr[h->device]) {
+        // once per device, with that device current: ask the runtime where the array lives on this device
+        void* addr = nullptr;
+        CK(h, cudaGetSymbolAddress(&addr, g_static_scratch));
+        g_scratch_addr[h->device] = static_cast<unsigned char*>(addr);
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (stream != h->stream) { CK(h, cudaStreamSynchronize(h->stream)); h->stream = stream; }
+
+    // carve the step's arrays out of the scratch (same roles as the handle's own workspace)
+    Carver c{g_scratch_addr[h->device]};
+    const size_t n = (size_t)STATIC_MAX_INDICES + 2;
+    uint32_t *keyA = c.take<uint32_t>(n), *keyB = c.take<uint32_t>(n), *valA = c.take<uint32_t>(n), *valB = c.take<uint32_t>(n);
+    Work w{};
+    w.bag_of = c.take<int32_t>(n); w.kidx = c.take<uint32_t>(n); w.occ_loc = c.take<int32_t>(n); w.occ_b = c.take<int32_t>(n);
+    w.uniq_row = c.take<int32_t>(n); w.uniq_t = c.take<int32_t>(n); w.seg = c.take<int32_t>(n); w.loc = c.take<int32_t>(n);
+    w.final_loc = c.take<int32_t>(n); w.uset = c.take<int32_t>(n); w.hot_base = c.take<int32_t>(n); w.victim = c.take<int32_t>(n);
+    const size_t max_tiles = (STATIC_MAX_INDICES + SORT_TILE - 1) / SORT_TILE + STATIC_MAX_TABLES + 1;
+    uint32_t* hist = c.take<uint32_t>(256 * max_tiles);
+    uint32_t* block_sums = c.take<uint32_t>(256 * max_tiles / SCAN_TILE + 2 + STATIC_MAX_INDICES / SCAN_TILE + 2);
+    w.table_start = c.take<int32_t>(STATIC_MAX_TABLES + 1); w.tile_base = c.take<int32_t>(STATIC_MAX_TABLES + 1);
+    w.ustart = c.take<int32_t>(STATIC_MAX_TABLES + 1); w.ctile_base = c.take<int32_t>(STATIC_MAX_TABLES + 1);
+    w.hot_k = c.take<int32_t>(STATIC_MAX_INDICES / HOT_MIN + 2); w.task_k = c.take<int32_t>(STATIC_MAX_INDICES / HOT_MIN + 2);
+    w.ctr = c.take<Counters>(1);
+    if (c.used > STATIC_SCRATCH_BYTES) return MPE_ERR_ARG;      // cannot happen: the size formula above mirrors this list
+
+    const State& s = h->st;
+    const int T = h->T;
+    const uint32_t L = (uint32_t)total_indices;
+    ++h->epoch;
+    // the array keeps whatever the previous call left: the counters are the only part that must start from zero
+    CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), stream));
+    LAUNCH(h, "prelude", k_prelude, 1, 32, 0, w, d_offsets, T, batch, L);
+    LAUNCH(h, "make_keys", k_make_keys, grid_for(h, bags, 8, 8), 256, 0, s, w, d_indices, d_offsets, batch, keyA);
+    // segmented radix sort, as in mpe_forward, on the carved buffers
+    LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, (const int32_t*)w.table_start, T, w.tile_base, &w.ctr->hist_len,
+           (const uint32_t*)&w.ctr->abort);
+    const int64_t tiles_upper = (total_indices + SORT_TILE - 1) / SORT_TILE + T;
+    const int gsort = grid_for(h, tiles_upper, 1, 3);
+    const int gscan = grid_for(h, 256 * tiles_upper, SCAN_TILE, 8);
+    const int passes = (bits_for((uint32_t)h->max_rows) + 7) / 8;
+    uint32_t *kin = keyA, *kout = keyB, *vin = nullptr, *vout = valB;
+    for (int p = 0; p < passes; ++p) {
+        LAUNCH(h, "sort_hist", k_sort_hist, gsort, SORT_THREADS, 0, (const uint32_t*)kin, (const int32_t*)w.table_start,
+               (const int32_t*)w.tile_base, T, 8 * p, hist);
+        LAUNCH(h, "scan_reduce", k_scan_reduce, gscan, SCAN_THREADS, 0, (const uint32_t*)hist, (const uint32_t*)&w.ctr->hist_len, block_sums);
+        LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, block_sums, (const uint32_t*)&w.ctr->hist_len,
+               (uint32_t)SCAN_TILE, (uint32_t*)nullptr);
+        LAUNCH(h, "scan_apply", k_scan_apply, gscan, SCAN_THREADS, 0, hist, (const uint32_t*)&w.ctr->hist_len, (const uint32_t*)block_sums);
+        LAUNCH(h, "sort_scatter", k_sort_scatter, gsort, SORT_THREADS, 0, (const uint32_t*)kin, (const uint32_t*)vin, kout, vout,
+               (const int32_t*)w.table_start, (const int32_t*)w.tile_base, T, 8 * p, (const uint32_t*)hist);
+        std::swap(kin, kout);
+        vin = vout; vout = (vout == valB) ? valA : valB;
+    }
+    const uint32_t* skey = kin;
+    const uint32_t* spos = vin;
+    const int gs = grid_for(h, total_indices, SCAN_TILE, 8);
+    LAUNCH(h, "unique_count", k_unique<false>, gs, SCAN_THREADS, 0, w, T, skey, block_sums);
+    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);
+    LAUNCH(h, "unique_write", k_unique<true>, gs, SCAN_THREADS, 0, w, T, skey, block_sums);
+    LAUNCH(h, "ustart", k_ustart, 1, 256, 0, w, T);
+    LAUNCH(h, "probe", k_probe, grid_for(h, total_indices, 256, 8), 256, 0, s, w, h->epoch);
+    LAUNCH(h, "broadcast", k_broadcast, grid_for(h, total_indices, 256, 8), 256, 0, s, w, spos, batch);
+    const int gp = grid_for(h, bags, 256 / s.lanes, 8);
+    dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
+        auto kern = k_pool<decltype(bc)::value, decltype(lc)::value>;
+        LAUNCH(h, "pool", kern, gp, 256, 0, s, w, d_indices, d_offsets, batch, d_out);
+    });
+    return check_launch(h);
+}
