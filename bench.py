@@ -134,12 +134,29 @@ def byte_model(cfg, L, U, U_hit, occ_hit, admissions, evictions, hot_occ, passes
     return step, m
 
 
+def shard_config(cfg, rank):
+    """Table-wise sharding without a data-path collective: every rank trains its own set of tables of the
+    configuration's shapes (its own seed, hence its own rows and index streams): weak scaling."""
+    cfg.seed = cfg.seed + 7919 * rank
+    return cfg
+
+
+def aggregate(times, rows, world, device):
+    """Whole-job figures from per-rank ones: the slowest rank's times (MAX) and everybody's rows (SUM)."""
+    if world <= 1:
+        return [float(x) for x in times], [float(x) for x in rows]
+    t = torch.tensor(times, dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    r = torch.tensor(rows, dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(r, op=torch.distributed.ReduceOp.SUM)
+    return [float(x) for x in t], [float(x) for x in r]
+
+
 def run_ours(args, cfg, rank, world, local_rank):
     from paper_2010_11305_b200 import binding as mpe
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
-    # every rank owns its own shard of tables (same shapes, different seed): weak scaling
-    cfg.seed = cfg.seed + 7919 * rank
+    cfg = shard_config(cfg, rank)
     stream_gen = wl.Stream(cfg, dev)
     h = mpe.Mpe(cfg.num_rows, cfg.dim, cfg.bits, cfg.cache_fraction, cfg.ways, cfg.policy, cfg.optimizer, cfg.eps,
                 cfg.init_lo, cfg.init_hi, cfg.seed, local_rank)
@@ -209,14 +226,7 @@ def run_ours(args, cfg, rank, world, local_rank):
     d2h = float(h_out.numel() * 4)
 
     # aggregate over ranks: total rows / max time
-    rows_timed = float(ds[0])
-    if world > 1:
-        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        r = torch.tensor([rows_timed, float(e2e_rows)], dtype=torch.float64, device=dev)
-        torch.distributed.all_reduce(r, op=torch.distributed.ReduceOp.SUM)
-        ms, e2e_s = float(t[0]), float(t[1])
-        rows_timed, e2e_rows = float(r[0]), float(r[1])
+    (ms, e2e_s), (rows_timed, e2e_rows) = aggregate([ms, e2e_s], [float(ds[0]), float(e2e_rows)], world, dev)
     if rank != 0:
         return None
 
