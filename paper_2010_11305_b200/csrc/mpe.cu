@@ -377,7 +377,7 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
     dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
         constexpr int LANES = decltype(lc)::value;
         auto hot = k_hot_partial<LANES>;
-        LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, L / HOT_MIN + 1, 1, 2), 8 * LANES, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
+        LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, L / HOT_MIN + 1, 1, 1), 8 * LANES, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
     });
     CK(h, cudaEventRecord(h->ev_join, h->side));
     LAUNCH(h, "priority", k_priority, grid_for(h, L, 256, 8), 256, 0, s, w, (uint32_t)step, h->ckeyA);

@@ -279,6 +279,8 @@ k_pool(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __re
     const bool abort = w.ctr->abort != 0;
     const char* slab_col = reinterpret_cast<const char*>(s.slab) + 16 * sub;
     int64_t bag = blockIdx.x * gpb + threadIdx.x / LANES;
+    int t = (int)(bag / B);
+    int64_t b = bag - (int64_t)t * B;
     // (slot, row id) of the first LANES indices of a bag, one per lane; fetched one bag ahead
     int32_t lo = 0, hi = 0; int wloc = LOC_INVALID; int32_t wrow = 0;
     auto open_bag = [&](int64_t bg) {
@@ -290,8 +292,6 @@ k_pool(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __re
     };
     open_bag(bag);
     for (; bag < nbags; bag += ng) {
-        const int t = (int)(bag / B);
-        const int b = (int)(bag - (int64_t)t * B);
         const int64_t row_base = s.tables[t].row_base;
         const int32_t clo = lo, chi = hi;
         int myloc = wloc; int32_t myrow = wrow;
@@ -309,33 +309,56 @@ k_pool(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __re
             }
             return x;
         };
+        auto fetch_hit = [&](int src_lane) {          // the row is known to be cache resident
+            const uint32_t lc = (uint32_t)__shfl_sync(gmask, myloc, gbase + src_lane);
+            return __ldg(reinterpret_cast<const float4*>(slab_col + (size_t)lc * (size_t)(dim * 4)));
+        };
         for (int32_t p0 = clo; p0 < chi; p0 += LANES) {
             if (p0 > clo) {                           // later windows of a long bag
                 myloc = LOC_INVALID;
                 if (p0 + sub < chi) { myloc = w.occ_loc[p0 + sub]; myrow = indices[p0 + sub]; }
             }
             const int n = min(LANES, chi - p0);
+            const uint32_t hits = (__ballot_sync(gmask, myloc >= 0) & gmask) >> gbase;    // bit u: row u of the window is cached
+            constexpr uint32_t FULL = (1u << NB) - 1u;
             float4 xa[NB], xb[NB];
+            if ((hits & FULL) == FULL) {
 #pragma unroll
-            for (int u = 0; u < NB; ++u) xa[u] = fetch(u);
+                for (int u = 0; u < NB; ++u) xa[u] = fetch_hit(u);
+            } else {
+#pragma unroll
+                for (int u = 0; u < NB; ++u) xa[u] = fetch(u);
+            }
             for (int u0 = 0; u0 < n; u0 += 2 * NB) {  // rows are added in index order
                 if (u0 + NB < n) {
+                    if (((hits >> (u0 + NB)) & FULL) == FULL) {
 #pragma unroll
-                    for (int u = 0; u < NB; ++u) xb[u] = fetch((u0 + NB + u) & (LANES - 1));
+                        for (int u = 0; u < NB; ++u) xb[u] = fetch_hit(u0 + NB + u);
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < NB; ++u) xb[u] = fetch((u0 + NB + u) & (LANES - 1));
+                    }
                 }
 #pragma unroll
                 for (int u = 0; u < NB; ++u) acc = add4(acc, xa[u]);
                 if (u0 + NB < n) {
                     if (u0 + 2 * NB < n) {
+                        if (((hits >> (u0 + 2 * NB)) & FULL) == FULL) {
 #pragma unroll
-                        for (int u = 0; u < NB; ++u) xa[u] = fetch((u0 + 2 * NB + u) & (LANES - 1));
+                            for (int u = 0; u < NB; ++u) xa[u] = fetch_hit(u0 + 2 * NB + u);
+                        } else {
+#pragma unroll
+                            for (int u = 0; u < NB; ++u) xa[u] = fetch((u0 + 2 * NB + u) & (LANES - 1));
+                        }
                     }
 #pragma unroll
                     for (int u = 0; u < NB; ++u) acc = add4(acc, xb[u]);
                 }
             }
         }
-        reinterpret_cast<float4*>(out + ((int64_t)b * s.T + t) * dim)[sub] = acc;
+        reinterpret_cast<float4*>(out + (b * s.T + t) * dim)[sub] = acc;
+        b += ng;
+        while (b >= B) { b -= B; ++t; }
     }
 }
 
@@ -507,23 +530,27 @@ __device__ __forceinline__ float4 sum_chunk(const int32_t* __restrict__ occ_b, c
                                             int32_t first, int len, uint32_t gmask, int gbase, int sub) {
     constexpr int NB = LANES < 8 ? LANES : 8;
     float4 acc;
-    if (LANES == 32 && len == 32) {       // a full chunk handled by a whole warp: no bounds to check
+    if (LANES == 32 && len == 32) {       // a full chunk handled by a whole warp: no bounds to check, 16 rows in flight
         const uint32_t myb = (uint32_t)occ_b[first + sub];
-        float4 v[8];
+        float4 va[8], vb[8];
+        auto row = [&](int u) { return __ldg(reinterpret_cast<const float4*>(gcol + (size_t)__shfl_sync(0xffffffffU, myb, u) * stride_bytes)); };
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-            v[u] = __ldg(reinterpret_cast<const float4*>(gcol + (size_t)__shfl_sync(0xffffffffU, myb, u) * stride_bytes));
-        acc = v[0];
+        for (int u = 0; u < 8; ++u) va[u] = row(u);
 #pragma unroll
-        for (int u = 1; u < 8; ++u) acc = add4(acc, v[u]);
+        for (int u = 0; u < 8; ++u) vb[u] = row(8 + u);
+        acc = va[0];
 #pragma unroll
-        for (int u0 = 8; u0 < 32; u0 += 8) {
+        for (int u = 1; u < 8; ++u) acc = add4(acc, va[u]);
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
-                v[u] = __ldg(reinterpret_cast<const float4*>(gcol + (size_t)__shfl_sync(0xffffffffU, myb, u0 + u) * stride_bytes));
+        for (int u = 0; u < 8; ++u) va[u] = row(16 + u);
 #pragma unroll
-            for (int u = 0; u < 8; ++u) acc = add4(acc, v[u]);
-        }
+        for (int u = 0; u < 8; ++u) acc = add4(acc, vb[u]);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) vb[u] = row(24 + u);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc = add4(acc, va[u]);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc = add4(acc, vb[u]);
         return acc;
     }
     acc = make_float4(0.f, 0.f, 0.f, 0.f);
