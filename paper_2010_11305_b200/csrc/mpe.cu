@@ -332,7 +332,7 @@ int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offset
     h->B = batch; h->L = total_indices; ++h->epoch;
 
     LAUNCH(h, "prelude", k_prelude, 1, 32, 0, w, d_offsets, T, batch, L);
-    LAUNCH(h, "make_keys", k_make_keys, grid_for(h, bags, 8, 8), 256, 0, s, w, d_indices, d_offsets, batch, h->keyA);
+    LAUNCH(h, "make_keys", k_make_keys, grid_for(h, bags, 32, 8), 256, 0, s, w, d_indices, d_offsets, batch, h->keyA);
     // sort the row indices of the mini-batch (Section 5.1), table by table
     const int which = seg_sort(h, h->keyA, h->keyB, h->valA, h->valB, w.table_start, w.tile_base, &w.ctr->hist_len,
                                bits_for((uint32_t)h->max_rows), total_indices);
@@ -380,7 +380,7 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
         LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, L / HOT_MIN + 1, 1, 1), 8 * LANES, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
     });
     CK(h, cudaEventRecord(h->ev_join, h->side));
-    LAUNCH(h, "priority", k_priority, grid_for(h, L, 256, 8), 256, 0, s, w, (uint32_t)step, h->ckeyA);
+    LAUNCH(h, "priority", k_priority, grid_for(h, L, 1024, 8), 256, 0, s, w, (uint32_t)step, h->ckeyA);
     if (h->max_sets > 0) {
         // group the rows that missed by cache set, keeping ascending row id inside a set
         const int which = seg_sort(h, h->ckeyA, h->ckeyB, h->cvalA, h->cvalB, w.ustart, w.ctile_base, &w.ctr->chist_len,
@@ -728,7 +728,7 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     // the array keeps whatever the previous call left: the counters are the only part that must start from zero
     CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), stream));
     LAUNCH(h, "prelude", k_prelude, 1, 32, 0, w, d_offsets, T, batch, L);
-    LAUNCH(h, "make_keys", k_make_keys, grid_for(h, bags, 8, 8), 256, 0, s, w, d_indices, d_offsets, batch, keyA);
+    LAUNCH(h, "make_keys", k_make_keys, grid_for(h, bags, 32, 8), 256, 0, s, w, d_indices, d_offsets, batch, keyA);
     // segmented radix sort, as in mpe_forward, on the carved buffers
     LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, (const int32_t*)w.table_start, T, w.tile_base, &w.ctr->hist_len,
            (const uint32_t*)&w.ctr->abort);

@@ -88,32 +88,36 @@ __global__ void k_prelude(Work w, const int32_t* __restrict__ offsets, int T, in
     }
 }
 
-// keys for the sort: the row id, or N_t for an id outside [0, N_t); one warp per bag
-__global__ void k_make_keys(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets,
-                            int B, uint32_t* __restrict__ keys) {
-    const int lane = threadIdx.x & 31;
+// keys for the sort: the row id, or N_t for an id outside [0, N_t); eight lanes per bag, four bags per warp
+__global__ void __launch_bounds__(256)
+k_make_keys(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets,
+            int B, uint32_t* __restrict__ keys) {
+    const int sub = threadIdx.x & 7;
     const int64_t nbags = (int64_t)s.T * B;
-    const int64_t nw = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t ng = (int64_t)gridDim.x * (blockDim.x >> 3);
     const int32_t L = (int32_t)w.ctr->L;
-    for (int64_t bag = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); bag < nbags; bag += nw) {
+    int64_t bag = (int64_t)blockIdx.x * (blockDim.x >> 3) + (threadIdx.x >> 3);
+    int t = (int)(bag / B);
+    int64_t b = bag - (int64_t)t * B;
+    unsigned long long bad = 0;
+    for (; bag < nbags; bag += ng) {
         const int32_t lo = offsets[bag], hi = offsets[bag + 1];
         if (lo < 0 || hi < lo || hi > L) {
-            if (lane == 0) { w.ctr->abort = 1; atomicAdd(&w.ctr->err[ERR_OFFSETS], 1ULL); }
-            continue;
+            if (sub == 0) { w.ctr->abort = 1; atomicAdd(&w.ctr->err[ERR_OFFSETS], 1ULL); }
+        } else {
+            const int32_t N = s.tables[t].N;
+            for (int32_t p = lo + sub; p < hi; p += 8) {
+                const int32_t r = indices[p];
+                const bool ok = r >= 0 && r < N;
+                keys[p] = ok ? (uint32_t)r : (uint32_t)N;
+                w.bag_of[p] = (int32_t)bag;
+                bad += !ok;
+            }
         }
-        const int t = (int)(bag / B);
-        const int32_t N = s.tables[t].N;
-        int bad = 0;
-        for (int32_t p = lo + lane; p < hi; p += 32) {
-            const int32_t r = indices[p];
-            const bool ok = r >= 0 && r < N;
-            keys[p] = ok ? (uint32_t)r : (uint32_t)N;
-            w.bag_of[p] = (int32_t)bag;
-            bad += !ok;
-        }
-        bad = __reduce_add_sync(0xffffffffU, bad);
-        if (lane == 0 && bad) { atomicAdd(&w.ctr->dropped, (unsigned long long)bad); atomicAdd(&w.ctr->err[ERR_INDEX], (unsigned long long)bad); }
+        b += ng;
+        while (b >= B) { b -= B; ++t; }
     }
+    if (bad) { atomicAdd(&w.ctr->dropped, bad); atomicAdd(&w.ctr->err[ERR_INDEX], bad); }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -131,10 +135,21 @@ k_unique(Work w, int T, const uint32_t* __restrict__ skey, uint32_t* __restrict_
         uint32_t flag[SCAN_ITEMS];
         int tcur[SCAN_ITEMS];
         uint32_t sum = 0;
+        uint32_t keyv[SCAN_ITEMS];
         if (base < n) {
             int t = find_segment(w.table_start, T, (int32_t)base);
             while (w.table_start[t + 1] <= (int32_t)base) ++t;     // skip empty tables that start here
             uint32_t prev = base > 0 ? skey[base - 1] : 0;
+            if (base + SCAN_ITEMS <= n) {                           // 16 keys as four 16-byte loads
+#pragma unroll
+                for (int i = 0; i < SCAN_ITEMS; i += 4) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(skey + base + i);
+                    keyv[i] = v.x; keyv[i + 1] = v.y; keyv[i + 2] = v.z; keyv[i + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < SCAN_ITEMS; ++i) keyv[i] = base + i < n ? skey[base + i] : 0;
+            }
 #pragma unroll
             for (int i = 0; i < SCAN_ITEMS; ++i) {
                 const uint32_t e = base + i;
@@ -142,7 +157,7 @@ k_unique(Work w, int T, const uint32_t* __restrict__ skey, uint32_t* __restrict_
                 if (e < n) {
                     while (w.table_start[t + 1] <= (int32_t)e) ++t;
                     tcur[i] = t;
-                    const uint32_t k = skey[e];
+                    const uint32_t k = keyv[i];
                     flag[i] = (e == (uint32_t)w.table_start[t] || k != prev) ? 1u : 0u;
                     prev = k;
                     sum += flag[i];
@@ -150,7 +165,7 @@ k_unique(Work w, int T, const uint32_t* __restrict__ skey, uint32_t* __restrict_
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < SCAN_ITEMS; ++i) { flag[i] = 0; tcur[i] = 0; }
+            for (int i = 0; i < SCAN_ITEMS; ++i) { flag[i] = 0; tcur[i] = 0; keyv[i] = 0; }
         }
         uint32_t total;
         uint32_t ex = block_exclusive_scan<SCAN_THREADS>(sum, &total, tmp);
@@ -158,15 +173,21 @@ k_unique(Work w, int T, const uint32_t* __restrict__ skey, uint32_t* __restrict_
             if (threadIdx.x == 0) block_sums[b] = total;
         } else {
             ex += block_sums[b];
+            uint32_t kout[SCAN_ITEMS];
 #pragma unroll
             for (int i = 0; i < SCAN_ITEMS; ++i) {
                 const uint32_t e = base + i;
-                if (e < n) {
-                    ex += flag[i];
-                    const uint32_t k = ex - 1;
-                    w.kidx[e] = k;
-                    if (flag[i]) { w.uniq_row[k] = (int32_t)skey[e]; w.uniq_t[k] = tcur[i]; w.seg[k] = (int32_t)e; }
-                }
+                ex += flag[i];
+                kout[i] = ex - 1;
+                if (e < n && flag[i]) { w.uniq_row[kout[i]] = (int32_t)keyv[i]; w.uniq_t[kout[i]] = tcur[i]; w.seg[kout[i]] = (int32_t)e; }
+            }
+            if (base + SCAN_ITEMS <= n) {
+#pragma unroll
+                for (int i = 0; i < SCAN_ITEMS; i += 4)
+                    *reinterpret_cast<uint4*>(w.kidx + base + i) = make_uint4(kout[i], kout[i + 1], kout[i + 2], kout[i + 3]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < SCAN_ITEMS; ++i) if (base + i < n) w.kidx[base + i] = kout[i];
             }
         }
     }
@@ -240,7 +261,8 @@ k_probe(State s, Work w, uint32_t epoch) {
 }
 
 // per sorted element: where its row lives (by index position) and which sample it belongs to
-__global__ void k_broadcast(State s, Work w, const uint32_t* __restrict__ spos, int B) {
+__global__ void __launch_bounds__(256)
+k_broadcast(State s, Work w, const uint32_t* __restrict__ spos, int B) {
     if (w.ctr->abort) return;
     const int64_t L = w.ctr->L;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < L; i += (int64_t)gridDim.x * blockDim.x) {
@@ -365,48 +387,65 @@ k_pool(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __re
 // ---------------------------------------------------------------------------------------------
 // backward 1: "Update PV[i]" for every i in I_U (Algorithm 2), candidate keys, hot-row tasks, counters
 // ---------------------------------------------------------------------------------------------
-__global__ void k_priority(State s, Work w, uint32_t step, uint32_t* __restrict__ ckey) {
+__global__ void __launch_bounds__(256)
+k_priority(State s, Work w, uint32_t step, uint32_t* __restrict__ ckey) {
     if (w.ctr->abort) return;
+    constexpr int Q = 4;                                     // independent rows per thread: the counter updates are random accesses
     const int64_t U = w.ctr->U;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int64_t U32 = (U + 31) & ~31LL;
-    for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < U32; k += (int64_t)gridDim.x * blockDim.x) {
-        int t = -1; unsigned long long m = 0, hitm = 0, uh = 0, un = 0;
-        if (k < U) {
-            t = w.uniq_t[k];
-            const TableDev tb = s.tables[t];
-            const int32_t row = w.uniq_row[k];
-            const int loc = w.loc[k];
-            const uint32_t mult = (uint32_t)(w.seg[k + 1] - w.seg[k]);
-            uint32_t key = (uint32_t)tb.n_sets;              // sorts behind every real set: not a candidate
-            if (loc != LOC_INVALID) {
-                m = mult; un = 1;
-                if (s.policy == 1) {                         // LFU: access count of the row, saturating
-                    uint32_t* c = s.cnt + tb.row_base + row;
-                    const uint32_t old = *c;
-                    *c = old + mult < old ? 0xffffffffU : old + mult;
-                } else if (loc >= 0) {
-                    s.ts[loc] = step;                        // LRU: time stamp of the cached row
-                }
-                if (loc >= 0) { hitm = mult; uh = 1; }
-                else if (tb.n_sets > 0) key = (uint32_t)w.uset[k];
-            }
-            ckey[k] = key;
+    for (int64_t k0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k0 < U32; k0 += Q * stride) {
+        int t[Q], loc[Q]; int32_t row[Q]; uint32_t mult[Q], old[Q]; int64_t rb[Q]; int32_t nsets[Q];
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            const int64_t k = k0 + q * stride;
+            t[q] = -1;
+            if (k < U) { t[q] = w.uniq_t[k]; row[q] = w.uniq_row[k]; loc[q] = w.loc[k]; mult[q] = (uint32_t)(w.seg[k + 1] - w.seg[k]); }
         }
-        // counters: one atomic per warp when the warp sits inside one table
-        const int t0 = __shfl_sync(0xffffffffU, t, 0);
-        const bool same = __all_sync(0xffffffffU, t == t0 || t < 0);
-        if (same && t0 >= 0) {
-            for (int o = 16; o > 0; o >>= 1) {
-                m += __shfl_xor_sync(0xffffffffU, m, o); hitm += __shfl_xor_sync(0xffffffffU, hitm, o);
-                uh += __shfl_xor_sync(0xffffffffU, uh, o); un += __shfl_xor_sync(0xffffffffU, un, o);
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            old[q] = 0;
+            if (t[q] >= 0) {
+                const TableDev tb = s.tables[t[q]];
+                rb[q] = tb.row_base; nsets[q] = tb.n_sets;
+                if (s.policy == 1 && loc[q] != LOC_INVALID) old[q] = s.cnt[rb[q] + row[q]];
             }
-            if ((threadIdx.x & 31) == 0) {
-                unsigned long long* st = s.stats + (int64_t)t0 * 8;
+        }
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            const int64_t k = k0 + q * stride;
+            unsigned long long m = 0, hitm = 0, uh = 0, un = 0;
+            if (t[q] >= 0) {
+                uint32_t key = (uint32_t)nsets[q];           // sorts behind every real set: not a candidate
+                if (loc[q] != LOC_INVALID) {
+                    m = mult[q]; un = 1;
+                    if (s.policy == 1) {                     // LFU: access count of the row, saturating
+                        s.cnt[rb[q] + row[q]] = old[q] + mult[q] < old[q] ? 0xffffffffU : old[q] + mult[q];
+                    } else if (loc[q] >= 0) {
+                        s.ts[loc[q]] = step;                 // LRU: time stamp of the cached row
+                    }
+                    if (loc[q] >= 0) { hitm = mult[q]; uh = 1; }
+                    else if (nsets[q] > 0) key = (uint32_t)w.uset[k];
+                }
+                ckey[k] = key;
+            }
+            // counters: one atomic per warp when the warp sits inside one table
+            if (k0 + q * stride - (threadIdx.x & 31) >= U32) continue;       // warp-uniform: nothing left for this q
+            const int t0 = __shfl_sync(0xffffffffU, t[q], 0);
+            const bool same = __all_sync(0xffffffffU, t[q] == t0 || t[q] < 0);
+            if (same && t0 >= 0) {
+                for (int o = 16; o > 0; o >>= 1) {
+                    m += __shfl_xor_sync(0xffffffffU, m, o); hitm += __shfl_xor_sync(0xffffffffU, hitm, o);
+                    uh += __shfl_xor_sync(0xffffffffU, uh, o); un += __shfl_xor_sync(0xffffffffU, un, o);
+                }
+                if ((threadIdx.x & 31) == 0) {
+                    unsigned long long* st = s.stats + (int64_t)t0 * 8;
+                    atomicAdd(st + 0, m); atomicAdd(st + 1, hitm); atomicAdd(st + 2, un); atomicAdd(st + 3, uh);
+                }
+            } else if (t[q] >= 0) {
+                unsigned long long* st = s.stats + (int64_t)t[q] * 8;
                 atomicAdd(st + 0, m); atomicAdd(st + 1, hitm); atomicAdd(st + 2, un); atomicAdd(st + 3, uh);
             }
-        } else if (t >= 0) {
-            unsigned long long* st = s.stats + (int64_t)t * 8;
-            atomicAdd(st + 0, m); atomicAdd(st + 1, hitm); atomicAdd(st + 2, un); atomicAdd(st + 3, uh);
         }
     }
 }
