@@ -511,10 +511,10 @@ k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __r
                 if (s.policy == 1) cpv = s.cnt[tb.row_base + crow];
             }
             const int n = __popc(__ballot_sync(gmask, valid) & gmask);   // the valid lanes are a prefix of the group
-            for (int u = 0; u < n; ++u) {
-                const int32_t kk = __shfl_sync(gmask, ckk, gbase + u);
-                const int32_t row = __shfl_sync(gmask, crow, gbase + u);
-                const uint32_t pv = __shfl_sync(gmask, cpv, gbase + u);
+            // Between two replacements the set does not change, so every candidate that cannot beat the current
+            // minimum bypasses at once; only the candidates that replace are walked one by one.
+            int u = 0;
+            while (u < n) {
                 // empty ways rank below every priority; ties go to the lowest way
                 const uint32_t empties = __ballot_sync(gmask, tag < 0) & gmask;
                 int jw; bool jempty; uint32_t jpri = 0;
@@ -524,22 +524,27 @@ k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __r
                     jw = __ffs(__ballot_sync(gmask, pri == jpri) & gmask) - 1 - gbase;
                     jempty = false;
                 }
-                bool replace = jempty || pv > jpri;
-                if (ways == 1 && s.policy == 0) replace = true;              // direct-mapped LRU never compares
-                if (replace) {
-                    ++n_admit;
-                    if (!jempty) ++n_evict;
-                    if (way == jw) {
-                        if (tag >= 0 && cand < 0) {
-                            // a row that was resident when the step began leaves the cache
-                            if (s.hit_epoch[slot] == epoch) { w.final_loc[s.hit_k[slot]] = LOC_MISS; vict = VICTIM_DEFER; }
-                            else vict = tag;
-                        }
-                        tag = row; pri = pv; cand = kk;
+                // lane `way` holds candidate number `way` of this batch
+                const bool always = ways == 1 && s.policy == 0;                 // direct-mapped LRU never compares
+                const bool would = valid && way >= u && (jempty || always || cpv > jpri);
+                const uint32_t wm = (__ballot_sync(gmask, would) & gmask) >> gbase;
+                if (wm == 0) { n_bypass += (uint32_t)(n - u); break; }
+                const int f = __ffs(wm) - 1;                                    // the first candidate that replaces
+                n_bypass += (uint32_t)(f - u);
+                const int32_t kk = __shfl_sync(gmask, ckk, gbase + f);
+                const int32_t row = __shfl_sync(gmask, crow, gbase + f);
+                const uint32_t pv = __shfl_sync(gmask, cpv, gbase + f);
+                ++n_admit;
+                if (!jempty) ++n_evict;
+                if (way == jw) {
+                    if (tag >= 0 && cand < 0) {
+                        // a row that was resident when the step began leaves the cache
+                        if (s.hit_epoch[slot] == epoch) { w.final_loc[s.hit_k[slot]] = LOC_MISS; vict = VICTIM_DEFER; }
+                        else vict = tag;
                     }
-                } else {
-                    ++n_bypass;
+                    tag = row; pri = pv; cand = kk;
                 }
+                u = f + 1;
             }
             if (n < ways) break;
         }
