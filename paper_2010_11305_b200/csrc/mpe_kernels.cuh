@@ -707,8 +707,8 @@ __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefe
 struct RawRow { float4 f; uint32_t q; float2 sb; };
 
 constexpr int UPD_WARPS = 4;     // warps per block of k_update
-constexpr int UPD_RING = 16;     // gradient rows a group can have in shared memory
-constexpr int UPD_GROUPS = 4;    // copy groups a group keeps in flight (each up to 4 rows)
+constexpr int UPD_RING = 8;      // gradient rows a group can have in shared memory
+constexpr int UPD_GROUPS = 2;    // copy groups a group keeps in flight (each up to 4 rows)
 constexpr int UPD_NB = 4;        // rows per copy group
 constexpr int UPD_META = 16;     // ints of bookkeeping per staged row
 constexpr int UPD_SMEM = UPD_WARPS * (UPD_RING * 32 * 16 + 32 * UPD_META * 4);
