@@ -391,7 +391,7 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
         LAUNCH(h, "policy", k_policy, grid_for(h, std::min<int64_t>(L, h->total_sets), 256 / s.ways, 8), 256, 0, s, w, ck, cv,
                (uint32_t)step, h->epoch);
     }
-    const int gu = grid_for(h, (L + 31) / 32, UPD_WARPS, 7);
+    const int gu = grid_for(h, (L + 31) / 32, UPD_WARPS, 8);
     const int gh = grid_for(h, L / HOT_MIN + 1, 256 / s.lanes, 4);
     dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
         constexpr int BITS = decltype(bc)::value, LANES = decltype(lc)::value;

@@ -721,7 +721,7 @@ constexpr int UPD_SMEM = UPD_WARPS * (UPD_RING * 32 * 16 + 32 * UPD_META * 4);
 // while earlier ones are being added (in index order, radix-32 tree), independent of where one
 // embedding row ends and the next begins.
 template <int BITS, int LANES>
-__global__ void __launch_bounds__(UPD_WARPS * 32)
+__global__ void __launch_bounds__(UPD_WARPS * 32, 8)
 k_update(State s, Work w, const float* __restrict__ grad, int B, float lr, uint64_t step) {
     extern __shared__ __align__(16) unsigned char upd_smem[];
     if (w.ctr->abort) return;
