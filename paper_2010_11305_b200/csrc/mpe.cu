@@ -159,7 +159,7 @@ int seg_sort(mpe_handle* h, uint32_t* kA, uint32_t* kB, uint32_t* vA, uint32_t* 
     const int T = h->T;
     LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, seg_start, T, tile_base, hist_len, (const uint32_t*)&h->wk.ctr->abort);
     const int64_t max_tiles = (n_upper + SORT_TILE - 1) / SORT_TILE + T;
-    const int g = grid_for(h, max_tiles, 1, 3);
+    const int g = grid_for(h, max_tiles, 1, 5);
     const int passes = (key_bits + 7) / 8;
     uint32_t *kin = kA, *kout = kB, *vin = nullptr, *vout = vB;
     for (int p = 0; p < passes; ++p) {
@@ -733,7 +733,7 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, (const int32_t*)w.table_start, T, w.tile_base, &w.ctr->hist_len,
            (const uint32_t*)&w.ctr->abort);
     const int64_t tiles_upper = (total_indices + SORT_TILE - 1) / SORT_TILE + T;
-    const int gsort = grid_for(h, tiles_upper, 1, 3);
+    const int gsort = grid_for(h, tiles_upper, 1, 5);
     const int gscan = grid_for(h, 256 * tiles_upper, SCAN_TILE, 8);
     const int passes = (bits_for((uint32_t)h->max_rows) + 7) / 8;
     uint32_t *kin = keyA, *kout = keyB, *vin = nullptr, *vout = valB;

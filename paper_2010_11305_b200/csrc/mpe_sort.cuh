@@ -14,8 +14,8 @@
 namespace mpe {
 
 constexpr int SORT_THREADS = 256;
-constexpr int SORT_ITEMS = 16;
-constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;   // 4096 keys per block
+constexpr int SORT_ITEMS = 8;
+constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;   // keys per block
 constexpr int SCAN_THREADS = 256;
 constexpr int SCAN_ITEMS = 16;
 constexpr int SCAN_TILE = SCAN_THREADS * SCAN_ITEMS;
@@ -102,7 +102,7 @@ k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_s
 
 // ---- pass 3 of 3: stable scatter ------------------------------------------------
 // vals_in == nullptr means "the payload is the element's position" (first pass).
-__global__ void __launch_bounds__(SORT_THREADS, 3)
+__global__ void __launch_bounds__(SORT_THREADS, 5)
 k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
                uint32_t* __restrict__ keys_out, uint32_t* __restrict__ vals_out,
                const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base, int T, int shift,
