@@ -45,6 +45,8 @@ struct mpe_handle {
     cudaStream_t stream = nullptr;
     cudaStream_t side = nullptr;            // runs the hot rows' partial sums next to the policy kernels
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;   // mpe_step_host: host<->device copies next to the kernels
+    cudaEvent_t ev_idx = nullptr, ev_grad = nullptr, ev_fwd = nullptr, ev_start = nullptr;
     bool have_forward = false;
     int64_t last_step = 0;
     uint64_t steps = 0;
@@ -241,7 +243,13 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
     cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, device);
     if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess) { delete h; return MPE_ERR_CUDA; }
+        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_idx, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_grad, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_fwd, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming) != cudaSuccess) { delete h; return MPE_ERR_CUDA; }
     h->T = num_tables; h->dim = dim; h->bits = bits; h->ways = ways; h->policy = policy; h->optimizer = optimizer;
     h->code_bytes = dim * bits / 8; h->eps = eps; h->lo = init_lo; h->hi = init_hi; h->seed = seed;
     h->tables.resize(num_tables);
@@ -433,16 +441,27 @@ int mpe_step_host(mpe_handle* h, const int32_t* h_indices, const int32_t* h_offs
         if ((rc = dmalloc(h, &h->sh_grad, h->sh_cap_out, nullptr)) != MPE_OK) return rc;
         if ((rc = dmalloc(h, &h->sh_out, h->sh_cap_out, nullptr)) != MPE_OK) return rc;
     }
+    // The gradient upload runs next to the forward kernels and the output download next to the backward
+    // kernels (PCIe moves data in both directions at once); only the indices are needed before anything starts.
     cudaStream_t st = h->stream;
-    if (total_indices) CK(h, cudaMemcpyAsync(h->sh_idx, h_indices, sizeof(int32_t) * total_indices, cudaMemcpyHostToDevice, st));
-    CK(h, cudaMemcpyAsync(h->sh_off, h_offsets, sizeof(int32_t) * noff, cudaMemcpyHostToDevice, st));
-    if (nout) CK(h, cudaMemcpyAsync(h->sh_grad, h_grad_out, sizeof(float) * nout, cudaMemcpyHostToDevice, st));
+    CK(h, cudaEventRecord(h->ev_start, st));
+    CK(h, cudaStreamWaitEvent(h->copy_in, h->ev_start, 0));
+    if (total_indices) CK(h, cudaMemcpyAsync(h->sh_idx, h_indices, sizeof(int32_t) * total_indices, cudaMemcpyHostToDevice, h->copy_in));
+    CK(h, cudaMemcpyAsync(h->sh_off, h_offsets, sizeof(int32_t) * noff, cudaMemcpyHostToDevice, h->copy_in));
+    CK(h, cudaEventRecord(h->ev_idx, h->copy_in));
+    if (nout) CK(h, cudaMemcpyAsync(h->sh_grad, h_grad_out, sizeof(float) * nout, cudaMemcpyHostToDevice, h->copy_in));
+    CK(h, cudaEventRecord(h->ev_grad, h->copy_in));
+    CK(h, cudaStreamWaitEvent(st, h->ev_idx, 0));
     int rc = mpe_forward(h, h->sh_idx, h->sh_off, batch, total_indices, h->sh_out, (void*)st);
-    if (rc != MPE_OK) return rc;
+    if (rc != MPE_OK) { cudaStreamSynchronize(h->copy_in); return rc; }
+    CK(h, cudaEventRecord(h->ev_fwd, st));
+    CK(h, cudaStreamWaitEvent(h->copy_out, h->ev_fwd, 0));
+    if (nout) CK(h, cudaMemcpyAsync(h_out, h->sh_out, sizeof(float) * nout, cudaMemcpyDeviceToHost, h->copy_out));
+    CK(h, cudaStreamWaitEvent(st, h->ev_grad, 0));
     rc = mpe_backward(h, h->sh_grad, lr, step);
+    cudaError_t e1 = cudaStreamSynchronize(h->copy_out), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(h->copy_in);
     if (rc != MPE_OK) return rc;
-    if (nout) CK(h, cudaMemcpyAsync(h_out, h->sh_out, sizeof(float) * nout, cudaMemcpyDeviceToHost, st));
-    CK(h, cudaStreamSynchronize(st));
+    CK(h, e1); CK(h, e2); CK(h, e3);
     return MPE_OK;
 }
 
@@ -467,6 +486,9 @@ int mpe_destroy(mpe_handle* h) {
     if (h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); }
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->copy_in) { cudaStreamSynchronize(h->copy_in); cudaStreamDestroy(h->copy_in); }
+    if (h->copy_out) { cudaStreamSynchronize(h->copy_out); cudaStreamDestroy(h->copy_out); }
+    for (cudaEvent_t e : {h->ev_idx, h->ev_grad, h->ev_fwd, h->ev_start}) if (e) cudaEventDestroy(e);
     free_workspace(h);
     State& s = h->st;
     cudaFree(h->d_tables); cudaFree(s.codes); cudaFree(s.sb); cudaFree(s.cnt); cudaFree(s.G); cudaFree(s.slab);
