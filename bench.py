@@ -313,6 +313,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep5", action="store_true", help="run every point of the policy/skew sweep (configuration 5): one JSON line per point")
     ap.add_argument("--tables", type=int, default=None, help="profiling aid: keep only the first TABLES tables")
     ap.add_argument("--rows-div", type=int, default=1, help="profiling aid: divide every table's row count")
     ap.add_argument("--batch-div", type=int, default=1, help="profiling aid: divide the batch size")
@@ -346,6 +347,16 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if args.sweep5:
+        # hit rate, rows/s and effective GB/s per point; 50 warm-up steps fill the caches, then `--steps` are timed
+        args.e2e_steps = 0
+        args.warmup = max(args.warmup, 50)
+        for point in wl.sweep5():
+            r = run_ours(args, point, 0, 1, local_rank)
+            print(json.dumps({"point": point.name, "rows_per_s": r["value"], "ms_per_step": r["ms_per_step"],
+                              "index_hit_rate": r["per_step"]["index_hit_rate"], "effective_gbs": r["effective"]["gbs"],
+                              "distinct_rows": r["per_step"]["distinct_rows"], "gpu_launches": r["gpu_launches"]}), flush=True)
+        return
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     result = run_ours(args, cfg, rank, world, local_rank)
