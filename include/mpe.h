@@ -178,6 +178,12 @@ int mpe_export_cache(mpe_handle* h, int32_t table, int32_t* h_tags, float* h_row
 int mpe_export_aux(mpe_handle* h, int32_t table, const int64_t* h_rows, int64_t n, uint32_t* h_cnt,
                    float* h_adagrad);
 
+/* Steps of up to about four million indices are bound by kernel-launch latency, so by default each half of
+ * the step is captured once into a CUDA graph (sized for the reserved workspace) and replayed; the per-call
+ * arguments reach the kernels through device memory.  enable = 0 switches to plain launches (larger steps and
+ * steps issued while profiling or while the caller captures the stream always use plain launches). */
+int mpe_use_graphs(mpe_handle* h, int32_t enable);
+
 /* ---- instrumentation ---------------------------------------------------------------------------- */
 /* Number of kernels this handle has launched so far. */
 int mpe_kernel_launches(mpe_handle* h, uint64_t* count);

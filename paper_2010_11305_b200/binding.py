@@ -22,7 +22,7 @@ STATIC_MAX_INDICES, STATIC_MAX_BAGS, STATIC_MAX_TABLES = 32768, 32768, 64
 EXPORTS = [
     "mpe_create", "mpe_reserve", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_step_host", "mpe_flush", "mpe_destroy",
     "mpe_last_error", "mpe_stats", "mpe_memory_bytes", "mpe_cache_geometry", "mpe_step_info", "mpe_export_rows",
-    "mpe_export_cache", "mpe_export_aux", "mpe_kernel_launches", "mpe_profile", "mpe_profile_read", "mpe_error_string",
+    "mpe_export_cache", "mpe_export_aux", "mpe_use_graphs", "mpe_kernel_launches", "mpe_profile", "mpe_profile_read", "mpe_error_string",
 ]
 
 
@@ -55,6 +55,7 @@ _lib.mpe_step_info.argtypes = [_vp, _vp]
 _lib.mpe_export_rows.argtypes = [_vp, _i32, _vp, _i64, _vp, _vp, _vp]
 _lib.mpe_export_cache.argtypes = [_vp, _i32, _vp, _vp, _vp]
 _lib.mpe_export_aux.argtypes = [_vp, _i32, _vp, _i64, _vp, _vp]
+_lib.mpe_use_graphs.argtypes = [_vp, _i32]
 _lib.mpe_kernel_launches.argtypes = [_vp, C.POINTER(_u64)]
 _lib.mpe_profile.argtypes = [_vp, _i32]
 _lib.mpe_profile_read.argtypes = [_vp, _i32, _vp, _vp, _vp, C.POINTER(_i32)]
@@ -184,6 +185,9 @@ class Mpe:
         G = np.zeros(max(rows.size, 1), np.float32)
         _check(_lib.mpe_export_aux(self._h, table, rows.ctypes.data, rows.size, cnt.ctypes.data, G.ctypes.data), "mpe_export_aux")
         return cnt[:rows.size], G[:rows.size]
+
+    def use_graphs(self, enable):
+        _check(_lib.mpe_use_graphs(self._h, 1 if enable else 0), "mpe_use_graphs")
 
     # ---- instrumentation --------------------------------------------------------------------
     def kernel_launches(self):

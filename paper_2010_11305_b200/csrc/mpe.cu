@@ -53,6 +53,14 @@ struct mpe_handle {
     uint32_t epoch = 0;
     int32_t B = 0; int64_t L = 0;
     const uint32_t *skey = nullptr, *spos = nullptr;
+    StepArgs args{};                        // the current call's arguments (passed by value when launching directly)
+    // CUDA graphs of the two halves of a step (small batches are launch-latency bound)
+    bool graphs_enabled = true;
+    cudaStream_t cap = nullptr;             // stream the step is captured on
+    cudaGraph_t g_fwd = nullptr, g_bwd = nullptr;
+    cudaGraphExec_t x_fwd = nullptr, x_bwd = nullptr;
+    cudaGraphNode_t n_fwd = nullptr, n_bwd = nullptr;      // the nodes that write the per-call arguments
+    uint64_t k_fwd = 0, k_bwd = 0;                         // kernel nodes per graph
     // instrumentation
     uint64_t launches = 0;
     bool profiling = false;
@@ -113,7 +121,16 @@ int dmalloc(mpe_handle* h, T** p, int64_t n, std::vector<void*>* track) {
     return MPE_OK;
 }
 
+void drop_graphs(mpe_handle* h) {
+    if (h->x_fwd) cudaGraphExecDestroy(h->x_fwd);
+    if (h->x_bwd) cudaGraphExecDestroy(h->x_bwd);
+    if (h->g_fwd) cudaGraphDestroy(h->g_fwd);
+    if (h->g_bwd) cudaGraphDestroy(h->g_bwd);
+    h->x_fwd = h->x_bwd = nullptr; h->g_fwd = h->g_bwd = nullptr; h->n_fwd = h->n_bwd = nullptr;
+}
+
 void free_workspace(mpe_handle* h) {
+    drop_graphs(h);                       // they hold the workspace's addresses
     for (void* p : h->ws_allocs) cudaFree(p);
     h->ws_allocs.clear();
     h->cap_L = 0; h->cap_bags = 0;
@@ -133,7 +150,7 @@ int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
     const int64_t max_tiles = (L + SORT_TILE - 1) / SORT_TILE + T + 1;
     A(h->hist, 256 * max_tiles);
     A(h->block_sums, std::max<int64_t>(256 * max_tiles, n) / SCAN_TILE + 2);
-    A(w.ctr, 1);
+    A(w.ctr, 1); A(w.args, 1);
     A(w.table_start, T + 1); A(w.tile_base, T + 1); A(w.ustart, T + 1); A(w.ctile_base, T + 1);
     A(w.bag_of, n); A(w.kidx, n); A(w.occ_loc, n); A(w.occ_b, n);
     A(w.uniq_row, n); A(w.uniq_t, n); A(w.seg, n + 1); A(w.loc, n); A(w.final_loc, n); A(w.victim, n);
@@ -242,6 +259,7 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
     DeviceGuard guard(device);
     cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, device);
     if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&h->cap, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess ||
         cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking) != cudaSuccess ||
@@ -320,6 +338,135 @@ int mpe_reserve(mpe_handle* h, int32_t max_batch, int64_t max_total_indices) {
     return alloc_workspace(h, std::max(max_total_indices, h->cap_L), std::max(bags, h->cap_bags));
 }
 
+}  // extern "C"
+
+namespace {
+
+// Launch sizes follow L_grid / bags_grid (upper bounds: every kernel walks its range with a grid stride and reads the
+// true sizes from device memory), so one captured graph serves every batch that fits the workspace.
+int enqueue_forward(mpe_handle* h, int64_t L_grid, int64_t bags_grid, bool ind) {
+    const State& s = h->st;
+    Work& w = h->wk;
+    const int T = h->T;
+    const StepArgs av = h->args;
+    LAUNCH(h, "prelude", (ind ? k_prelude<true> : k_prelude<false>), 1, 32, 0, w, T, av);
+    LAUNCH(h, "make_keys", (ind ? k_make_keys<true> : k_make_keys<false>), grid_for(h, bags_grid, 32, 8), 256, 0, s, w, h->keyA, av);
+    // sort the row indices of the mini-batch (Section 5.1), table by table
+    const int which = seg_sort(h, h->keyA, h->keyB, h->valA, h->valB, w.table_start, w.tile_base, &w.ctr->hist_len,
+                               bits_for((uint32_t)h->max_rows), L_grid);
+    h->skey = which ? h->keyB : h->keyA;
+    h->spos = which ? h->valB : h->valA;
+    // distinct rows
+    const int gs = grid_for(h, L_grid, SCAN_TILE, 8);
+    LAUNCH(h, "unique_count", k_unique<false>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
+    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);
+    LAUNCH(h, "unique_write", k_unique<true>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
+    LAUNCH(h, "ustart", k_ustart, 1, 256, 0, w, T);
+    // tag lookup, then fetch + pool
+    LAUNCH(h, "probe", (ind ? k_probe<true> : k_probe<false>), grid_for(h, L_grid, 256, 8), 256, 0, s, w, av);
+    LAUNCH(h, "broadcast", (ind ? k_broadcast<true> : k_broadcast<false>), grid_for(h, L_grid, 256, 8), 256, 0, s, w, h->spos, av);
+    const int gp = grid_for(h, bags_grid, 256 / s.lanes, 8);
+    dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
+        constexpr int BITS = decltype(bc)::value, LANES = decltype(lc)::value;
+        auto kern = ind ? k_pool<BITS, LANES, true> : k_pool<BITS, LANES, false>;
+        LAUNCH(h, "pool", kern, gp, 256, 0, s, w, av);
+    });
+    return check_launch(h);
+}
+
+int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
+    const State& s = h->st;
+    Work& w = h->wk;
+    const StepArgs av = h->args;
+    // the hot rows' partial gradient sums only need the sorted batch: they run on a second stream next to the
+    // priority / candidate-sort / policy kernels, which leave most of the machine idle
+    CK(h, cudaEventRecord(h->ev_fork, h->stream));
+    CK(h, cudaStreamWaitEvent(h->side, h->ev_fork, 0));
+    dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
+        constexpr int LANES = decltype(lc)::value;
+        auto hot = ind ? k_hot_partial<LANES, true> : k_hot_partial<LANES, false>;
+        LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, L / HOT_MIN + 1, 1, 1), 8 * LANES, 32 * s.dim * sizeof(float), s, w, av);
+    });
+    CK(h, cudaEventRecord(h->ev_join, h->side));
+    LAUNCH(h, "priority", (ind ? k_priority<true> : k_priority<false>), grid_for(h, L, 1024, 8), 256, 0, s, w, h->ckeyA, av);
+    if (h->max_sets > 0) {
+        // group the rows that missed by cache set, keeping ascending row id inside a set
+        const int which = seg_sort(h, h->ckeyA, h->ckeyB, h->cvalA, h->cvalB, w.ustart, w.ctile_base, &w.ctr->chist_len,
+                                   bits_for((uint32_t)h->max_sets), L);
+        const uint32_t* ck = which ? h->ckeyB : h->ckeyA;
+        const uint32_t* cv = which ? h->cvalB : h->cvalA;
+        LAUNCH(h, "policy_heads", k_policy_heads, grid_for(h, L, 256, 8), 256, 0, s, w, ck);
+        LAUNCH(h, "policy", (ind ? k_policy<true> : k_policy<false>), grid_for(h, std::min<int64_t>(L, h->total_sets), 256 / s.ways, 8), 256, 0, s, w, ck, cv, av);
+    }
+    const int gu = grid_for(h, (L + 31) / 32, UPD_WARPS, 8);
+    const int gh = grid_for(h, L / HOT_MIN + 1, 256 / s.lanes, 4);
+    dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
+        constexpr int BITS = decltype(bc)::value, LANES = decltype(lc)::value;
+        auto upd = ind ? k_update<BITS, LANES, true> : k_update<BITS, LANES, false>;
+        auto lst = ind ? k_update_list<BITS, LANES, true> : k_update_list<BITS, LANES, false>;
+        static bool smem_set = false;     // one flag per instantiation of this lambda
+        if (!smem_set) {
+            cudaFuncSetAttribute(k_update<BITS, LANES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, UPD_SMEM);
+            cudaFuncSetAttribute(k_update<BITS, LANES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, UPD_SMEM);
+            smem_set = true;
+        }
+        LAUNCH(h, "update", upd, gu, UPD_WARPS * 32, UPD_SMEM, s, w, av);
+        cudaStreamWaitEvent(h->stream, h->ev_join, 0);
+        LAUNCH(h, "update_hot", lst, gh, 256, 0, s, w, (const int32_t*)w.hot_k, (const uint32_t*)&w.ctr->hot_rows, 0, av);
+        if (h->max_sets > 0)
+            LAUNCH(h, "update_deferred", lst, gh, 256, 0, s, w, (const int32_t*)w.defer_k, (const uint32_t*)&w.ctr->deferred, 1, av);
+    });
+    return check_launch(h);
+}
+
+// Steps this small are bound by launch latency; above it the launches hide behind the kernels.
+constexpr int64_t GRAPH_MAX_INDICES = 4 << 20;
+
+bool may_use_graph(mpe_handle* h) {
+    if (!h->graphs_enabled || h->profiling || h->cap_L > GRAPH_MAX_INDICES) return false;
+    cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(h->stream, &st) != cudaSuccess || st != cudaStreamCaptureStatusNone) return false;   // the caller captures: plain launches join his graph
+    return true;
+}
+
+// Capture one half of the step (sized for the whole workspace) into a graph; `head` is the kernel that writes the arguments.
+template <class Body>
+int capture(mpe_handle* h, cudaGraph_t* graph, cudaGraphExec_t* exec, cudaGraphNode_t* args_node, uint64_t* kernels, const void* head,
+            Body&& body) {
+    cudaStream_t user = h->stream;
+    const uint64_t launches_before = h->launches;
+    h->stream = h->cap;
+    cudaError_t e = cudaStreamBeginCapture(h->cap, cudaStreamCaptureModeThreadLocal);
+    int rc = MPE_OK;
+    if (e == cudaSuccess) {
+        rc = body();
+        e = cudaStreamEndCapture(h->cap, graph);
+    }
+    h->stream = user;
+    h->launches = launches_before;
+    if (e != cudaSuccess || rc != MPE_OK || !*graph) { h->last_cuda_error = (int)e; cudaGetLastError(); return rc != MPE_OK ? rc : MPE_ERR_CUDA; }
+    CK(h, cudaGraphInstantiate(exec, *graph, 0));
+    size_t n = 0;
+    CK(h, cudaGraphGetNodes(*graph, nullptr, &n));
+    std::vector<cudaGraphNode_t> nodes(n);
+    CK(h, cudaGraphGetNodes(*graph, nodes.data(), &n));
+    *args_node = nullptr; *kernels = 0;
+    for (cudaGraphNode_t nd : nodes) {
+        cudaGraphNodeType ty;
+        CK(h, cudaGraphNodeGetType(nd, &ty));
+        if (ty != cudaGraphNodeTypeKernel) continue;
+        ++*kernels;
+        cudaKernelNodeParams kp{};
+        CK(h, cudaGraphKernelNodeGetParams(nd, &kp));
+        if (kp.func == head) *args_node = nd;
+    }
+    return *args_node ? MPE_OK : MPE_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
 int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch,
                 int64_t total_indices, float* d_out, void* cuda_stream) {
     if (!h || !d_offsets || batch < 0 || total_indices < 0 || total_indices > 0x7ffffff0LL) return MPE_ERR_ARG;
@@ -333,34 +480,32 @@ int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offset
         int rc = mpe_reserve(h, batch, total_indices);
         if (rc != MPE_OK) return rc;
     }
-    const State& s = h->st;
     Work& w = h->wk;
-    const int T = h->T;
-    const uint32_t L = (uint32_t)total_indices;
+    uint32_t L = (uint32_t)total_indices;
     h->B = batch; h->L = total_indices; ++h->epoch;
-
-    LAUNCH(h, "prelude", k_prelude, 1, 32, 0, w, d_offsets, T, batch, L);
-    LAUNCH(h, "make_keys", k_make_keys, grid_for(h, bags, 32, 8), 256, 0, s, w, d_indices, d_offsets, batch, h->keyA);
-    // sort the row indices of the mini-batch (Section 5.1), table by table
-    const int which = seg_sort(h, h->keyA, h->keyB, h->valA, h->valB, w.table_start, w.tile_base, &w.ctr->hist_len,
-                               bits_for((uint32_t)h->max_rows), total_indices);
-    h->skey = which ? h->keyB : h->keyA;
-    h->spos = which ? h->valB : h->valA;
-    // distinct rows
-    const int gs = grid_for(h, total_indices, SCAN_TILE, 8);
-    LAUNCH(h, "unique_count", k_unique<false>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
-    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);
-    LAUNCH(h, "unique_write", k_unique<true>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
-    LAUNCH(h, "ustart", k_ustart, 1, 256, 0, w, T);
-    // tag lookup, then fetch + pool
-    LAUNCH(h, "probe", k_probe, grid_for(h, total_indices, 256, 8), 256, 0, s, w, h->epoch);
-    LAUNCH(h, "broadcast", k_broadcast, grid_for(h, total_indices, 256, 8), 256, 0, s, w, h->spos, batch);
-    const int gp = grid_for(h, bags, 256 / s.lanes, 8);
-    dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
-        auto kern = k_pool<decltype(bc)::value, decltype(lc)::value>;
-        LAUNCH(h, "pool", kern, gp, 256, 0, s, w, d_indices, d_offsets, batch, d_out);
-    });
-    int rc = check_launch(h);
+    h->args.indices = d_indices; h->args.offsets = d_offsets; h->args.out = d_out; h->args.B = batch; h->args.L = L; h->args.epoch = h->epoch;
+    int rc = MPE_OK;
+    if (may_use_graph(h)) {
+        if (!h->x_fwd) {
+            rc = capture(h, &h->g_fwd, &h->x_fwd, &h->n_fwd, &h->k_fwd, (const void*)k_set_args_forward, [&]() {
+                LAUNCH(h, "set_args", k_set_args_forward, 1, 1, 0, w.args, d_indices, d_offsets, d_out, batch, L, h->epoch);
+                return enqueue_forward(h, h->cap_L, h->cap_bags, true);
+            });
+            if (rc != MPE_OK) { drop_graphs(h); h->graphs_enabled = false; }      // fall back to plain launches for good
+        }
+        if (rc == MPE_OK) {
+            StepArgs* a = w.args;
+            void* params[] = {&a, &d_indices, &d_offsets, &d_out, &batch, &L, &h->epoch};
+            cudaKernelNodeParams kp{};
+            kp.func = (void*)k_set_args_forward; kp.gridDim = dim3(1); kp.blockDim = dim3(1); kp.kernelParams = params;
+            CK(h, cudaGraphExecKernelNodeSetParams(h->x_fwd, h->n_fwd, &kp));
+            CK(h, cudaGraphLaunch(h->x_fwd, h->stream));
+            h->launches += h->k_fwd;
+            h->have_forward = true;
+            return MPE_OK;
+        }
+    }
+    rc = enqueue_forward(h, total_indices, bags, false);
     if (rc != MPE_OK) return rc;
     h->have_forward = true;
     return MPE_OK;
@@ -373,53 +518,43 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
     if (reinterpret_cast<uintptr_t>(d_grad_out) & 15) return MPE_ERR_ARG;   // rows are moved 16 bytes at a time
     if (step <= h->last_step) return MPE_ERR_SEQUENCE;
     DeviceGuard guard(h->device);
-    const State& s = h->st;
     Work& w = h->wk;
-    const int64_t L = h->L;
-    const int B = h->B;
-
-    // the hot rows' partial gradient sums only need the sorted batch: they run on a second stream next to the
-    // priority / candidate-sort / policy kernels, which leave most of the machine idle
-    CK(h, cudaEventRecord(h->ev_fork, h->stream));
-    CK(h, cudaStreamWaitEvent(h->side, h->ev_fork, 0));
-    dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
-        constexpr int LANES = decltype(lc)::value;
-        auto hot = k_hot_partial<LANES>;
-        LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, L / HOT_MIN + 1, 1, 1), 8 * LANES, 32 * s.dim * sizeof(float), s, w, d_grad_out, B);
-    });
-    CK(h, cudaEventRecord(h->ev_join, h->side));
-    LAUNCH(h, "priority", k_priority, grid_for(h, L, 1024, 8), 256, 0, s, w, (uint32_t)step, h->ckeyA);
-    if (h->max_sets > 0) {
-        // group the rows that missed by cache set, keeping ascending row id inside a set
-        const int which = seg_sort(h, h->ckeyA, h->ckeyB, h->cvalA, h->cvalB, w.ustart, w.ctile_base, &w.ctr->chist_len,
-                                   bits_for((uint32_t)h->max_sets), L);
-        const uint32_t* ck = which ? h->ckeyB : h->ckeyA;
-        const uint32_t* cv = which ? h->cvalB : h->cvalA;
-        LAUNCH(h, "policy_heads", k_policy_heads, grid_for(h, L, 256, 8), 256, 0, s, w, ck);
-        LAUNCH(h, "policy", k_policy, grid_for(h, std::min<int64_t>(L, h->total_sets), 256 / s.ways, 8), 256, 0, s, w, ck, cv,
-               (uint32_t)step, h->epoch);
+    unsigned long long ustep = (unsigned long long)step;
+    h->args.grad = d_grad_out; h->args.lr = lr; h->args.step = ustep;
+    int rc = MPE_OK;
+    bool done = false;
+    if (may_use_graph(h)) {
+        if (!h->x_bwd) {
+            rc = capture(h, &h->g_bwd, &h->x_bwd, &h->n_bwd, &h->k_bwd, (const void*)k_set_args_backward, [&]() {
+                LAUNCH(h, "set_args", k_set_args_backward, 1, 1, 0, w.args, d_grad_out, lr, ustep);
+                return enqueue_backward(h, h->cap_L, true);
+            });
+            if (rc != MPE_OK) { drop_graphs(h); h->graphs_enabled = false; }
+        }
+        if (rc == MPE_OK) {
+            StepArgs* a = w.args;
+            void* params[] = {&a, &d_grad_out, &lr, &ustep};
+            cudaKernelNodeParams kp{};
+            kp.func = (void*)k_set_args_backward; kp.gridDim = dim3(1); kp.blockDim = dim3(1); kp.kernelParams = params;
+            CK(h, cudaGraphExecKernelNodeSetParams(h->x_bwd, h->n_bwd, &kp));
+            CK(h, cudaGraphLaunch(h->x_bwd, h->stream));
+            h->launches += h->k_bwd;
+            done = true;
+        }
     }
-    const int gu = grid_for(h, (L + 31) / 32, UPD_WARPS, 8);
-    const int gh = grid_for(h, L / HOT_MIN + 1, 256 / s.lanes, 4);
-    dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
-        constexpr int BITS = decltype(bc)::value, LANES = decltype(lc)::value;
-        auto upd = k_update<BITS, LANES>;
-        auto lst = k_update_list<BITS, LANES>;
-        static bool smem_set = false;     // one flag per instantiation of this lambda
-        if (!smem_set) { cudaFuncSetAttribute(upd, cudaFuncAttributeMaxDynamicSharedMemorySize, UPD_SMEM); smem_set = true; }
-        LAUNCH(h, "update", upd, gu, UPD_WARPS * 32, UPD_SMEM, s, w, d_grad_out, B, lr, (uint64_t)step);
-        cudaStreamWaitEvent(h->stream, h->ev_join, 0);
-        LAUNCH(h, "update_hot", lst, gh, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step, (const int32_t*)w.hot_k,
-               (const uint32_t*)&w.ctr->hot_rows, 0);
-        if (h->max_sets > 0)
-            LAUNCH(h, "update_deferred", lst, gh, 256, 0, s, w, d_grad_out, B, lr, (uint64_t)step, (const int32_t*)w.defer_k,
-                   (const uint32_t*)&w.ctr->deferred, 1);
-    });
-    int rc = check_launch(h);
-    if (rc != MPE_OK) return rc;
+    if (!done) {
+        rc = enqueue_backward(h, h->L, false);
+        if (rc != MPE_OK) return rc;
+    }
     h->have_forward = false;
     h->last_step = step;
     ++h->steps;
+    return MPE_OK;
+}
+
+int mpe_use_graphs(mpe_handle* h, int32_t enable) {
+    if (!h) return MPE_ERR_ARG;
+    h->graphs_enabled = enable != 0;
     return MPE_OK;
 }
 
@@ -484,6 +619,7 @@ int mpe_destroy(mpe_handle* h) {
     DeviceGuard guard(h->device);
     cudaStreamSynchronize(h->stream);
     if (h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); }
+    if (h->cap) cudaStreamDestroy(h->cap);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->copy_in) { cudaStreamSynchronize(h->copy_in); cudaStreamDestroy(h->copy_in); }
@@ -693,7 +829,7 @@ constexpr size_t STATIC_SCRATCH_BYTES =
               STATIC_MAX_INDICES / SCAN_TILE + 2) * 4) +                                               // block sums
     4 * align256((STATIC_MAX_TABLES + 1) * 4) +                                                        // per-table starts
     2 * align256((STATIC_MAX_INDICES / HOT_MIN + 2) * 4) +                                             // hot-row lists
-    align256(sizeof(Counters));
+    align256(sizeof(Counters)) + align256(sizeof(StepArgs));
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress; it is not a device address.
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
@@ -741,6 +877,7 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     w.ustart = c.take<int32_t>(STATIC_MAX_TABLES + 1); w.ctile_base = c.take<int32_t>(STATIC_MAX_TABLES + 1);
     w.hot_k = c.take<int32_t>(STATIC_MAX_INDICES / HOT_MIN + 2); w.task_k = c.take<int32_t>(STATIC_MAX_INDICES / HOT_MIN + 2);
     w.ctr = c.take<Counters>(1);
+    w.args = c.take<StepArgs>(1);
     if (c.used > STATIC_SCRATCH_BYTES) return MPE_ERR_ARG;      // cannot happen: the size formula above mirrors this list
 
     const State& s = h->st;
@@ -749,8 +886,10 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     ++h->epoch;
     // the array keeps whatever the previous call left: the counters are the only part that must start from zero
     CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), stream));
-    LAUNCH(h, "prelude", k_prelude, 1, 32, 0, w, d_offsets, T, batch, L);
-    LAUNCH(h, "make_keys", k_make_keys, grid_for(h, bags, 32, 8), 256, 0, s, w, d_indices, d_offsets, batch, keyA);
+    StepArgs av{};
+    av.indices = d_indices; av.offsets = d_offsets; av.out = d_out; av.B = batch; av.L = L; av.epoch = h->epoch;
+    LAUNCH(h, "prelude", k_prelude<false>, 1, 32, 0, w, T, av);
+    LAUNCH(h, "make_keys", k_make_keys<false>, grid_for(h, bags, 32, 8), 256, 0, s, w, keyA, av);
     // segmented radix sort, as in mpe_forward, on the carved buffers
     LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, (const int32_t*)w.table_start, T, w.tile_base, &w.ctr->hist_len,
            (const uint32_t*)&w.ctr->abort);
@@ -778,12 +917,12 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);
     LAUNCH(h, "unique_write", k_unique<true>, gs, SCAN_THREADS, 0, w, T, skey, block_sums);
     LAUNCH(h, "ustart", k_ustart, 1, 256, 0, w, T);
-    LAUNCH(h, "probe", k_probe, grid_for(h, total_indices, 256, 8), 256, 0, s, w, h->epoch);
-    LAUNCH(h, "broadcast", k_broadcast, grid_for(h, total_indices, 256, 8), 256, 0, s, w, spos, batch);
+    LAUNCH(h, "probe", k_probe<false>, grid_for(h, total_indices, 256, 8), 256, 0, s, w, av);
+    LAUNCH(h, "broadcast", k_broadcast<false>, grid_for(h, total_indices, 256, 8), 256, 0, s, w, spos, av);
     const int gp = grid_for(h, bags, 256 / s.lanes, 8);
     dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
-        auto kern = k_pool<decltype(bc)::value, decltype(lc)::value>;
-        LAUNCH(h, "pool", kern, gp, 256, 0, s, w, d_indices, d_offsets, batch, d_out);
+        auto kern = k_pool<decltype(bc)::value, decltype(lc)::value, false>;
+        LAUNCH(h, "pool", kern, gp, 256, 0, s, w, av);
     });
     return check_launch(h);
 }

@@ -53,8 +53,17 @@ struct State {
     unsigned long long* stats;   // [T][8]
 };
 
+// What changes from call to call.  It lives in device memory so that a captured CUDA graph of the step stays valid:
+// the kernels read it, one tiny kernel at the head of the graph writes it.
+struct StepArgs {
+    const int32_t* indices; const int32_t* offsets; float* out; const float* grad;
+    int32_t B; uint32_t L; uint32_t epoch; float lr;
+    unsigned long long step;
+};
+
 struct Work {
     Counters* ctr;
+    StepArgs* args;
     int32_t *table_start, *tile_base, *ustart, *ctile_base;   // [T+1]
     int32_t* bag_of;       // [L] bag of every index position
     uint32_t* kidx;        // [L] unique-row index of the i-th sorted element
@@ -71,8 +80,21 @@ struct Work {
 // ---------------------------------------------------------------------------------------------
 // step prologue
 // ---------------------------------------------------------------------------------------------
-__global__ void k_prelude(Work w, const int32_t* __restrict__ offsets, int T, int B, uint32_t L) {
+__global__ void k_set_args_forward(StepArgs* a, const int32_t* indices, const int32_t* offsets, float* out, int32_t B, uint32_t L,
+                                   uint32_t epoch) {
+    a->indices = indices; a->offsets = offsets; a->out = out; a->B = B; a->L = L; a->epoch = epoch;
+}
+__global__ void k_set_args_backward(StepArgs* a, const float* grad, float lr, unsigned long long step) {
+    a->grad = grad; a->lr = lr; a->step = step;
+}
+
+template <bool IND>
+__global__ void k_prelude(Work w, int T, StepArgs av) {
+    StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
     if (threadIdx.x == 0 && blockIdx.x == 0) {
+        const int32_t* __restrict__ offsets = a.offsets;
+        const int B = a.B;
+        const uint32_t L = a.L;
         Counters* c = w.ctr;
         c->L = L; c->U = 0; c->hot_rows = 0; c->hot_tasks = 0; c->abort = 0; c->dropped = 0; c->hot_occ = 0; c->deferred = 0; c->n_heads = 0; c->upd_next = 0;
         bool bad = offsets[0] != 0 || offsets[(int64_t)T * B] != (int32_t)L;
@@ -89,9 +111,13 @@ __global__ void k_prelude(Work w, const int32_t* __restrict__ offsets, int T, in
 }
 
 // keys for the sort: the row id, or N_t for an id outside [0, N_t); eight lanes per bag, four bags per warp
+template <bool IND>
 __global__ void __launch_bounds__(256)
-k_make_keys(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets,
-            int B, uint32_t* __restrict__ keys) {
+k_make_keys(State s, Work w, uint32_t* __restrict__ keys, StepArgs av) {
+    StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
+    const int32_t* __restrict__ indices = a.indices;
+    const int32_t* __restrict__ offsets = a.offsets;
+    const int B = a.B;
     const int sub = threadIdx.x & 7;
     const int64_t nbags = (int64_t)s.T * B;
     const int64_t ng = (int64_t)gridDim.x * (blockDim.x >> 3);
@@ -206,8 +232,11 @@ __global__ void k_ustart(Work w, int T) {
 // ---------------------------------------------------------------------------------------------
 // cache tag lookup: one group of `ways` lanes per distinct row (Section 3 "Cache Structure")
 // ---------------------------------------------------------------------------------------------
+template <bool IND>
 __global__ void __launch_bounds__(256)
-k_probe(State s, Work w, uint32_t epoch) {
+k_probe(State s, Work w, StepArgs av) {
+    StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
+    const uint32_t epoch = a.epoch;
     // A warp takes 32 consecutive distinct rows: lane l works out row l's set (32 rows at a time), then the
     // warp compares the tags of 32/ways rows per round, `ways` lanes per row.
     if (w.ctr->abort) return;
@@ -261,9 +290,12 @@ k_probe(State s, Work w, uint32_t epoch) {
 }
 
 // per sorted element: where its row lives (by index position) and which sample it belongs to
+template <bool IND>
 __global__ void __launch_bounds__(256)
-k_broadcast(State s, Work w, const uint32_t* __restrict__ spos, int B) {
+k_broadcast(State s, Work w, const uint32_t* __restrict__ spos, StepArgs av) {
+    StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
     if (w.ctr->abort) return;
+    const int B = a.B;
     const int64_t L = w.ctr->L;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < L; i += (int64_t)gridDim.x * blockDim.x) {
         const uint32_t k = w.kidx[i];
@@ -287,10 +319,14 @@ __device__ __forceinline__ float4 fetch4(const State& s, const TableDev& tb, int
     return dequant4<BITS, RO>(s.codes, s.sb, tb.row_base + row, s.dim, sub);
 }
 
-template <int BITS, int LANES>
+template <int BITS, int LANES, bool IND>
 __global__ void __launch_bounds__(256)
-k_pool(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __restrict__ offsets, int B,
-       float* __restrict__ out) {
+k_pool(State s, Work w, StepArgs av) {
+    StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
+    const int32_t* __restrict__ indices = a.indices;
+    const int32_t* __restrict__ offsets = a.offsets;
+    float* __restrict__ out = a.out;
+    const int B = a.B;
     constexpr int NB = LANES < 4 ? LANES : 4;        // rows per batch; two batches are in flight
     constexpr int dim = 4 * LANES;
     const int sub = threadIdx.x & (LANES - 1);
@@ -387,9 +423,12 @@ k_pool(State s, Work w, const int32_t* __restrict__ indices, const int32_t* __re
 // ---------------------------------------------------------------------------------------------
 // backward 1: "Update PV[i]" for every i in I_U (Algorithm 2), candidate keys, hot-row tasks, counters
 // ---------------------------------------------------------------------------------------------
+template <bool IND>
 __global__ void __launch_bounds__(256)
-k_priority(State s, Work w, uint32_t step, uint32_t* __restrict__ ckey) {
+k_priority(State s, Work w, uint32_t* __restrict__ ckey, StepArgs av) {
+    StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
     if (w.ctr->abort) return;
+    const uint32_t step = (uint32_t)a.step;
     constexpr int Q = 4;                                     // independent rows per thread: the counter updates are random accesses
     const int64_t U = w.ctr->U;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -480,10 +519,12 @@ __global__ void k_policy_heads(State s, Work w, const uint32_t* __restrict__ cke
     }
 }
 
+template <bool IND>
 __global__ void __launch_bounds__(256)
-k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __restrict__ cval,
-         uint32_t step, uint32_t epoch) {
+k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __restrict__ cval, StepArgs av) {
+    StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
     if (w.ctr->abort) return;
+    const uint32_t step = (uint32_t)a.step, epoch = a.epoch;
     const int ways = s.ways;
     const int lane = threadIdx.x & 31, way = lane & (ways - 1), gbase = lane & ~(ways - 1);
     const uint32_t gmask = group_mask(ways);
@@ -635,11 +676,13 @@ __device__ __forceinline__ float4 tree_reduce(const Term& term, int64_t first, i
 
 // rows with more than HOT_SPAN occurrences: one block per HOT_SPAN occurrences computes two tree levels
 // (8 groups of LANES lanes share the 32 chunks of a task)
-template <int LANES>
+template <int LANES, bool IND>
 __global__ void __launch_bounds__(8 * LANES)
-k_hot_partial(State s, Work w, const float* __restrict__ grad, int B) {
+k_hot_partial(State s, Work w, StepArgs av) {
+    StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
     extern __shared__ float chunk_sums[];     // [32][dim]
     if (w.ctr->abort) return;
+    const float* __restrict__ grad = a.grad;
     const int dim = s.dim;
     const int sub = threadIdx.x & (LANES - 1), grp = threadIdx.x / LANES, ngrp = blockDim.x / LANES;
     const int gbase = (threadIdx.x & 31) & ~(LANES - 1);
@@ -720,11 +763,15 @@ constexpr int UPD_SMEM = UPD_WARPS * (UPD_RING * 32 * 16 + 32 * UPD_META * 4);
 // asynchronous 16-byte copies bring up to UPD_GROUPS x UPD_NB gradient rows into a shared-memory ring
 // while earlier ones are being added (in index order, radix-32 tree), independent of where one
 // embedding row ends and the next begins.
-template <int BITS, int LANES>
+template <int BITS, int LANES, bool IND>
 __global__ void __launch_bounds__(UPD_WARPS * 32, 8)
-k_update(State s, Work w, const float* __restrict__ grad, int B, float lr, uint64_t step) {
+k_update(State s, Work w, StepArgs av) {
+    StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
     extern __shared__ __align__(16) unsigned char upd_smem[];
     if (w.ctr->abort) return;
+    const float* __restrict__ grad = a.grad;
+    const float lr = a.lr;
+    const uint64_t step = a.step;
     constexpr int dim = 4 * LANES, G = 32 / LANES, NB = LANES < UPD_NB ? LANES : UPD_NB;
     enum { M_LOC, M_FLOC, M_COL, M_ROW, M_FIRST, M_CNT, M_SKIP, M_VICTIM, M_KEY, M_VKEY, M_GROW_LO, M_GROW_HI, M_VROW_LO, M_VROW_HI };
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -879,11 +926,14 @@ k_update(State s, Work w, const float* __restrict__ grad, int B, float lr, uint6
 
 // Rows named by a list: the hot rows (gradient from the partial sums of k_hot_partial), and, in a
 // second launch, the newcomers whose slot had to be vacated by a row that was itself updated.
-template <int BITS, int LANES>
+template <int BITS, int LANES, bool IND>
 __global__ void __launch_bounds__(256)
-k_update_list(State s, Work w, const float* __restrict__ grad, int B, float lr, uint64_t step,
-              const int32_t* __restrict__ list, const uint32_t* __restrict__ count, int deferred_pass) {
+k_update_list(State s, Work w, const int32_t* __restrict__ list, const uint32_t* __restrict__ count, int deferred_pass, StepArgs av) {
+    StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
     if (w.ctr->abort) return;
+    const float* __restrict__ grad = a.grad;
+    const float lr = a.lr;
+    const uint64_t step = a.step;
     constexpr int dim = 4 * LANES;
     const int lane = threadIdx.x & 31;
     const int sub = lane & (LANES - 1), gbase = lane & ~(LANES - 1);

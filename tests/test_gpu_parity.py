@@ -312,3 +312,27 @@ def test_full_size_config5_points():
     pts = list(wl.sweep5())
     for i in (5, 30, 58):
         _full_size(pts[i], [1], 3).close()
+
+
+def test_graph_replay_and_plain_launches_agree_with_the_oracle():
+    """Small steps are replayed from a captured CUDA graph; the same handle must give the oracle's results when
+    the batch shrinks and grows under one graph, when the workspace regrows, and with graphs switched off."""
+    from parity_util import make_pair, compare_state
+    cfg = _cfg(num_rows=[4000, 900], dim=32, bits=4, batch=64, bag=("poisson", 5.0), zipf=[1.1, 1.0], policy=wl.LFU, ways=4,
+               cache_fraction=0.1, seed=5)
+    h, o = make_pair(cfg)
+    rng = np.random.default_rng(0)
+    step = 0
+    for batch, graphs in ((64, True), (64, True), (16, True), (64, True), (200, True), (64, False), (32, True)):
+        cfg.batch = batch
+        h.use_graphs(graphs)
+        step += 1
+        idx, off, grad = wl.Stream(cfg, "cpu").batch(step)
+        out = torch.empty(batch, cfg.num_tables * cfg.dim, device="cuda")
+        h.forward(idx.cuda(), off.cuda(), batch, out)
+        ref = o.forward(idx.numpy(), off.numpy(), batch)
+        assert np.array_equal(out.cpu().numpy(), ref), f"step {step}"
+        h.backward(grad.cuda(), cfg.lr, step)
+        o.backward(grad.numpy(), cfg.lr, step)
+        compare_state(h, o, cfg, [0, 1], rng)
+    assert h.last_error() == (0, 0)
