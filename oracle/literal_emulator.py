@@ -116,7 +116,8 @@ class Emulator:
     """One table, one FP32 array, Algorithm 2 on top."""
 
     def __init__(self, N, d, bits, n_sets, ways, policy, optimizer="sgd", eps=1e-8, lo=-0.05, hi=0.05, seed=0,
-                 table=0):
+                 table=0, rounding="stochastic"):
+        self.rounding = rounding
         self.N, self.d, self.bits, self.n, self.alpha = N, d, bits, n_sets, ways
         self.policy, self.optimizer, self.eps, self.seed, self.table = policy, optimizer, F(eps), seed, table
         self.T = np.zeros((N, d), F)
@@ -185,7 +186,7 @@ class Emulator:
             self.T[i] = np.array([fma32(-mult, g[c], self.T[i, c]) for c in range(self.d)], F)
             key_i = rowkey(self.seed, 2, self.table, i, step)
             if self.n == 0:
-                self.T[i] = fake_quantize(self.T[i], self.bits, "stochastic", key_i)[0]
+                self.T[i] = fake_quantize(self.T[i], self.bits, self.rounding, key_i)[0]
                 continue
             if resident[i]:
                 continue
@@ -197,11 +198,11 @@ class Emulator:
             if self.alpha == 1 and self.policy == "lru":
                 bypass = False
             if bypass:
-                self.T[i] = fake_quantize(self.T[i], self.bits, "stochastic", key_i)[0]
+                self.T[i] = fake_quantize(self.T[i], self.bits, self.rounding, key_i)[0]
             else:
                 j = self.I_C[s, w_j]
                 if j >= 0:
-                    self.T[j] = fake_quantize(self.T[j], self.bits, "stochastic",
+                    self.T[j] = fake_quantize(self.T[j], self.bits, self.rounding,
                                               rowkey(self.seed, 2, self.table, int(j), step))[0]
                 self.I_C[s, w_j] = i
                 if self.policy == "lru":

@@ -122,23 +122,20 @@ void orc_dequantize(const uint8_t* q, int32_t d, float scale, float bias, float*
     for (int c = 0; c < d; ++c) x[c] = fmaf((float)q[c], scale, bias); /* q*s + b */
 }
 
+/* 8/bits codes per byte, lowest column in the lowest bits (INT4: column 2k in the low nibble of byte k) */
 void orc_pack(const uint8_t* q, int32_t d, int32_t bits, uint8_t* packed) {
-    if (bits == 8) {
-        memcpy(packed, q, (size_t)d);
-    } else { /* 4 bits: column 2k in the low nibble of byte k, column 2k+1 in the high nibble */
-        for (int k = 0; k < d / 2; ++k) packed[k] = (uint8_t)((q[2 * k] & 15) | ((q[2 * k + 1] & 15) << 4));
+    const int per = 8 / bits, mask = (1 << bits) - 1;
+    for (int k = 0; k < d / per; ++k) {
+        unsigned v = 0;
+        for (int j = 0; j < per; ++j) v |= (unsigned)(q[per * k + j] & mask) << (bits * j);
+        packed[k] = (uint8_t)v;
     }
 }
 
 void orc_unpack(const uint8_t* packed, int32_t d, int32_t bits, uint8_t* q) {
-    if (bits == 8) {
-        memcpy(q, packed, (size_t)d);
-    } else {
-        for (int k = 0; k < d / 2; ++k) {
-            q[2 * k] = packed[k] & 15;
-            q[2 * k + 1] = packed[k] >> 4;
-        }
-    }
+    const int per = 8 / bits, mask = (1 << bits) - 1;
+    for (int k = 0; k < d / per; ++k)
+        for (int j = 0; j < per; ++j) q[per * k + j] = (uint8_t)((packed[k] >> (bits * j)) & mask);
 }
 
 void orc_init_row(uint64_t seed, uint32_t table, uint32_t row, int32_t d, float lo, float hi, float* x) {
@@ -205,6 +202,7 @@ struct orc {
     int32_t* indices; int32_t* offsets; int32_t batch; int64_t total; int have_forward;
     int64_t dropped;
     int64_t last_step;
+    int32_t rounding;   /* how update() down-converts: ORC_SR (default) or ORC_RTN (Section 3 "Rounding") */
 };
 
 static uint64_t hash64(int64_t k) {
@@ -274,14 +272,14 @@ orc* orc_create(const int64_t* num_rows, int32_t num_tables, int32_t dim, int32_
                 double cache_fraction, int32_t ways, int32_t policy, int32_t optimizer,
                 float eps, float init_lo, float init_hi, uint64_t seed) {
     if (num_tables < 1 || dim < 4 || dim > 1024 || (dim & (dim - 1)) != 0) return NULL;
-    if (bits != 8 && bits != 4) return NULL;
+    if (bits != 8 && bits != 4 && bits != 2) return NULL;
     if (ways == 0) ways = 32;
     if (ways < 1 || ways > 32 || (ways & (ways - 1)) != 0) return NULL;
     if (!(cache_fraction >= 0.0 && cache_fraction <= 1.0)) return NULL;
     orc* o = (orc*)calloc(1, sizeof(orc));
     o->T = num_tables; o->d = dim; o->bits = bits; o->ways = ways; o->policy = policy;
     o->optimizer = optimizer; o->code_bytes = dim * bits / 8; o->cache_fraction = cache_fraction;
-    o->eps = eps; o->lo = init_lo; o->hi = init_hi; o->seed = seed;
+    o->eps = eps; o->lo = init_lo; o->hi = init_hi; o->seed = seed; o->rounding = ORC_SR;
     o->tb = (table_t*)calloc((size_t)num_tables, sizeof(table_t));
     for (int t = 0; t < num_tables; ++t) {
         table_t* tb = &o->tb[t];
@@ -319,6 +317,8 @@ void orc_destroy(orc* o) {
     free(o);
 }
 
+void orc_set_rounding(orc* o, int32_t mode) { o->rounding = mode == ORC_RTN ? ORC_RTN : ORC_SR; }
+
 void orc_set_table_mask(orc* o, const uint8_t* table_mask) {
     free(o->mask);
     o->mask = NULL;
@@ -352,13 +352,13 @@ static void fetch(orc* o, int32_t t, int64_t row, float* x) {
     orc_dequantize(q, o->d, tb->scale[id], tb->bias[id], x);
 }
 
-/* down-convert x into T[row] with stochastic rounding */
+/* down-convert x into T[row] with the rounding method of choice (stochastic unless set otherwise) */
 static void store_quantized(orc* o, int32_t t, int64_t row, const float* x, uint32_t domain, int64_t step) {
     table_t* tb = &o->tb[t];
     int64_t id = rec_get(o, t, row);
     uint8_t q[1024];
     uint32_t key = orc_rowkey(o->seed, domain, (uint32_t)t, (uint32_t)row, (uint64_t)step);
-    orc_quantize(x, o->d, o->bits, ORC_SR, key, q, &tb->scale[id], &tb->bias[id]);
+    orc_quantize(x, o->d, o->bits, o->rounding, key, q, &tb->scale[id], &tb->bias[id]);
     orc_pack(q, o->d, o->bits, tb->codes + id * o->code_bytes);
 }
 

@@ -60,6 +60,8 @@ void orc_destroy(orc* o);
 /* only tables with table_mask[t] != 0 are processed (NULL = all); lets a test
  * run a sample of the tables of a large configuration */
 void orc_set_table_mask(orc* o, const uint8_t* table_mask);
+/* rounding used when a row is down-converted during training and flush: ORC_SR (default) or ORC_RTN */
+void orc_set_rounding(orc* o, int32_t mode);
 int  orc_forward(orc* o, const int32_t* indices, const int32_t* offsets, int32_t batch,
                  int64_t total_indices, float* out);
 int  orc_backward(orc* o, const float* grad_out, float lr, int64_t step);

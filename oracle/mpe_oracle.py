@@ -52,6 +52,7 @@ _create = _sig("orc_create", C.c_void_p, _i64p, C.c_int32, C.c_int32, C.c_int32,
                C.c_int32, C.c_int32, C.c_float, C.c_float, C.c_float, C.c_uint64)
 _destroy = _sig("orc_destroy", None, C.c_void_p)
 _set_mask = _sig("orc_set_table_mask", None, C.c_void_p, C.c_void_p)
+_set_rounding = _sig("orc_set_rounding", None, C.c_void_p, C.c_int32)
 _forward = _sig("orc_forward", C.c_int, C.c_void_p, _i32p, _i32p, C.c_int32, C.c_int64, _f32p)
 _backward = _sig("orc_backward", C.c_int, C.c_void_p, _f32p, C.c_float, C.c_int64)
 _flush = _sig("orc_flush", C.c_int, C.c_void_p)
@@ -163,6 +164,9 @@ class Oracle:
 
     def __del__(self):
         self.close()
+
+    def set_rounding(self, mode):
+        _set_rounding(self._h, mode)
 
     def set_table_mask(self, mask):
         if mask is None:

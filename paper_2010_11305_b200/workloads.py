@@ -63,7 +63,7 @@ def _cfg2_rows(seed=0, lo=3, hi=10_000_000, n=26, target=33_000_000, tol=0.05):
 
 
 def config(i: int) -> Config:
-    """The five benchmark configurations (1-based, as listed in the baseline description)."""
+    """The five benchmark configurations (1-based)."""
     if i == 1:
         return Config("cfg1", [10_000], 16, 8, 0.05, 8, LRU, SGD, 0.01, 128, ("fixed", 4), [1.05], 10, seed=0)
     if i == 2:

@@ -75,7 +75,7 @@ def test_num_sets_follows_the_budget():
 
 
 # ----------------------------------------------------------- quantizer ---
-@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("bits", [8, 4, 2])
 @pytest.mark.parametrize("d", [4, 16, 64, 128])
 def test_quantizer_closed_forms(bits, d):
     rng = np.random.default_rng(bits * 100 + d)
@@ -132,9 +132,13 @@ def test_int4_packing_low_nibble_first():
     assert list(p) == [0x10, 0x32, 0x54, 0x76, 0x98, 0xBA, 0xDC, 0xFE]
     assert np.array_equal(orc.unpack(p, 16, 4), q)
     assert np.array_equal(orc.pack(q, 8), q)
+    q2 = np.array([0, 1, 2, 3, 3, 2, 1, 0], np.uint8)          # INT2: four codes per byte, lowest column in the lowest bits
+    p2 = orc.pack(q2, 2)
+    assert list(p2) == [0b11100100, 0b00011011]
+    assert np.array_equal(orc.unpack(p2, 8, 2), q2)
 
 
-@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("bits", [8, 4, 2])
 def test_stochastic_rounding_is_unbiased_and_nearest_is_not(bits):
     rng = np.random.default_rng(5)
     d, K = 16, 100_000
@@ -323,14 +327,19 @@ def test_full_cache_equals_fp32_embedding_bag_training(policy, opt):
 @pytest.mark.parametrize("bits,ways,policy,opt,frac", [
     (8, 2, "lru", "sgd", 0.25), (4, 4, "lfu", "sgd", 0.25), (8, 4, "lfu", "adagrad", 0.25),
     (4, 2, "lru", "adagrad", 0.25), (8, 1, "lru", "sgd", 0.1), (8, 1, "lfu", "sgd", 0.1),
-    (8, 2, "lru", "sgd", 0.0), (4, 2, "lfu", "sgd", 0.0),
+    (8, 2, "lru", "sgd", 0.0), (4, 2, "lfu", "sgd", 0.0), (2, 4, "lfu", "sgd", 0.25), (2, 2, "lru", "adagrad", 0.0),
+    (-8, 2, "lru", "sgd", 0.25), (-4, 4, "lfu", "sgd", 0.0),      # negative width: round to nearest while training
 ])
 def test_two_space_oracle_equals_single_array_emulation(bits, ways, policy, opt, frac):
+    nearest = bits < 0
+    bits = abs(bits)
     N, d, B, lr, seed = 24, 8, 6, 0.05, 21
     pol = orc.LRU if policy == "lru" else orc.LFU
     op = orc.SGD if opt == "sgd" else orc.ROWWISE_ADAGRAD
     o = orc.Oracle([N], d, bits, frac, ways, pol, optimizer=op, seed=seed)
-    e = emu.Emulator(N, d, bits, o.sets(0), ways, policy, optimizer=opt, seed=seed)
+    e = emu.Emulator(N, d, bits, o.sets(0), ways, policy, optimizer=opt, seed=seed, rounding="nearest" if nearest else "stochastic")
+    if nearest:
+        o.set_rounding(orc.RTN)
     rng = np.random.default_rng(bits * 7 + ways)
     for r in range(N):
         assert np.array_equal(o.fetch_value(0, r), e.T[r])
@@ -365,17 +374,13 @@ def test_memory_compression_factors_of_the_appendix():
     checked = 0
     for bits, ratio, factor in rows:
         bits, ratio, factor = int(bits), float(ratio), float(factor)
-        if bits == 2:
-            # INT2 is outside the build (INT8/INT4 only): check the formula's arithmetic directly
-            got = (2 * D + 64 + (32 if ratio > 0 else 0) + 32 * ratio + 32 * D * ratio) / (32 * D)
-        else:
-            o = orc.Oracle([N], D, bits, ratio, 32, orc.LFU)
-            m = o.memory_bytes().astype(np.float64)
-            got = (m[0] + m[1] + m[2] + m[3]) / m[5]
-            o.close()
-            checked += 1
+        o = orc.Oracle([N], D, bits, ratio, 32, orc.LFU)
+        m = o.memory_bytes().astype(np.float64)
+        got = (m[0] + m[1] + m[2] + m[3]) / m[5]
+        o.close()
+        checked += 1
         assert abs(got - factor) < 6e-6, (bits, ratio, got, factor)
-    assert checked == 7
+    assert checked == 10
 
 
 def test_table1_sizes_fixture():
@@ -462,3 +467,29 @@ def test_hit_rates_behave_like_the_paper_says():
     assert lfu32 > 0.8 * ideal
     assert lfu32 >= lfu1 >= lru1 - 0.01                 # ordering of the paper's hit-rate table
     assert hit_rate(32, orc.LFU, 1.05, frac=0.2) > lfu32  # larger cache, higher hit rate
+
+
+def test_nearest_rounding_in_training_loses_small_updates_and_stochastic_does_not():
+    """Section 3 "Rounding" and the no-cache accuracy table: with round-to-nearest an update smaller than half a
+    quantization step is lost every time, with stochastic rounding it survives on average."""
+    d, N = 8, 4
+    res = {}
+    for mode in (orc.RTN, orc.SR):
+        o = orc.Oracle([N], d, 8, 0.0, 8, orc.LRU, seed=2)
+        o.set_rounding(mode)
+        x0 = o.fetch_value(0, 1).astype(np.float64)
+        step_size = float(o.row(0, 1)[1])
+        # each update moves the interior columns by a fifth of a quantization step; the columns holding the row's
+        # minimum and maximum stay put, so scale and bias do not follow the update
+        x0f = x0.astype(F)
+        inner = np.ones(d, bool)
+        inner[[int(np.argmin(x0f)), int(np.argmax(x0f))]] = False
+        g = np.zeros((1, d), F)
+        g[0, inner] = 0.2 * step_size
+        idx, off, B = _bags_to_arrays([[[1]]])
+        for step in range(1, 101):
+            o.forward(idx, off, B)
+            o.backward(g, 1.0, step)
+        res[mode] = ((x0 - o.fetch_value(0, 1).astype(np.float64)) / step_size)[inner]
+    assert np.all(np.abs(res[orc.RTN]) < 1.0)             # nothing accumulated: 100 updates of 0.2 steps all rounded away
+    assert np.all(res[orc.SR] > 8.0)                      # expectation 20 quantization steps (until a column reaches the minimum)
