@@ -30,11 +30,12 @@ typedef struct { int64_t num_rows; int32_t dim; } mpe_table_spec;
 
 enum { MPE_LRU = 0, MPE_LFU = 1 };
 enum { MPE_SGD = 0, MPE_ROWWISE_ADAGRAD = 1 };
+enum { MPE_ROUND_NEAREST = 0, MPE_ROUND_STOCHASTIC = 1 };
 
 enum {
     MPE_OK = 0,
     MPE_ERR_ARG = -1,          /* NULL pointer, negative size, value out of range */
-    MPE_ERR_UNSUPPORTED = -2,  /* unequal dims, dim not a power of two in [4,128], bits not 8/4, ways not 2^k <= 32 */
+    MPE_ERR_UNSUPPORTED = -2,  /* unequal dims, dim not a power of two in [4,128], bits not 8/4/2, ways not 2^k <= 32 */
     MPE_ERR_CUDA = -3,         /* a CUDA runtime call failed (detail = cudaError_t) */
     MPE_ERR_SEQUENCE = -4,     /* backward without a preceding forward, or step not strictly increasing */
     MPE_ERR_INDEX = -5,        /* device saw row ids outside [0, num_rows) (detail = how many); they were dropped */
@@ -47,7 +48,7 @@ enum {
  * Create the tables, the caches and the policy state on `device`.
  *   tables[num_tables]  row count and dimension of each table; all dims must be equal
  *                       (a power of two in [4,128]); num_rows in [1, 2^31-2].
- *   bits                8 or 4: width of the integer codes (Section 3 "Precision").
+ *   bits                8, 4 or 2: width of the integer codes, ranges [0,255], [0,15], [0,3] (Section 3 "Precision").
  *   cache_fraction      in [0,1]; table t gets n_t = max(1, floor(cache_fraction*N_t + 1e-6) / ways) sets
  *                       of `ways` FP32 rows (Section 3 "Cache Structure"); 0 = no cache at all.
  *   ways                associativity alpha, a power of two <= 32; 0 selects 32 (Section 5.1).
@@ -100,6 +101,12 @@ int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offset
  * the same way.  Must follow exactly one mpe_forward (else MPE_ERR_SEQUENCE).  Returns without waiting.
  */
 int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step);
+
+/* How update() down-converts a row into the low-precision table (Section 3 "Rounding"): MPE_ROUND_STOCHASTIC
+ * (the default: one of the two neighbouring codes, with expectation equal to the value) or MPE_ROUND_NEAREST
+ * (the closer code, ties to even).  Applies to mpe_backward and mpe_flush from the next call on; not allowed between
+ * a forward and its backward (MPE_ERR_SEQUENCE).  Waits for the handle's stream. */
+int mpe_set_rounding(mpe_handle* h, int32_t mode);
 
 /* One whole step from HOST buffers: copies indices, offsets and grad_out to the device, runs
  * forward and backward, copies the pooled output back and waits for it.  Layouts as above.

@@ -16,11 +16,12 @@ LIB_PATH = os.path.join(_HERE, "libmpe.so")
 
 LRU, LFU = 0, 1
 SGD, ROWWISE_ADAGRAD = 0, 1
+ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
 OK, ERR_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_SEQUENCE, ERR_INDEX, ERR_OFFSETS, ERR_NOMEM, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6, -7, -8
 STATIC_MAX_INDICES, STATIC_MAX_BAGS, STATIC_MAX_TABLES = 32768, 32768, 64
 
 EXPORTS = [
-    "mpe_create", "mpe_reserve", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_step_host", "mpe_flush", "mpe_destroy",
+    "mpe_create", "mpe_reserve", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_set_rounding", "mpe_step_host", "mpe_flush", "mpe_destroy",
     "mpe_last_error", "mpe_stats", "mpe_memory_bytes", "mpe_cache_geometry", "mpe_step_info", "mpe_export_rows",
     "mpe_export_cache", "mpe_export_aux", "mpe_use_graphs", "mpe_kernel_launches", "mpe_profile", "mpe_profile_read", "mpe_error_string",
 ]
@@ -56,6 +57,7 @@ _lib.mpe_export_rows.argtypes = [_vp, _i32, _vp, _i64, _vp, _vp, _vp]
 _lib.mpe_export_cache.argtypes = [_vp, _i32, _vp, _vp, _vp]
 _lib.mpe_export_aux.argtypes = [_vp, _i32, _vp, _i64, _vp, _vp]
 _lib.mpe_use_graphs.argtypes = [_vp, _i32]
+_lib.mpe_set_rounding.argtypes = [_vp, _i32]
 _lib.mpe_kernel_launches.argtypes = [_vp, C.POINTER(_u64)]
 _lib.mpe_profile.argtypes = [_vp, _i32]
 _lib.mpe_profile_read.argtypes = [_vp, _i32, _vp, _vp, _vp, C.POINTER(_i32)]
@@ -185,6 +187,9 @@ class Mpe:
         G = np.zeros(max(rows.size, 1), np.float32)
         _check(_lib.mpe_export_aux(self._h, table, rows.ctypes.data, rows.size, cnt.ctypes.data, G.ctypes.data), "mpe_export_aux")
         return cnt[:rows.size], G[:rows.size]
+
+    def set_rounding(self, mode):
+        _check(_lib.mpe_set_rounding(self._h, mode), "mpe_set_rounding")
 
     def use_graphs(self, enable):
         _check(_lib.mpe_use_graphs(self._h, 1 if enable else 0), "mpe_use_graphs")

@@ -206,7 +206,8 @@ void dispatch(int bits, int lanes, F&& f) {
         }
     };
     if (bits == 8) by_lanes(std::integral_constant<int, 8>{});
-    else by_lanes(std::integral_constant<int, 4>{});
+    else if (bits == 4) by_lanes(std::integral_constant<int, 4>{});
+    else by_lanes(std::integral_constant<int, 2>{});
 }
 
 int check_launch(mpe_handle* h) {
@@ -242,7 +243,7 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
     if (!(cache_fraction >= 0.0 && cache_fraction <= 1.0)) return MPE_ERR_ARG;
     if (policy != MPE_LRU && policy != MPE_LFU) return MPE_ERR_ARG;
     if (optimizer != MPE_SGD && optimizer != MPE_ROWWISE_ADAGRAD) return MPE_ERR_ARG;
-    if (bits != 8 && bits != 4) return MPE_ERR_UNSUPPORTED;
+    if (bits != 8 && bits != 4 && bits != 2) return MPE_ERR_UNSUPPORTED;
     if (ways == 0) ways = 32;
     if (ways < 1 || ways > 32 || (ways & (ways - 1))) return MPE_ERR_UNSUPPORTED;
     const int dim = tables[0].dim;
@@ -292,7 +293,7 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
 
     State& s = h->st;
     s.T = num_tables; s.dim = dim; s.lanes = dim / 4; s.ways = ways; s.policy = policy; s.optimizer = optimizer;
-    s.bits = bits; s.seed = seed; s.eps = eps;
+    s.bits = bits; s.seed = seed; s.eps = eps; s.rounding = 1;
     int rc = MPE_OK;
     auto fail = [&](int code) { mpe_destroy(h); return code; };
     if ((rc = dmalloc(h, &h->d_tables, num_tables, nullptr)) != MPE_OK) return fail(rc);
@@ -319,7 +320,8 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
     for (int t = 0; t < num_tables; ++t) {
         const int g = grid_for(h, h->tables[t].N, 256 / s.lanes, 8);
         if (bits == 8) LAUNCH(h, "init_table", k_init_table<8>, g, 256, 0, s, t, init_lo, init_hi);
-        else LAUNCH(h, "init_table", k_init_table<4>, g, 256, 0, s, t, init_lo, init_hi);
+        else if (bits == 4) LAUNCH(h, "init_table", k_init_table<4>, g, 256, 0, s, t, init_lo, init_hi);
+        else LAUNCH(h, "init_table", k_init_table<2>, g, 256, 0, s, t, init_lo, init_hi);
     }
     CKC(cudaGetLastError());
     CKC(cudaDeviceSynchronize());
@@ -552,6 +554,16 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
     return MPE_OK;
 }
 
+int mpe_set_rounding(mpe_handle* h, int32_t mode) {
+    if (!h || (mode != MPE_ROUND_NEAREST && mode != MPE_ROUND_STOCHASTIC)) return MPE_ERR_ARG;
+    if (h->have_forward) return MPE_ERR_SEQUENCE;
+    DeviceGuard guard(h->device);
+    CK(h, cudaStreamSynchronize(h->stream));
+    h->st.rounding = mode;
+    drop_graphs(h);           // the captured kernels carry the old setting
+    return MPE_OK;
+}
+
 int mpe_use_graphs(mpe_handle* h, int32_t enable) {
     if (!h) return MPE_ERR_ARG;
     h->graphs_enabled = enable != 0;
@@ -609,7 +621,8 @@ int mpe_flush(mpe_handle* h) {
         if (nslot == 0) continue;
         const int g = grid_for(h, nslot, 256 / s.lanes, 8);
         if (h->bits == 8) LAUNCH(h, "flush", k_flush<8>, g, 256, 0, s, t, (uint64_t)h->last_step);
-        else LAUNCH(h, "flush", k_flush<4>, g, 256, 0, s, t, (uint64_t)h->last_step);
+        else if (h->bits == 4) LAUNCH(h, "flush", k_flush<4>, g, 256, 0, s, t, (uint64_t)h->last_step);
+        else LAUNCH(h, "flush", k_flush<2>, g, 256, 0, s, t, (uint64_t)h->last_step);
     }
     return check_launch(h);
 }

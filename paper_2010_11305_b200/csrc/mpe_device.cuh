@@ -47,51 +47,52 @@ __device__ __forceinline__ uint32_t group_mask(int lanes_per_row) {
     return lanes_per_row == 32 ? 0xffffffffU : (((1U << lanes_per_row) - 1U) << (lane & ~(lanes_per_row - 1)));
 }
 
-// four codes (packed in q, lowest column in the lowest bits) -> q*scale + bias (Algorithm 1, up-conversion)
+// The four codes of one lane (columns 4*sub .. 4*sub+3) are BITS*4 adjacent bits of the row: one u32 (INT8),
+// one u16 (INT4) or one byte (INT2); the lowest column sits in the lowest bits.
+template <int BITS, bool RO>
+__device__ __forceinline__ uint32_t load_codes4(const uint8_t* codes, int64_t grow, int dim, int sub) {
+    const uint8_t* row = codes + grow * (dim * BITS / 8);
+    if (BITS == 8) return RO ? __ldg(reinterpret_cast<const uint32_t*>(row) + sub) : reinterpret_cast<const uint32_t*>(row)[sub];
+    if (BITS == 4) return RO ? __ldg(reinterpret_cast<const uint16_t*>(row) + sub) : reinterpret_cast<const uint16_t*>(row)[sub];
+    return RO ? __ldg(row + sub) : row[sub];
+}
+template <int BITS>
+__device__ __forceinline__ void store_codes4(uint8_t* codes, int64_t grow, int dim, int sub, uint32_t q0, uint32_t q1, uint32_t q2, uint32_t q3) {
+    uint8_t* row = codes + grow * (dim * BITS / 8);
+    const uint32_t q = q0 | (q1 << BITS) | (q2 << (2 * BITS)) | (q3 << (3 * BITS));
+    if (BITS == 8) reinterpret_cast<uint32_t*>(row)[sub] = q;
+    else if (BITS == 4) reinterpret_cast<uint16_t*>(row)[sub] = (uint16_t)q;
+    else row[sub] = (uint8_t)q;
+}
+
+// four packed codes -> q*scale + bias (Algorithm 1, up-conversion)
 template <int BITS>
 __device__ __forceinline__ float4 decode4(uint32_t q, float2 p) {
+    constexpr uint32_t M = (1u << BITS) - 1u;
     float4 x;
-    if (BITS == 8) {
-        x.x = __fmaf_rn(__uint2float_rn(q & 255u), p.x, p.y);
-        x.y = __fmaf_rn(__uint2float_rn((q >> 8) & 255u), p.x, p.y);
-        x.z = __fmaf_rn(__uint2float_rn((q >> 16) & 255u), p.x, p.y);
-        x.w = __fmaf_rn(__uint2float_rn(q >> 24), p.x, p.y);
-    } else {
-        x.x = __fmaf_rn(__uint2float_rn(q & 15u), p.x, p.y);
-        x.y = __fmaf_rn(__uint2float_rn((q >> 4) & 15u), p.x, p.y);
-        x.z = __fmaf_rn(__uint2float_rn((q >> 8) & 15u), p.x, p.y);
-        x.w = __fmaf_rn(__uint2float_rn((q >> 12) & 15u), p.x, p.y);
-    }
+    x.x = __fmaf_rn(__uint2float_rn(q & M), p.x, p.y);
+    x.y = __fmaf_rn(__uint2float_rn((q >> BITS) & M), p.x, p.y);
+    x.z = __fmaf_rn(__uint2float_rn((q >> (2 * BITS)) & M), p.x, p.y);
+    x.w = __fmaf_rn(__uint2float_rn((q >> (3 * BITS)) & M), p.x, p.y);
     return x;
 }
 
 // RO = the table is not written by the running kernel, so the read-only data path may serve the loads
 template <int BITS, bool RO>
 __device__ __forceinline__ float4 dequant4(const uint8_t* codes, const float2* sb, int64_t grow, int dim, int sub) {
-    // up-conversion q*s + b (Algorithm 1, last line of the loop)
-    float2 p;
-    uint32_t q;
-    if (RO) {
-        p = __ldg(sb + grow);
-        if (BITS == 8) q = __ldg(reinterpret_cast<const uint32_t*>(codes + grow * dim) + sub);
-        else           q = __ldg(reinterpret_cast<const uint16_t*>(codes + grow * (dim >> 1)) + sub);
-    } else {
-        p = sb[grow];
-        if (BITS == 8) q = reinterpret_cast<const uint32_t*>(codes + grow * dim)[sub];
-        else           q = reinterpret_cast<const uint16_t*>(codes + grow * (dim >> 1))[sub];
-    }
-    return decode4<BITS>(q, p);
+    const float2 p = RO ? __ldg(sb + grow) : sb[grow];
+    return decode4<BITS>(load_codes4<BITS, RO>(codes, grow, dim, sub), p);
 }
 
 __device__ __forceinline__ float4 add4(float4 a, float4 b) {
     return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
 }
 
-template <int BITS, bool STOCHASTIC>
-__device__ __forceinline__ uint32_t quant1(float x, float mn, float inv, float qmax, uint32_t key, uint32_t column) {
+// one value -> its code; `stochastic` picks the rounding of Section 3 "Rounding" (it is the same for a whole kernel)
+__device__ __forceinline__ uint32_t quant1(float x, float mn, float inv, float qmax, uint32_t key, uint32_t column, bool stochastic) {
     float y = __fmul_rn(__fsub_rn(x, mn), inv);           // (x - b)/s as (x - b) * (1/s)
     y = fminf(fmaxf(y, 0.0f), qmax);
-    if (STOCHASTIC) {
+    if (stochastic) {
         const float f = floorf(y);
         const float p = __fsub_rn(y, f);                   // exact
         const float u = uniform01(key, column);
@@ -101,9 +102,9 @@ __device__ __forceinline__ uint32_t quant1(float x, float mn, float inv, float q
 }
 
 // Down-convert one FP32 row (four columns per lane) into the low-precision table.
-template <int BITS, bool STOCHASTIC>
+template <int BITS>
 __device__ __forceinline__ void quantize_store(float4 x, uint8_t* __restrict__ codes, float2* __restrict__ sb,
-                                               int64_t grow, int dim, int sub, int lanes_per_row, uint32_t key) {
+                                               int64_t grow, int dim, int sub, int lanes_per_row, uint32_t key, bool stochastic) {
     const uint32_t mask = group_mask(lanes_per_row);
     float mn = fminf(fminf(x.x, x.y), fminf(x.z, x.w));
     float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
@@ -118,12 +119,11 @@ __device__ __forceinline__ void quantize_store(float4 x, uint8_t* __restrict__ c
     if (s >= 1.17549435e-38f) inv = __fdiv_rn(1.0f, s);
     if (inv == 0.0f) s = 0.0f;
     const uint32_t c = 4u * (uint32_t)sub;
-    const uint32_t q0 = quant1<BITS, STOCHASTIC>(x.x, mn, inv, qmax, key, c);
-    const uint32_t q1 = quant1<BITS, STOCHASTIC>(x.y, mn, inv, qmax, key, c + 1);
-    const uint32_t q2 = quant1<BITS, STOCHASTIC>(x.z, mn, inv, qmax, key, c + 2);
-    const uint32_t q3 = quant1<BITS, STOCHASTIC>(x.w, mn, inv, qmax, key, c + 3);
-    if (BITS == 8) reinterpret_cast<uint32_t*>(codes + grow * dim)[sub] = q0 | (q1 << 8) | (q2 << 16) | (q3 << 24);
-    else reinterpret_cast<uint16_t*>(codes + grow * (dim >> 1))[sub] = (uint16_t)(q0 | (q1 << 4) | (q2 << 8) | (q3 << 12));
+    const uint32_t q0 = quant1(x.x, mn, inv, qmax, key, c, stochastic);
+    const uint32_t q1 = quant1(x.y, mn, inv, qmax, key, c + 1, stochastic);
+    const uint32_t q2 = quant1(x.z, mn, inv, qmax, key, c + 2, stochastic);
+    const uint32_t q3 = quant1(x.w, mn, inv, qmax, key, c + 3, stochastic);
+    store_codes4<BITS>(codes, grow, dim, sub, q0, q1, q2, q3);
     if (sub == 0) sb[grow] = make_float2(s, mn);
 }
 

@@ -38,6 +38,7 @@ struct Counters {
 
 struct State {
     int T, dim, lanes, ways, policy, optimizer, bits;
+    int rounding;          // how rows are down-converted while training: 1 stochastic (default), 0 nearest-even
     uint64_t seed;
     float eps;
     const TableDev* tables;
@@ -736,12 +737,12 @@ __device__ __forceinline__ void apply_update(const State& s, const TableDev& tb,
     if (floc >= 0) {
         float4* dst = reinterpret_cast<float4*>(s.slab + (int64_t)floc * dim) + sub;
         if (loc < 0 && victim >= 0)     // the row this newcomer displaces is down-converted and placed back in T
-            quantize_store<BITS, true>(*dst, s.codes, s.sb, tb.row_base + victim, dim, sub, LANES,
-                                       rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)victim, step));
+            quantize_store<BITS>(*dst, s.codes, s.sb, tb.row_base + victim, dim, sub, LANES,
+                                rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)victim, step), s.rounding != 0);
         *dst = xn;                      // cached rows keep full precision, a newcomer enters verbatim
     } else {
-        quantize_store<BITS, true>(xn, s.codes, s.sb, grow, dim, sub, LANES,
-                                   rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)row, step));
+        quantize_store<BITS>(xn, s.codes, s.sb, grow, dim, sub, LANES,
+                            rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)row, step), s.rounding != 0);
     }
 }
 
@@ -849,8 +850,7 @@ k_update(State s, Work w, StepArgs av) {
             } else {
                 const int64_t grow = ((int64_t)meta[cr][M_GROW_HI] << 32) | (uint32_t)meta[cr][M_GROW_LO];
                 xr.sb = s.sb[grow];
-                if (BITS == 8) xr.q = reinterpret_cast<const uint32_t*>(s.codes + grow * dim)[sub];
-                else           xr.q = reinterpret_cast<const uint16_t*>(s.codes + grow * (dim >> 1))[sub];
+                xr.q = load_codes4<BITS, false>(s.codes, grow, dim, sub);
             }
         };
         if (cr < nrow) load_x();
@@ -911,11 +911,11 @@ k_update(State s, Work w, StepArgs av) {
                     float4* dst = reinterpret_cast<float4*>(s.slab + (int64_t)floc * dim) + sub;
                     if (loc < 0 && mc[M_VICTIM] >= 0) {  // the row this newcomer displaces is down-converted and placed back in T
                         const int64_t vrow = ((int64_t)mc[M_VROW_HI] << 32) | (uint32_t)mc[M_VROW_LO];
-                        quantize_store<BITS, true>(*dst, s.codes, s.sb, vrow, dim, sub, LANES, (uint32_t)mc[M_VKEY]);
+                        quantize_store<BITS>(*dst, s.codes, s.sb, vrow, dim, sub, LANES, (uint32_t)mc[M_VKEY], s.rounding != 0);
                     }
                     *dst = xn;                           // cached rows keep full precision, a newcomer enters verbatim
                 } else {
-                    quantize_store<BITS, true>(xn, s.codes, s.sb, grow, dim, sub, LANES, (uint32_t)mc[M_KEY]);
+                    quantize_store<BITS>(xn, s.codes, s.sb, grow, dim, sub, LANES, (uint32_t)mc[M_KEY], s.rounding != 0);
                 }
                 cr = valid_from(cr + G); co = 0;
                 if (cr < nrow) load_x();
@@ -985,7 +985,7 @@ __global__ void k_init_table(State s, int t, float lo, float hi) {
         x.y = __fmaf_rn(uniform01(key, 4 * sub + 1), width, lo);
         x.z = __fmaf_rn(uniform01(key, 4 * sub + 2), width, lo);
         x.w = __fmaf_rn(uniform01(key, 4 * sub + 3), width, lo);
-        quantize_store<BITS, false>(x, s.codes, s.sb, tb.row_base + row, s.dim, sub, lanes, 0u);
+        quantize_store<BITS>(x, s.codes, s.sb, tb.row_base + row, s.dim, sub, lanes, 0u, false);
     }
 }
 
@@ -1001,8 +1001,8 @@ __global__ void k_flush(State s, int t, uint64_t step) {
         const int32_t tag = s.tags[slot];
         if (tag < 0) continue;
         const float4 x = reinterpret_cast<const float4*>(s.slab + slot * s.dim)[sub];
-        quantize_store<BITS, true>(x, s.codes, s.sb, tb.row_base + tag, s.dim, sub, lanes,
-                                   rowkey(s.seed, DOMAIN_FLUSH, (uint32_t)t, (uint32_t)tag, step));
+        quantize_store<BITS>(x, s.codes, s.sb, tb.row_base + tag, s.dim, sub, lanes,
+                             rowkey(s.seed, DOMAIN_FLUSH, (uint32_t)t, (uint32_t)tag, step), s.rounding != 0);
     }
 }
 

@@ -41,7 +41,8 @@ def test_config2_lfu_many_tables():
 @pytest.mark.parametrize("bits,policy,opt,ways,dim", [
     (8, wl.LRU, wl.SGD, 8, 16), (4, wl.LRU, wl.ROWWISE_ADAGRAD, 16, 64), (4, wl.LFU, wl.SGD, 32, 128),
     (8, wl.LFU, wl.ROWWISE_ADAGRAD, 32, 64), (4, wl.LFU, wl.SGD, 2, 32), (8, wl.LRU, wl.SGD, 1, 8),
-    (4, wl.LFU, wl.SGD, 1, 4), (8, wl.LRU, wl.SGD, 4, 128),
+    (4, wl.LFU, wl.SGD, 1, 4), (8, wl.LRU, wl.SGD, 4, 128), (2, wl.LFU, wl.SGD, 32, 128), (2, wl.LRU, wl.ROWWISE_ADAGRAD, 8, 16),
+    (2, wl.LFU, wl.SGD, 2, 4),
 ])
 def test_small_tables_every_variant(bits, policy, opt, ways, dim):
     """Small tables with a skewed stream: many hits, admissions, evictions, bypasses and chains per step."""
@@ -336,3 +337,38 @@ def test_graph_replay_and_plain_launches_agree_with_the_oracle():
         o.backward(grad.numpy(), cfg.lr, step)
         compare_state(h, o, cfg, [0, 1], rng)
     assert h.last_error() == (0, 0)
+
+
+@pytest.mark.parametrize("bits", [8, 4, 2])
+def test_round_to_nearest_while_training(bits):
+    """Section 3 "Rounding": the nearest-even option instead of stochastic rounding, for updates, evictions and flush."""
+    from parity_util import make_pair, compare_state
+    from paper_2010_11305_b200 import binding as mpe
+    cfg = _cfg(num_rows=[2500, 300], dim=32, bits=bits, batch=80, bag=("poisson", 5.0), zipf=[1.1, 0.9], policy=wl.LFU, ways=4,
+               cache_fraction=0.1, seed=9 + bits)
+    h, o = make_pair(cfg)
+    rng = np.random.default_rng(0)
+    st = wl.Stream(cfg, "cpu")
+    for step in range(1, 7):
+        if step == 1:
+            h.set_rounding(mpe.ROUND_NEAREST)
+            o.set_rounding(0)
+        if step == 5:                                   # and back, on the same handle
+            h.set_rounding(mpe.ROUND_STOCHASTIC)
+            o.set_rounding(1)
+        idx, off, grad = st.batch(step)
+        out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, device="cuda")
+        h.forward(idx.cuda(), off.cuda(), cfg.batch, out)
+        ref = o.forward(idx.numpy(), off.numpy(), cfg.batch)
+        assert np.array_equal(out.cpu().numpy(), ref)
+        if step == 3:
+            with pytest.raises(mpe.MpeError) as e:      # not between a forward and its backward
+                h.set_rounding(mpe.ROUND_STOCHASTIC)
+            assert e.value.code == mpe.ERR_SEQUENCE
+        h.backward(grad.cuda(), cfg.lr, step)
+        o.backward(grad.numpy(), cfg.lr, step)
+        compare_state(h, o, cfg, [0, 1], rng)
+        if step in (4, 6):
+            h.flush()
+            o.flush()
+            compare_state(h, o, cfg, [0, 1], rng)

@@ -37,7 +37,7 @@ def _batch(cfg, step, drop=0):
     return idx, off, cfg.batch
 
 
-@pytest.mark.parametrize("bits,dim,policy", [(4, 128, wl.LFU), (8, 16, wl.LRU)])
+@pytest.mark.parametrize("bits,dim,policy", [(4, 128, wl.LFU), (8, 16, wl.LRU), (2, 64, wl.LFU)])
 def test_static_forward_matches_forward_on_two_calls_in_a_row(bits, dim, policy):
     if not torch.cuda.is_available():
         pytest.fail("needs a CUDA device")
