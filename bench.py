@@ -329,6 +329,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep5", action="store_true", help="run every point of the policy/skew sweep (configuration 5): one JSON line per point")
+    ap.add_argument("--sweep-assoc", action="store_true", help="associativity sweep (1..32 ways, LRU and LFU) on configuration 5's shape")
     ap.add_argument("--tables", type=int, default=None, help="profiling aid: keep only the first TABLES tables")
     ap.add_argument("--rows-div", type=int, default=1, help="profiling aid: divide every table's row count")
     ap.add_argument("--batch-div", type=int, default=1, help="profiling aid: divide the batch size")
@@ -362,6 +363,21 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if args.sweep_assoc:
+        # hit rate per (ways, policy, cache size) on a Zipf(1.05) stream: the layout of the paper's hit-rate table
+        from dataclasses import replace
+        args.e2e_steps = 0
+        args.warmup = max(args.warmup, 50)
+        for frac in (0.05, 0.10, 0.30, 0.50):
+            for policy in (wl.LRU, wl.LFU):
+                for ways in (1, 2, 4, 8, 16, 32):
+                    point = replace(wl.config(5), name=f"c{frac:g}-{'lru' if policy == wl.LRU else 'lfu'}-{ways}way", ways=ways,
+                                    policy=policy, cache_fraction=frac)
+                    r = run_ours(args, point, 0, 1, local_rank)
+                    print(json.dumps({"point": point.name, "cache_fraction": frac, "policy": "lru" if policy == wl.LRU else "lfu",
+                                      "ways": ways, "index_hit_rate": r["per_step"]["index_hit_rate"], "ms_per_step": r["ms_per_step"],
+                                      "rows_per_s": r["value"]}), flush=True)
+        return
     if args.sweep5:
         # hit rate, rows/s and effective GB/s per point; 50 warm-up steps fill the caches, then `--steps` are timed
         args.e2e_steps = 0
