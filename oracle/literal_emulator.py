@@ -74,8 +74,28 @@ def fma32(a, b, c):
     return F(r)
 
 
+def fake_half(r, mode, key):
+    """FP16_to_FP32(FP32_to_FP16(x)) per element (Section 4.1), nearest or stochastic between the two FP16 neighbours."""
+    out = np.zeros(len(r), F)
+    for i, x in enumerate(r):
+        v = F(min(max(F(x), F(-65504.0)), F(65504.0)))
+        h = np.float16(v)                              # numpy converts with round-to-nearest-even
+        if mode == "nearest" or F(h) == v:
+            out[i] = F(h)
+            continue
+        if F(h) > v:
+            lo, hi = np.nextafter(h, np.float16(-np.inf)), h
+        else:
+            lo, hi = h, np.nextafter(h, np.float16(np.inf))
+        p = F(F(v - F(lo)) / F(F(hi) - F(lo)))
+        out[i] = F(hi) if uniform(key, i) < p else F(lo)
+    return out, None, None, None
+
+
 def fake_quantize(r, bits, mode, key):
     """Algorithm 1: r <- q*s + b with q = round_to_int((r-b)/s), in place semantics (returns a new row)."""
+    if bits == 16:
+        return fake_half(r, mode, key)
     d = len(r)
     b = F(min(r)) + F(0.0)
     mx = F(max(r))

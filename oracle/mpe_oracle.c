@@ -138,6 +138,60 @@ void orc_unpack(const uint8_t* packed, int32_t d, int32_t bits, uint8_t* q) {
         for (int j = 0; j < per; ++j) q[per * k + j] = (uint8_t)((packed[k] >> (bits * j)) & mask);
 }
 
+/* ------------------------------------------------------------------------ */
+/* FP16 table (Section 3 "Precision"/"Rounding": the two neighbours of x in    */
+/* FP16 differ by one unit in the last place)                                 */
+/* ------------------------------------------------------------------------ */
+float orc_half_to_float(uint16_t h) {
+    const int sign = h >> 15, e = (h >> 10) & 31, m = h & 1023;
+    float v;
+    if (e == 0) v = ldexpf((float)m, -24);                   /* zero and subnormals: m * 2^-24 */
+    else if (e == 31) v = m ? NAN : INFINITY;
+    else v = ldexpf((float)(m | 1024), e - 25);              /* 1.m * 2^(e-15) */
+    return sign ? -v : v;
+}
+
+/* FP32 -> FP16 with a chosen rounding direction: 0 nearest-even, 1 toward -inf, 2 toward +inf */
+uint16_t orc_float_to_half(float f, int32_t direction) {
+    uint32_t bits;
+    memcpy(&bits, &f, 4);
+    const uint32_t sign = bits >> 31, exp = (bits >> 23) & 255, man = bits & 0x7FFFFF;
+    if (exp == 255) return (uint16_t)((sign << 15) | 0x7C00 | (man ? 0x200 : 0));
+    /* |f| = m24 * 2^(e-23); FP32 subnormals are far below the smallest FP16 step and only leave a sticky bit */
+    const uint32_t m24 = exp ? (man | 0x800000) : man;
+    const int e = exp ? (int)exp - 127 : -126;
+    uint32_t h, rem, half_point;
+    if (e > 15) {                                             /* beyond the FP16 range (the caller clamps before) */
+        h = 0x7BFF; rem = 1; half_point = 0;
+    } else if (e >= -14) {                                    /* normal FP16: keep 11 of the 24 significand bits */
+        h = ((uint32_t)(e + 15) << 10) | ((m24 >> 13) & 1023);
+        rem = m24 & 0x1FFF; half_point = 0x1000;
+    } else {                                                  /* subnormal FP16: multiples of 2^-24 */
+        const int shift = 13 + (-14 - e);
+        if (shift >= 32) { h = 0; rem = m24 ? 1 : 0; half_point = 2; }
+        else { h = m24 >> shift; rem = m24 & ((1u << shift) - 1); half_point = 1u << (shift - 1); }
+    }
+    int up;                                                   /* whether the magnitude moves to the next code */
+    if (direction == 0) up = rem > half_point || (rem == half_point && rem != 0 && (h & 1));
+    else if (direction == 1) up = sign && rem != 0;
+    else up = !sign && rem != 0;
+    if (up) h += 1;                                           /* a carry runs into the exponent field, as it should */
+    return (uint16_t)((sign << 15) | h);
+}
+
+/* down-convert one row to FP16; codes16[c] receives the half-precision bits */
+void orc_to_half_row(const float* x, int32_t d, int32_t mode, uint32_t rowkey, uint16_t* codes16) {
+    for (int c = 0; c < d; ++c) {
+        const float v = fminf(fmaxf(x[c], -65504.0f), 65504.0f);      /* stay inside the finite FP16 range */
+        if (mode == ORC_RTN) { codes16[c] = orc_float_to_half(v, 0); continue; }
+        const uint16_t lo = orc_float_to_half(v, 1), hi = orc_float_to_half(v, 2);    /* x- <= x <= x+ */
+        if (lo == hi) { codes16[c] = lo; continue; }
+        const float flo = orc_half_to_float(lo), fhi = orc_half_to_float(hi);
+        const float p = (v - flo) / (fhi - flo);                  /* exact: both differences fit FP32, the step is a power of two */
+        codes16[c] = orc_uniform(rowkey, (uint32_t)c) < p ? hi : lo;  /* x+ with probability p: expectation x */
+    }
+}
+
 void orc_init_row(uint64_t seed, uint32_t table, uint32_t row, int32_t d, float lo, float hi, float* x) {
     uint32_t key = orc_rowkey(seed, ORC_DOMAIN_INIT, table, row, 0);
     float width = hi - lo;
@@ -231,6 +285,7 @@ static void initial_row(const orc* o, int32_t t, int64_t row, uint8_t* packed, f
     float x[1024];
     uint8_t q[1024];
     orc_init_row(o->seed, (uint32_t)t, (uint32_t)row, o->d, o->lo, o->hi, x);
+    if (o->bits == 16) { orc_to_half_row(x, o->d, ORC_RTN, 0, (uint16_t*)packed); *s = 1.0f; *b = 0.0f; return; }
     orc_quantize(x, o->d, o->bits, ORC_RTN, 0, q, s, b);
     orc_pack(q, o->d, o->bits, packed);
 }
@@ -272,7 +327,7 @@ orc* orc_create(const int64_t* num_rows, int32_t num_tables, int32_t dim, int32_
                 double cache_fraction, int32_t ways, int32_t policy, int32_t optimizer,
                 float eps, float init_lo, float init_hi, uint64_t seed) {
     if (num_tables < 1 || dim < 4 || dim > 1024 || (dim & (dim - 1)) != 0) return NULL;
-    if (bits != 8 && bits != 4 && bits != 2) return NULL;
+    if (bits != 8 && bits != 4 && bits != 2 && bits != 16) return NULL;
     if (ways == 0) ways = 32;
     if (ways < 1 || ways > 32 || (ways & (ways - 1)) != 0) return NULL;
     if (!(cache_fraction >= 0.0 && cache_fraction <= 1.0)) return NULL;
@@ -348,6 +403,11 @@ static void fetch(orc* o, int32_t t, int64_t row, float* x) {
     }
     int64_t id = rec_get(o, t, row);
     uint8_t q[1024];
+    if (o->bits == 16) {   /* FP16 table: the up-conversion is exact */
+        const uint16_t* hrow = (const uint16_t*)(tb->codes + id * o->code_bytes);
+        for (int c = 0; c < o->d; ++c) x[c] = orc_half_to_float(hrow[c]);
+        return;
+    }
     orc_unpack(tb->codes + id * o->code_bytes, o->d, o->bits, q);
     orc_dequantize(q, o->d, tb->scale[id], tb->bias[id], x);
 }
@@ -358,6 +418,7 @@ static void store_quantized(orc* o, int32_t t, int64_t row, const float* x, uint
     int64_t id = rec_get(o, t, row);
     uint8_t q[1024];
     uint32_t key = orc_rowkey(o->seed, domain, (uint32_t)t, (uint32_t)row, (uint64_t)step);
+    if (o->bits == 16) { orc_to_half_row(x, o->d, o->rounding, key, (uint16_t*)(tb->codes + id * o->code_bytes)); return; }
     orc_quantize(x, o->d, o->bits, o->rounding, key, q, &tb->scale[id], &tb->bias[id]);
     orc_pack(q, o->d, o->bits, tb->codes + id * o->code_bytes);
 }
@@ -622,7 +683,7 @@ void orc_memory_bytes(const orc* o, uint64_t out6[6]) {
     uint64_t lowprec = 0, cache = 0, tags = 0, pv = 0, opt = 0, fp32 = 0;
     for (int t = 0; t < o->T; ++t) {
         const uint64_t N = (uint64_t)o->tb[t].N, slots = (uint64_t)o->tb[t].n_sets * (uint64_t)o->ways;
-        lowprec += N * ((uint64_t)o->bits * (uint64_t)o->d + 64) / 8;   /* E x (bitwidth x D + 64) bits */
+        lowprec += N * ((uint64_t)o->bits * (uint64_t)o->d + (o->bits == 16 ? 0 : 64)) / 8;   /* E x (bitwidth x D + 64) bits; FP16 has no scale/bias */
         cache += slots * 4 * (uint64_t)o->d;                            /* 4 alpha n d bytes */
         tags += slots * 4;                                              /* INT32 per cached row */
         if (slots > 0) pv += o->policy == ORC_LFU ? N * 4 : slots * 4;  /* INT32 counter per embedding row (LFU) */

@@ -48,6 +48,11 @@ void orc_quantize(const float* x, int32_t d, int32_t bits, int32_t mode, uint32_
 void orc_dequantize(const uint8_t* q, int32_t d, float scale, float bias, float* x);
 void orc_pack(const uint8_t* q, int32_t d, int32_t bits, uint8_t* packed);
 void orc_unpack(const uint8_t* packed, int32_t d, int32_t bits, uint8_t* q);
+/* FP16 table: conversions with a chosen rounding direction (0 nearest-even, 1 toward -inf, 2 toward +inf) and the
+ * row-wise down-conversion with nearest or stochastic rounding between the two FP16 neighbours */
+float    orc_half_to_float(uint16_t h);
+uint16_t orc_float_to_half(float f, int32_t direction);
+void orc_to_half_row(const float* x, int32_t d, int32_t mode, uint32_t rowkey, uint16_t* codes16);
 void orc_init_row(uint64_t seed, uint32_t table, uint32_t row, int32_t d, float lo, float hi, float* x);
 /* Radix-32 summation tree over m rows of d floats (terms[j] points to row j). */
 void orc_tree_sum(const float* const* terms, int64_t m, int32_t d, float* out);

@@ -45,6 +45,9 @@ _quantize = _sig("orc_quantize", None, _f32p, C.c_int32, C.c_int32, C.c_int32, C
 _dequantize = _sig("orc_dequantize", None, _u8p, C.c_int32, C.c_float, C.c_float, _f32p)
 _pack = _sig("orc_pack", None, _u8p, C.c_int32, C.c_int32, _u8p)
 _unpack = _sig("orc_unpack", None, _u8p, C.c_int32, C.c_int32, _u8p)
+_h2f = _sig("orc_half_to_float", C.c_float, C.c_uint16)
+_f2h = _sig("orc_float_to_half", C.c_uint16, C.c_float, C.c_int32)
+_to_half_row = _sig("orc_to_half_row", None, _f32p, C.c_int32, C.c_int32, C.c_uint32, np.ctypeslib.ndpointer(np.uint16, flags="C_CONTIGUOUS"))
 _init_row = _sig("orc_init_row", None, C.c_uint64, C.c_uint32, C.c_uint32, C.c_int32, C.c_float, C.c_float, _f32p)
 _tree_sum = _sig("orc_tree_sum", None, C.POINTER(C.c_void_p), C.c_int64, C.c_int32, _f32p)
 
@@ -123,6 +126,22 @@ def unpack(packed, d, bits):
     packed = np.ascontiguousarray(packed, np.uint8)
     out = np.zeros(d, np.uint8)
     _unpack(packed, d, bits, out)
+    return out
+
+
+def half_to_float(h):
+    return np.float32(_h2f(int(h)))
+
+
+def float_to_half(f, direction=0):
+    """FP16 bits of f; direction 0 nearest-even, 1 toward -inf, 2 toward +inf."""
+    return int(_f2h(float(np.float32(f)), direction))
+
+
+def to_half_row(x, mode=RTN, key=0):
+    x = np.ascontiguousarray(x, np.float32)
+    out = np.zeros(x.shape[0], np.uint16)
+    _to_half_row(x, x.shape[0], mode, key, out)
     return out
 
 
@@ -260,4 +279,6 @@ class Oracle:
         if hit.size:
             return rows[hit[0]].copy()
         codes, s, b = self.row(t, row)
+        if self.bits == 16:
+            return codes.view(np.float16).astype(np.float32)
         return dequantize(unpack(codes, self.d, self.bits), s, b)

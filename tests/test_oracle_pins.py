@@ -329,6 +329,7 @@ def test_full_cache_equals_fp32_embedding_bag_training(policy, opt):
     (4, 2, "lru", "adagrad", 0.25), (8, 1, "lru", "sgd", 0.1), (8, 1, "lfu", "sgd", 0.1),
     (8, 2, "lru", "sgd", 0.0), (4, 2, "lfu", "sgd", 0.0), (2, 4, "lfu", "sgd", 0.25), (2, 2, "lru", "adagrad", 0.0),
     (-8, 2, "lru", "sgd", 0.25), (-4, 4, "lfu", "sgd", 0.0),      # negative width: round to nearest while training
+    (16, 2, "lru", "sgd", 0.25), (16, 4, "lfu", "adagrad", 0.0), (-16, 2, "lfu", "sgd", 0.25),   # FP16 table
 ])
 def test_two_space_oracle_equals_single_array_emulation(bits, ways, policy, opt, frac):
     nearest = bits < 0
@@ -493,3 +494,41 @@ def test_nearest_rounding_in_training_loses_small_updates_and_stochastic_does_no
         res[mode] = ((x0 - o.fetch_value(0, 1).astype(np.float64)) / step_size)[inner]
     assert np.all(np.abs(res[orc.RTN]) < 1.0)             # nothing accumulated: 100 updates of 0.2 steps all rounded away
     assert np.all(res[orc.SR] > 8.0)                      # expectation 20 quantization steps (until a column reaches the minimum)
+
+
+# --------------------------------------------------------- FP16 table ----
+def test_half_conversions_against_numpy_and_bracketing():
+    rng = np.random.default_rng(3)
+    xs = np.concatenate([rng.normal(0, 1, 4000), rng.normal(0, 1e-4, 2000), rng.normal(0, 3e-7, 2000), rng.uniform(-65504, 65504, 1000),
+                         [0.0, -0.0, 65504.0, -65504.0, 2.0 ** -24, 2.0 ** -25, 3 * 2.0 ** -25, 1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11,
+                          6.1e-5, 5.96e-8, 2.98e-8]]).astype(F)
+    for x in xs:
+        rn, rd, ru = (orc.float_to_half(x, m) for m in (0, 1, 2))
+        assert rn == int(np.float16(x).view(np.uint16)), x                     # numpy rounds to nearest even
+        lo, hi = orc.half_to_float(rd), orc.half_to_float(ru)
+        assert lo <= x <= hi
+        assert orc.half_to_float(rd) == np.array(rd, np.uint16).view(np.float16).astype(F)
+        if lo != hi:                                                            # neighbours: one unit in the last place apart
+            assert np.nextafter(np.array(rd, np.uint16).view(np.float16), np.float16(np.inf)).view(np.uint16) == ru or (lo == 0 and hi == 0)
+        else:
+            assert F(np.float16(x)) == x
+
+
+def test_half_stochastic_rounding_is_unbiased():
+    x = np.array([0.1, -0.3337, 1.0 + 2.0 ** -12, 3.3e-6, 100.123, 0.5], F)
+    K = 60000
+    acc = np.zeros(len(x))
+    for step in range(K):
+        h = orc.to_half_row(x, orc.SR, orc.rowkey(1, orc.DOMAIN_SR, 0, 5, step))
+        acc += h.view(np.float16).astype(np.float64)
+    ulp = np.array([float(np.spacing(np.float16(v))) for v in x])
+    assert np.all(np.abs(acc / K - x) <= 4.5 * (np.abs(ulp) / 2) / np.sqrt(K) + 1e-12)
+    assert orc.to_half_row(x, orc.RTN)[5] == int(np.float16(0.5).view(np.uint16))       # representable values never move
+    assert np.all(orc.to_half_row(np.array([0.5, -2.0, 0.0], F), orc.SR, 77) == np.array([0.5, -2.0, 0.0], np.float16).view(np.uint16))
+
+
+def test_fp16_table_halves_the_memory():
+    # Section 4.3: the compression factor of a non-cached FP16 table is 0.5
+    o = orc.Oracle([1000], 128, 16, 0.0, 32, orc.LFU)
+    m = o.memory_bytes().astype(np.float64)
+    assert (m[0] + m[1] + m[2] + m[3]) / m[5] == 0.5
