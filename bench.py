@@ -91,7 +91,7 @@ class ClockSampler:
 def describe(cfg):
     pol = "LFU" if cfg.policy == wl.LFU else "LRU"
     opt = "row-wise Adagrad" if cfg.optimizer == wl.ROWWISE_ADAGRAD else "SGD"
-    return (f"{cfg.name}: {cfg.num_tables} tables x {max(cfg.num_rows):,} rows x dim {cfg.dim}, INT{cfg.bits} row-wise, "
+    return (f"{cfg.name}: {cfg.num_tables} tables x {max(cfg.num_rows):,} rows x dim {cfg.dim}, {"FP16" if cfg.bits == 16 else "INT%d row-wise" % cfg.bits}, "
             f"cache {cfg.cache_fraction:g} x rows, {cfg.ways or 32}-way {pol}, batch {cfg.batch}, bags {cfg.bag}, {opt}")
 
 
@@ -106,7 +106,7 @@ def byte_model(cfg, L, U, U_hit, occ_hit, admissions, evictions, hot_occ, passes
     implementation touches; it is the numerator of the per-kernel roofline figure.
     """
     d, T, B = cfg.dim, cfg.num_tables, cfg.batch
-    rb = d * cfg.bits // 8 + 8      # codes + FP32 scale + FP32 bias
+    rb = d * cfg.bits // 8 + (0 if cfg.bits == 16 else 8)      # codes + FP32 scale + FP32 bias (none for an FP16 table)
     fb = 4 * d
     occ_miss, U_miss = L - occ_hit, U - U_hit
     out_bytes = 4 * B * T * d

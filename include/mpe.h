@@ -35,7 +35,7 @@ enum { MPE_ROUND_NEAREST = 0, MPE_ROUND_STOCHASTIC = 1 };
 enum {
     MPE_OK = 0,
     MPE_ERR_ARG = -1,          /* NULL pointer, negative size, value out of range */
-    MPE_ERR_UNSUPPORTED = -2,  /* unequal dims, dim not a power of two in [4,128], bits not 8/4/2, ways not 2^k <= 32 */
+    MPE_ERR_UNSUPPORTED = -2,  /* unequal dims, dim not a power of two in [4,128], bits not 16/8/4/2, ways not 2^k <= 32 */
     MPE_ERR_CUDA = -3,         /* a CUDA runtime call failed (detail = cudaError_t) */
     MPE_ERR_SEQUENCE = -4,     /* backward without a preceding forward, or step not strictly increasing */
     MPE_ERR_INDEX = -5,        /* device saw row ids outside [0, num_rows) (detail = how many); they were dropped */
@@ -48,7 +48,8 @@ enum {
  * Create the tables, the caches and the policy state on `device`.
  *   tables[num_tables]  row count and dimension of each table; all dims must be equal
  *                       (a power of two in [4,128]); num_rows in [1, 2^31-2].
- *   bits                8, 4 or 2: width of the integer codes, ranges [0,255], [0,15], [0,3] (Section 3 "Precision").
+ *   bits                8, 4 or 2: width of the integer codes, ranges [0,255], [0,15], [0,3]; or 16: an IEEE FP16
+ *                       table without scale/bias, rounded between the two FP16 neighbours (Section 3 "Precision").
  *   cache_fraction      in [0,1]; table t gets n_t = max(1, floor(cache_fraction*N_t + 1e-6) / ways) sets
  *                       of `ways` FP32 rows (Section 3 "Cache Structure"); 0 = no cache at all.
  *   ways                associativity alpha, a power of two <= 32; 0 selects 32 (Section 5.1).

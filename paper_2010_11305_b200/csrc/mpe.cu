@@ -207,7 +207,8 @@ void dispatch(int bits, int lanes, F&& f) {
     };
     if (bits == 8) by_lanes(std::integral_constant<int, 8>{});
     else if (bits == 4) by_lanes(std::integral_constant<int, 4>{});
-    else by_lanes(std::integral_constant<int, 2>{});
+    else if (bits == 2) by_lanes(std::integral_constant<int, 2>{});
+    else by_lanes(std::integral_constant<int, 16>{});
 }
 
 int check_launch(mpe_handle* h) {
@@ -243,7 +244,7 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
     if (!(cache_fraction >= 0.0 && cache_fraction <= 1.0)) return MPE_ERR_ARG;
     if (policy != MPE_LRU && policy != MPE_LFU) return MPE_ERR_ARG;
     if (optimizer != MPE_SGD && optimizer != MPE_ROWWISE_ADAGRAD) return MPE_ERR_ARG;
-    if (bits != 8 && bits != 4 && bits != 2) return MPE_ERR_UNSUPPORTED;
+    if (bits != 8 && bits != 4 && bits != 2 && bits != 16) return MPE_ERR_UNSUPPORTED;
     if (ways == 0) ways = 32;
     if (ways < 1 || ways > 32 || (ways & (ways - 1))) return MPE_ERR_UNSUPPORTED;
     const int dim = tables[0].dim;
@@ -299,7 +300,7 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
     if ((rc = dmalloc(h, &h->d_tables, num_tables, nullptr)) != MPE_OK) return fail(rc);
     s.tables = h->d_tables;
     if ((rc = dmalloc(h, &s.codes, h->total_rows * h->code_bytes, nullptr)) != MPE_OK) return fail(rc);
-    if ((rc = dmalloc(h, &s.sb, h->total_rows, nullptr)) != MPE_OK) return fail(rc);
+    if (bits != 16 && (rc = dmalloc(h, &s.sb, h->total_rows, nullptr)) != MPE_OK) return fail(rc);   // an FP16 table has no scale/bias
     if (policy == MPE_LFU && (rc = dmalloc(h, &s.cnt, h->total_rows, nullptr)) != MPE_OK) return fail(rc);
     if (optimizer == MPE_ROWWISE_ADAGRAD && (rc = dmalloc(h, &s.G, h->total_rows, nullptr)) != MPE_OK) return fail(rc);
     if ((rc = dmalloc(h, &s.slab, h->total_slots * dim, nullptr)) != MPE_OK) return fail(rc);
@@ -321,7 +322,8 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
         const int g = grid_for(h, h->tables[t].N, 256 / s.lanes, 8);
         if (bits == 8) LAUNCH(h, "init_table", k_init_table<8>, g, 256, 0, s, t, init_lo, init_hi);
         else if (bits == 4) LAUNCH(h, "init_table", k_init_table<4>, g, 256, 0, s, t, init_lo, init_hi);
-        else LAUNCH(h, "init_table", k_init_table<2>, g, 256, 0, s, t, init_lo, init_hi);
+        else if (bits == 2) LAUNCH(h, "init_table", k_init_table<2>, g, 256, 0, s, t, init_lo, init_hi);
+        else LAUNCH(h, "init_table", k_init_table<16>, g, 256, 0, s, t, init_lo, init_hi);
     }
     CKC(cudaGetLastError());
     CKC(cudaDeviceSynchronize());
@@ -622,7 +624,8 @@ int mpe_flush(mpe_handle* h) {
         const int g = grid_for(h, nslot, 256 / s.lanes, 8);
         if (h->bits == 8) LAUNCH(h, "flush", k_flush<8>, g, 256, 0, s, t, (uint64_t)h->last_step);
         else if (h->bits == 4) LAUNCH(h, "flush", k_flush<4>, g, 256, 0, s, t, (uint64_t)h->last_step);
-        else LAUNCH(h, "flush", k_flush<2>, g, 256, 0, s, t, (uint64_t)h->last_step);
+        else if (h->bits == 2) LAUNCH(h, "flush", k_flush<2>, g, 256, 0, s, t, (uint64_t)h->last_step);
+        else LAUNCH(h, "flush", k_flush<16>, g, 256, 0, s, t, (uint64_t)h->last_step);
     }
     return check_launch(h);
 }
@@ -675,7 +678,7 @@ int mpe_stats(mpe_handle* h, int32_t table, uint64_t* out8) {
 int mpe_memory_bytes(mpe_handle* h, uint64_t* out6) {
     if (!h || !out6) return MPE_ERR_ARG;
     const uint64_t N = (uint64_t)h->total_rows, slots = (uint64_t)h->total_slots, d = (uint64_t)h->dim;
-    out6[0] = N * ((uint64_t)h->bits * d + 64) / 8;                  // E x (bitwidth x D + 64) bits
+    out6[0] = N * ((uint64_t)h->bits * d + (h->bits == 16 ? 0 : 64)) / 8;   // E x (bitwidth x D + 64) bits; FP16 has no scale/bias
     out6[1] = slots * 4 * d;                                         // 4 alpha n d bytes
     out6[2] = slots * 4;                                             // one INT32 tag per cached row
     uint64_t pv = 0;

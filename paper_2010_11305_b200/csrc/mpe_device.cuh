@@ -4,6 +4,7 @@
 // code is spelled with an explicit rounding intrinsic so that the compiler can
 // neither contract nor reorder it.
 #pragma once
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -47,40 +48,53 @@ __device__ __forceinline__ uint32_t group_mask(int lanes_per_row) {
     return lanes_per_row == 32 ? 0xffffffffU : (((1U << lanes_per_row) - 1U) << (lane & ~(lanes_per_row - 1)));
 }
 
-// The four codes of one lane (columns 4*sub .. 4*sub+3) are BITS*4 adjacent bits of the row: one u32 (INT8),
-// one u16 (INT4) or one byte (INT2); the lowest column sits in the lowest bits.
+// The four stored values of one lane (columns 4*sub .. 4*sub+3) are BITS*4 adjacent bits of the row: one byte (INT2),
+// one u16 (INT4), one u32 (INT8) or two u32 (FP16 table, BITS = 16); the lowest column sits in the lowest bits.
 template <int BITS, bool RO>
-__device__ __forceinline__ uint32_t load_codes4(const uint8_t* codes, int64_t grow, int dim, int sub) {
+__device__ __forceinline__ uint2 load_codes4(const uint8_t* codes, int64_t grow, int dim, int sub) {
     const uint8_t* row = codes + grow * (dim * BITS / 8);
-    if (BITS == 8) return RO ? __ldg(reinterpret_cast<const uint32_t*>(row) + sub) : reinterpret_cast<const uint32_t*>(row)[sub];
-    if (BITS == 4) return RO ? __ldg(reinterpret_cast<const uint16_t*>(row) + sub) : reinterpret_cast<const uint16_t*>(row)[sub];
-    return RO ? __ldg(row + sub) : row[sub];
+    if (BITS == 16) return RO ? __ldg(reinterpret_cast<const uint2*>(row) + sub) : reinterpret_cast<const uint2*>(row)[sub];
+    uint32_t q;
+    if (BITS == 8) q = RO ? __ldg(reinterpret_cast<const uint32_t*>(row) + sub) : reinterpret_cast<const uint32_t*>(row)[sub];
+    else if (BITS == 4) q = RO ? __ldg(reinterpret_cast<const uint16_t*>(row) + sub) : reinterpret_cast<const uint16_t*>(row)[sub];
+    else q = RO ? __ldg(row + sub) : row[sub];
+    return make_uint2(q, 0u);
 }
 template <int BITS>
 __device__ __forceinline__ void store_codes4(uint8_t* codes, int64_t grow, int dim, int sub, uint32_t q0, uint32_t q1, uint32_t q2, uint32_t q3) {
     uint8_t* row = codes + grow * (dim * BITS / 8);
-    const uint32_t q = q0 | (q1 << BITS) | (q2 << (2 * BITS)) | (q3 << (3 * BITS));
+    if (BITS == 16) { reinterpret_cast<uint2*>(row)[sub] = make_uint2(q0 | (q1 << 16), q2 | (q3 << 16)); return; }
+    const uint32_t q = q0 | (q1 << (BITS & 15)) | (q2 << ((2 * BITS) & 31)) | (q3 << ((3 * BITS) & 31));
     if (BITS == 8) reinterpret_cast<uint32_t*>(row)[sub] = q;
     else if (BITS == 4) reinterpret_cast<uint16_t*>(row)[sub] = (uint16_t)q;
     else row[sub] = (uint8_t)q;
 }
 
-// four packed codes -> q*scale + bias (Algorithm 1, up-conversion)
+// four stored values -> FP32: q*scale + bias for integer codes (Algorithm 1, up-conversion), exact for FP16
 template <int BITS>
-__device__ __forceinline__ float4 decode4(uint32_t q, float2 p) {
-    constexpr uint32_t M = (1u << BITS) - 1u;
+__device__ __forceinline__ float4 decode4(uint2 qq, float2 p) {
     float4 x;
+    if (BITS == 16) {
+        x.x = __half2float(__ushort_as_half((unsigned short)(qq.x & 0xffffu)));
+        x.y = __half2float(__ushort_as_half((unsigned short)(qq.x >> 16)));
+        x.z = __half2float(__ushort_as_half((unsigned short)(qq.y & 0xffffu)));
+        x.w = __half2float(__ushort_as_half((unsigned short)(qq.y >> 16)));
+        return x;
+    }
+    constexpr uint32_t M = (1u << (BITS & 15)) - 1u;
+    const uint32_t q = qq.x;
     x.x = __fmaf_rn(__uint2float_rn(q & M), p.x, p.y);
-    x.y = __fmaf_rn(__uint2float_rn((q >> BITS) & M), p.x, p.y);
-    x.z = __fmaf_rn(__uint2float_rn((q >> (2 * BITS)) & M), p.x, p.y);
-    x.w = __fmaf_rn(__uint2float_rn((q >> (3 * BITS)) & M), p.x, p.y);
+    x.y = __fmaf_rn(__uint2float_rn((q >> (BITS & 15)) & M), p.x, p.y);
+    x.z = __fmaf_rn(__uint2float_rn((q >> ((2 * BITS) & 31)) & M), p.x, p.y);
+    x.w = __fmaf_rn(__uint2float_rn((q >> ((3 * BITS) & 31)) & M), p.x, p.y);
     return x;
 }
 
 // RO = the table is not written by the running kernel, so the read-only data path may serve the loads
 template <int BITS, bool RO>
 __device__ __forceinline__ float4 dequant4(const uint8_t* codes, const float2* sb, int64_t grow, int dim, int sub) {
-    const float2 p = RO ? __ldg(sb + grow) : sb[grow];
+    float2 p = make_float2(1.0f, 0.0f);
+    if (BITS != 16) p = RO ? __ldg(sb + grow) : sb[grow];
     return decode4<BITS>(load_codes4<BITS, RO>(codes, grow, dim, sub), p);
 }
 
@@ -101,10 +115,29 @@ __device__ __forceinline__ uint32_t quant1(float x, float mn, float inv, float q
     return (uint32_t)rintf(y);                             // nearest, ties to even
 }
 
+// one value -> FP16 bits: the nearer neighbour, or one of the two neighbours x- <= x <= x+ (one unit in the last
+// place apart) with P(x+) = (x - x-)/(x+ - x-)   (Section 3 "Rounding")
+__device__ __forceinline__ uint32_t half1(float x, uint32_t key, uint32_t column, bool stochastic) {
+    const float v = fminf(fmaxf(x, -65504.0f), 65504.0f);                    // stay inside the finite FP16 range
+    if (!stochastic) return __half_as_ushort(__float2half_rn(v));
+    const __half lo = __float2half_rd(v), hi = __float2half_ru(v);
+    const unsigned short blo = __half_as_ushort(lo), bhi = __half_as_ushort(hi);
+    if (blo == bhi) return blo;
+    const float flo = __half2float(lo), fhi = __half2float(hi);
+    const float p = __fdiv_rn(__fsub_rn(v, flo), __fsub_rn(fhi, flo));        // exact
+    return uniform01(key, column) < p ? bhi : blo;
+}
+
 // Down-convert one FP32 row (four columns per lane) into the low-precision table.
 template <int BITS>
 __device__ __forceinline__ void quantize_store(float4 x, uint8_t* __restrict__ codes, float2* __restrict__ sb,
                                                int64_t grow, int dim, int sub, int lanes_per_row, uint32_t key, bool stochastic) {
+    if (BITS == 16) {       // FP16 table: element-wise, no scale or bias
+        const uint32_t c = 4u * (uint32_t)sub;
+        store_codes4<BITS>(codes, grow, dim, sub, half1(x.x, key, c, stochastic), half1(x.y, key, c + 1, stochastic),
+                           half1(x.z, key, c + 2, stochastic), half1(x.w, key, c + 3, stochastic));
+        return;
+    }
     const uint32_t mask = group_mask(lanes_per_row);
     float mn = fminf(fminf(x.x, x.y), fminf(x.z, x.w));
     float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
@@ -113,7 +146,7 @@ __device__ __forceinline__ void quantize_store(float4 x, uint8_t* __restrict__ c
         mx = fmaxf(mx, __shfl_xor_sync(mask, mx, o));
     }
     mn = __fadd_rn(mn, 0.0f);                              // -0 -> +0
-    const float qmax = (float)((1 << BITS) - 1);
+    const float qmax = (float)((1 << (BITS & 15)) - 1);
     float s = __fdiv_rn(__fsub_rn(mx, mn), qmax);          // s = (max - min)/(2^N - 1)
     float inv = 0.0f;
     if (s >= 1.17549435e-38f) inv = __fdiv_rn(1.0f, s);

@@ -748,7 +748,7 @@ __device__ __forceinline__ void apply_update(const State& s, const TableDev& tb,
 
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
-struct RawRow { float4 f; uint32_t q; float2 sb; };
+struct RawRow { float4 f; uint2 q; float2 sb; };
 
 constexpr int UPD_WARPS = 4;     // warps per block of k_update
 constexpr int UPD_RING = 8;      // gradient rows a group can have in shared memory
@@ -812,7 +812,7 @@ k_update(State s, Work w, StepArgs av) {
                     for (int o = 0; o < dim * 4; o += 128) prefetch_l2(src + o);
                 } else {
                     prefetch_l2(s.codes + grow * (dim * BITS / 8));
-                    prefetch_l2(s.sb + grow);
+                    if (BITS != 16) prefetch_l2(s.sb + grow);
                 }
                 if (newcomer && victim >= 0) {
                     const int64_t vrow = rb + victim;
@@ -849,7 +849,7 @@ k_update(State s, Work w, StepArgs av) {
                 xr.f = reinterpret_cast<const float4*>(s.slab + (int64_t)loc * dim)[sub];
             } else {
                 const int64_t grow = ((int64_t)meta[cr][M_GROW_HI] << 32) | (uint32_t)meta[cr][M_GROW_LO];
-                xr.sb = s.sb[grow];
+                if (BITS != 16) xr.sb = s.sb[grow];
                 xr.q = load_codes4<BITS, false>(s.codes, grow, dim, sub);
             }
         };
@@ -1016,7 +1016,7 @@ __global__ void k_gather_rows(State s, int t, const int64_t* __restrict__ rows, 
         const int64_t g = tb.row_base + r;
         if (codes) {
             for (int c = 0; c < code_bytes; ++c) codes[i * code_bytes + c] = s.codes[g * code_bytes + c];
-            scale[i] = s.sb[g].x; bias[i] = s.sb[g].y;
+            scale[i] = s.sb ? s.sb[g].x : 1.0f; bias[i] = s.sb ? s.sb[g].y : 0.0f;
         }
         if (cnt) cnt[i] = s.cnt ? s.cnt[g] : 0u;
         if (G) G[i] = s.G ? s.G[g] : 0.0f;

@@ -42,7 +42,7 @@ def test_config2_lfu_many_tables():
     (8, wl.LRU, wl.SGD, 8, 16), (4, wl.LRU, wl.ROWWISE_ADAGRAD, 16, 64), (4, wl.LFU, wl.SGD, 32, 128),
     (8, wl.LFU, wl.ROWWISE_ADAGRAD, 32, 64), (4, wl.LFU, wl.SGD, 2, 32), (8, wl.LRU, wl.SGD, 1, 8),
     (4, wl.LFU, wl.SGD, 1, 4), (8, wl.LRU, wl.SGD, 4, 128), (2, wl.LFU, wl.SGD, 32, 128), (2, wl.LRU, wl.ROWWISE_ADAGRAD, 8, 16),
-    (2, wl.LFU, wl.SGD, 2, 4),
+    (2, wl.LFU, wl.SGD, 2, 4), (16, wl.LRU, wl.SGD, 32, 128), (16, wl.LFU, wl.ROWWISE_ADAGRAD, 4, 16), (16, wl.LFU, wl.SGD, 1, 4),
 ])
 def test_small_tables_every_variant(bits, policy, opt, ways, dim):
     """Small tables with a skewed stream: many hits, admissions, evictions, bypasses and chains per step."""
@@ -339,7 +339,7 @@ def test_graph_replay_and_plain_launches_agree_with_the_oracle():
     assert h.last_error() == (0, 0)
 
 
-@pytest.mark.parametrize("bits", [8, 4, 2])
+@pytest.mark.parametrize("bits", [8, 4, 2, 16])
 def test_round_to_nearest_while_training(bits):
     """Section 3 "Rounding": the nearest-even option instead of stochastic rounding, for updates, evictions and flush."""
     from parity_util import make_pair, compare_state
