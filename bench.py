@@ -330,6 +330,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep5", action="store_true", help="run every point of the policy/skew sweep (configuration 5): one JSON line per point")
     ap.add_argument("--sweep-assoc", action="store_true", help="associativity sweep (1..32 ways, LRU and LFU) on configuration 5's shape")
+    ap.add_argument("--bits", type=int, default=None, help="override the table precision: 16 (FP16), 8, 4 or 2")
+    ap.add_argument("--policy", default=None, choices=["lru", "lfu"], help="override the replacement policy")
     ap.add_argument("--tables", type=int, default=None, help="profiling aid: keep only the first TABLES tables")
     ap.add_argument("--rows-div", type=int, default=1, help="profiling aid: divide every table's row count")
     ap.add_argument("--batch-div", type=int, default=1, help="profiling aid: divide the batch size")
@@ -342,6 +344,12 @@ def main():
         c = wl.config(args.config)
         if args.tables is not None or args.rows_div != 1 or args.batch_div != 1:
             c = wl.scaled(c, rows_div=args.rows_div, batch_div=args.batch_div, tables=args.tables)
+        if args.bits is not None:
+            c.bits = args.bits
+            c.name += f"/bits{args.bits}"
+        if args.policy is not None:
+            c.policy = wl.LRU if args.policy == "lru" else wl.LFU
+            c.name += f"/{args.policy}"
         return c
 
     cfg = make_cfg()
