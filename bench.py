@@ -286,6 +286,55 @@ def run_ours(args, cfg, rank, world, local_rank):
     return result
 
 
+def run_tiering(args, local_rank):
+    """Effective bandwidth of forward and backward against the cache hit rate, with the low-precision table in HBM
+    and in pinned host memory (the experiment of the paper's Section 5.2, on synthetic streams).  One JSON line per point."""
+    from dataclasses import replace
+    from paper_2010_11305_b200 import binding as mpe
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    base = replace(wl.config(5), bits=args.bits or 16, policy=wl.LRU, cache_fraction=0.01)     # FP16 + 1 % LRU cache
+    warm, K = 30, max(args.steps, 5)
+    for placement, pname in ((mpe.TABLE_DEVICE, "device"), (mpe.TABLE_HOST, "host")):
+        for a in (None, 0.6, 0.8, 0.95, 1.05, 1.2, 1.4):
+            cfg = replace(base, zipf=[a] * base.num_tables, name=f"{pname}-{'uniform' if a is None else 'z%g' % a}")
+            h = mpe.Mpe(cfg.num_rows, cfg.dim, cfg.bits, cfg.cache_fraction, cfg.ways, cfg.policy, cfg.optimizer, cfg.eps,
+                        cfg.init_lo, cfg.init_hi, cfg.seed, local_rank, placement)
+            st = wl.Stream(cfg, dev)
+            out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, device=dev)
+            cs = torch.cuda.current_stream(dev)
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * K)]
+            s0 = None
+            for step in range(1, warm + K + 1):
+                idx, off, grad = st.batch(step)
+                j = step - warm - 1
+                if j == 0:
+                    torch.cuda.synchronize(dev)
+                    s0 = np.sum([h.stats(t) for t in range(cfg.num_tables)], axis=0).astype(np.int64)
+                if j >= 0:
+                    ev[3 * j].record(cs)
+                h.forward(idx, off, cfg.batch, out, cs.cuda_stream)
+                if j >= 0:
+                    ev[3 * j + 1].record(cs)
+                h.backward(grad, cfg.lr, step)
+                if j >= 0:
+                    ev[3 * j + 2].record(cs)
+            torch.cuda.synchronize(dev)
+            ds = (np.sum([h.stats(t) for t in range(cfg.num_tables)], axis=0).astype(np.int64) - s0) / K
+            L, occ_hit, U, U_hit, adm, evi = (float(ds[i]) for i in range(6))
+            fwd_ms = float(np.median([ev[3 * j].elapsed_time(ev[3 * j + 1]) for j in range(K)]))
+            bwd_ms = float(np.median([ev[3 * j + 1].elapsed_time(ev[3 * j + 2]) for j in range(K)]))
+            d, T, B = cfg.dim, cfg.num_tables, cfg.batch
+            rb, fb = d * cfg.bits // 8 + (0 if cfg.bits == 16 else 8), 4 * d
+            fwd_bytes = 4 * L + occ_hit * fb + (L - occ_hit) * rb + 4 * B * T * d
+            bwd_bytes = L * fb + U_hit * 2 * fb + (U - U_hit) * 2 * rb + 4 * U_hit + evi * (fb + rb) + adm * fb
+            print(json.dumps({"placement": pname, "stream": "uniform" if a is None else f"zipf {a}", "index_hit_rate": occ_hit / max(L, 1),
+                              "fwd_ms": fwd_ms, "bwd_ms": bwd_ms, "fwd_effective_gbs": fwd_bytes / fwd_ms / 1e6,
+                              "bwd_effective_gbs": bwd_bytes / bwd_ms / 1e6, "rows_per_s": L / (fwd_ms + bwd_ms) * 1e3}), flush=True)
+            h.close()
+            del st
+
+
 def sample_tables(cfg, budget_rows):
     """How many tables of the configuration the CPU oracle can process in the time budget (~10-30 s)."""
     per_table = cfg.batch * (cfg.bag[1] if cfg.bag[0] != "fixed" else cfg.bag[1])
@@ -329,6 +378,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep5", action="store_true", help="run every point of the policy/skew sweep (configuration 5): one JSON line per point")
+    ap.add_argument("--tiering", action="store_true", help="forward/backward effective bandwidth vs hit rate, table in HBM and in host memory")
     ap.add_argument("--sweep-assoc", action="store_true", help="associativity sweep (1..32 ways, LRU and LFU) on configuration 5's shape")
     ap.add_argument("--bits", type=int, default=None, help="override the table precision: 16 (FP16), 8, 4 or 2")
     ap.add_argument("--policy", default=None, choices=["lru", "lfu"], help="override the replacement policy")
@@ -371,6 +421,9 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if args.tiering:
+        run_tiering(args, local_rank)
+        return
     if args.sweep_assoc:
         # hit rate per (ways, policy, cache size) on a Zipf(1.05) stream: the layout of the paper's hit-rate table
         from dataclasses import replace

@@ -67,6 +67,16 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
                double cache_fraction, int32_t ways, int32_t policy, int32_t optimizer, float eps,
                float init_lo, float init_hi, uint64_t seed, int32_t device);
 
+/* Same, with a choice of where the low-precision table lives.  MPE_TABLE_DEVICE keeps everything in HBM.
+ * MPE_TABLE_HOST keeps the codes and (scale, bias) in pinned host memory that the kernels read and write in place
+ * over the host link, while the FP32 cache and all policy and optimizer state stay in HBM: the arrangement of the
+ * paper's speed experiment (Section 5.2), where a table too large for the device sits behind the cache.  Results
+ * are bit-identical for both placements. */
+enum { MPE_TABLE_DEVICE = 0, MPE_TABLE_HOST = 1 };
+int mpe_create_placed(mpe_handle** out, const mpe_table_spec* tables, int32_t num_tables, int32_t bits,
+                      double cache_fraction, int32_t ways, int32_t policy, int32_t optimizer, float eps,
+                      float init_lo, float init_hi, uint64_t seed, int32_t device, int32_t table_placement);
+
 /* Size the per-step workspace for batches of up to max_batch samples and max_total_indices
  * indices, so that later steps allocate nothing.  mpe_forward grows the workspace by itself
  * (a synchronising reallocation) when a larger batch arrives. */

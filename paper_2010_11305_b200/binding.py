@@ -17,11 +17,12 @@ LIB_PATH = os.path.join(_HERE, "libmpe.so")
 LRU, LFU = 0, 1
 SGD, ROWWISE_ADAGRAD = 0, 1
 ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
+TABLE_DEVICE, TABLE_HOST = 0, 1
 OK, ERR_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_SEQUENCE, ERR_INDEX, ERR_OFFSETS, ERR_NOMEM, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6, -7, -8
 STATIC_MAX_INDICES, STATIC_MAX_BAGS, STATIC_MAX_TABLES = 32768, 32768, 64
 
 EXPORTS = [
-    "mpe_create", "mpe_reserve", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_set_rounding", "mpe_step_host", "mpe_flush", "mpe_destroy",
+    "mpe_create", "mpe_create_placed", "mpe_reserve", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_set_rounding", "mpe_step_host", "mpe_flush", "mpe_destroy",
     "mpe_last_error", "mpe_stats", "mpe_memory_bytes", "mpe_cache_geometry", "mpe_step_info", "mpe_export_rows",
     "mpe_export_cache", "mpe_export_aux", "mpe_use_graphs", "mpe_kernel_launches", "mpe_profile", "mpe_profile_read", "mpe_error_string",
 ]
@@ -41,6 +42,7 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
 _lib = load_library()
 _vp, _i32, _i64, _u64, _f32, _f64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64, C.c_float, C.c_double
 _lib.mpe_create.argtypes = [C.POINTER(_vp), C.POINTER(TableSpec), _i32, _i32, _f64, _i32, _i32, _i32, _f32, _f32, _f32, _u64, _i32]
+_lib.mpe_create_placed.argtypes = [C.POINTER(_vp), C.POINTER(TableSpec), _i32, _i32, _f64, _i32, _i32, _i32, _f32, _f32, _f32, _u64, _i32, _i32]
 _lib.mpe_reserve.argtypes = [_vp, _i32, _i64]
 _lib.mpe_forward.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp]
 _lib.mpe_forward_static.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp]
@@ -93,13 +95,17 @@ class Mpe:
     """Handle of one embedding collection on one GPU (see include/mpe.h for the semantics)."""
 
     def __init__(self, num_rows, dim, bits, cache_fraction, ways, policy, optimizer=SGD, eps=1e-8, init_lo=-0.05,
-                 init_hi=0.05, seed=0, device=0):
+                 init_hi=0.05, seed=0, device=0, table_placement=TABLE_DEVICE):
         self.T, self.dim, self.bits = len(num_rows), dim, bits
         self.num_rows = [int(n) for n in num_rows]
         specs = (TableSpec * self.T)(*[TableSpec(int(n), dim) for n in num_rows])
         h = _vp()
-        _check(_lib.mpe_create(C.byref(h), specs, self.T, bits, cache_fraction, ways, policy, optimizer, eps, init_lo,
-                               init_hi, seed, device), "mpe_create")
+        if table_placement == TABLE_DEVICE:
+            _check(_lib.mpe_create(C.byref(h), specs, self.T, bits, cache_fraction, ways, policy, optimizer, eps, init_lo,
+                                   init_hi, seed, device), "mpe_create")
+        else:
+            _check(_lib.mpe_create_placed(C.byref(h), specs, self.T, bits, cache_fraction, ways, policy, optimizer, eps,
+                                          init_lo, init_hi, seed, device, table_placement), "mpe_create_placed")
         self._h = h
         self.device = device
         self.ways = self.cache_geometry(0)[1]

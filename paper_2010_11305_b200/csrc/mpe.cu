@@ -23,6 +23,7 @@ struct ProfRec { int name; cudaEvent_t a, b; };
 
 struct mpe_handle {
     int device = 0, num_sms = 148;
+    bool table_on_host = false;
     int T = 0, dim = 0, bits = 0, ways = 0, policy = 0, optimizer = 0, code_bytes = 0;
     float eps = 0, lo = 0, hi = 0;
     uint64_t seed = 0;
@@ -239,7 +240,15 @@ const char* mpe_error_string(int code) {
 int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_tables, int32_t bits,
                double cache_fraction, int32_t ways, int32_t policy, int32_t optimizer, float eps,
                float init_lo, float init_hi, uint64_t seed, int32_t device) {
+    return mpe_create_placed(out, tables, num_tables, bits, cache_fraction, ways, policy, optimizer, eps, init_lo, init_hi, seed,
+                             device, MPE_TABLE_DEVICE);
+}
+
+int mpe_create_placed(mpe_handle** out, const mpe_table_spec* tables, int32_t num_tables, int32_t bits,
+                      double cache_fraction, int32_t ways, int32_t policy, int32_t optimizer, float eps,
+                      float init_lo, float init_hi, uint64_t seed, int32_t device, int32_t table_placement) {
     if (!out || !tables || num_tables < 1) return MPE_ERR_ARG;
+    if (table_placement != MPE_TABLE_DEVICE && table_placement != MPE_TABLE_HOST) return MPE_ERR_ARG;
     *out = nullptr;
     if (!(cache_fraction >= 0.0 && cache_fraction <= 1.0)) return MPE_ERR_ARG;
     if (policy != MPE_LRU && policy != MPE_LFU) return MPE_ERR_ARG;
@@ -258,6 +267,7 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
 
     mpe_handle* h = new mpe_handle();
     h->device = device;
+    h->table_on_host = table_placement == MPE_TABLE_HOST;
     DeviceGuard guard(device);
     cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, device);
     if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess ||
@@ -299,8 +309,17 @@ int mpe_create(mpe_handle** out, const mpe_table_spec* tables, int32_t num_table
     auto fail = [&](int code) { mpe_destroy(h); return code; };
     if ((rc = dmalloc(h, &h->d_tables, num_tables, nullptr)) != MPE_OK) return fail(rc);
     s.tables = h->d_tables;
-    if ((rc = dmalloc(h, &s.codes, h->total_rows * h->code_bytes, nullptr)) != MPE_OK) return fail(rc);
-    if (bits != 16 && (rc = dmalloc(h, &s.sb, h->total_rows, nullptr)) != MPE_OK) return fail(rc);   // an FP16 table has no scale/bias
+    if (h->table_on_host) {
+        // capacity tiering: the low-precision table stays in pinned host memory and is read and written in place over
+        // the host link; the FP32 cache, tags, counters and optimizer state stay in HBM
+        if (cudaHostAlloc((void**)&s.codes, (size_t)h->total_rows * h->code_bytes, cudaHostAllocMapped | cudaHostAllocPortable) != cudaSuccess)
+            return fail(MPE_ERR_NOMEM);
+        if (bits != 16 && cudaHostAlloc((void**)&s.sb, (size_t)h->total_rows * sizeof(float2), cudaHostAllocMapped | cudaHostAllocPortable) != cudaSuccess)
+            return fail(MPE_ERR_NOMEM);
+    } else {
+        if ((rc = dmalloc(h, &s.codes, h->total_rows * h->code_bytes, nullptr)) != MPE_OK) return fail(rc);
+        if (bits != 16 && (rc = dmalloc(h, &s.sb, h->total_rows, nullptr)) != MPE_OK) return fail(rc);   // an FP16 table has no scale/bias
+    }
     if (policy == MPE_LFU && (rc = dmalloc(h, &s.cnt, h->total_rows, nullptr)) != MPE_OK) return fail(rc);
     if (optimizer == MPE_ROWWISE_ADAGRAD && (rc = dmalloc(h, &s.G, h->total_rows, nullptr)) != MPE_OK) return fail(rc);
     if ((rc = dmalloc(h, &s.slab, h->total_slots * dim, nullptr)) != MPE_OK) return fail(rc);
@@ -643,7 +662,8 @@ int mpe_destroy(mpe_handle* h) {
     for (cudaEvent_t e : {h->ev_idx, h->ev_grad, h->ev_fwd, h->ev_start}) if (e) cudaEventDestroy(e);
     free_workspace(h);
     State& s = h->st;
-    cudaFree(h->d_tables); cudaFree(s.codes); cudaFree(s.sb); cudaFree(s.cnt); cudaFree(s.G); cudaFree(s.slab);
+    if (h->table_on_host) { cudaFreeHost(s.codes); cudaFreeHost(s.sb); } else { cudaFree(s.codes); cudaFree(s.sb); }
+    cudaFree(h->d_tables); cudaFree(s.cnt); cudaFree(s.G); cudaFree(s.slab);
     cudaFree(s.tags); cudaFree(s.ts); cudaFree(s.hit_epoch); cudaFree(s.hit_k); cudaFree(s.stats);
     cudaFree(h->sh_idx); cudaFree(h->sh_off); cudaFree(h->sh_grad); cudaFree(h->sh_out);
     for (auto& r : h->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }

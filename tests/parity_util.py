@@ -8,11 +8,11 @@ from oracle import mpe_oracle as orc
 from paper_2010_11305_b200 import workloads as wl
 
 
-def make_pair(cfg, tables=None):
+def make_pair(cfg, tables=None, table_placement=0):
     """(Mpe handle, Oracle) for a configuration; `tables` restricts the oracle to a sample of tables."""
     from paper_2010_11305_b200 import binding as mpe
     h = mpe.Mpe(cfg.num_rows, cfg.dim, cfg.bits, cfg.cache_fraction, cfg.ways, cfg.policy, cfg.optimizer, cfg.eps,
-                cfg.init_lo, cfg.init_hi, cfg.seed, 0)
+                cfg.init_lo, cfg.init_hi, cfg.seed, 0, table_placement)
     o = orc.Oracle(cfg.num_rows, cfg.dim, cfg.bits, cfg.cache_fraction, cfg.ways, cfg.policy, cfg.optimizer, cfg.eps,
                    cfg.init_lo, cfg.init_hi, cfg.seed)
     if tables is not None:

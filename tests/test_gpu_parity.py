@@ -372,3 +372,27 @@ def test_round_to_nearest_while_training(bits):
             h.flush()
             o.flush()
             compare_state(h, o, cfg, [0, 1], rng)
+
+
+@pytest.mark.parametrize("bits,policy", [(4, wl.LFU), (16, wl.LRU)])
+def test_table_in_host_memory_gives_the_same_results(bits, policy):
+    """Capacity tiering (Section 5.2): the low-precision table in pinned host memory, the FP32 cache in HBM."""
+    from parity_util import make_pair, compare_state
+    from paper_2010_11305_b200 import binding as mpe
+    cfg = _cfg(num_rows=[20000, 700], dim=64, bits=bits, batch=128, bag=("poisson", 8.0), zipf=[1.1, 1.0], policy=policy, ways=8,
+               cache_fraction=0.05, seed=31)
+    h, o = make_pair(cfg, table_placement=mpe.TABLE_HOST)
+    rng = np.random.default_rng(0)
+    st = wl.Stream(cfg, "cpu")
+    for step in range(1, 6):
+        idx, off, grad = st.batch(step)
+        out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, device="cuda")
+        h.forward(idx.cuda(), off.cuda(), cfg.batch, out)
+        ref = o.forward(idx.numpy(), off.numpy(), cfg.batch)
+        assert np.array_equal(out.cpu().numpy(), ref)
+        h.backward(grad.cuda(), cfg.lr, step)
+        o.backward(grad.numpy(), cfg.lr, step)
+    compare_state(h, o, cfg, [0, 1], rng)
+    h.flush()
+    o.flush()
+    compare_state(h, o, cfg, [0, 1], rng)
