@@ -98,6 +98,35 @@ int mpe_reserve(mpe_handle* h, int32_t max_batch, int64_t max_total_indices);
 int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch,
                 int64_t total_indices, float* d_out, void* cuda_stream);
 
+/* ---- Tables partitioned over several GPUs (Section 1: embeddings are placed model-parallel, with no replication) ----
+ * Each rank owns some of the tables and sees the whole batch's indices for them; sample b of a batch of `batch` samples
+ * belongs to rank b / (batch / n_ranks).  After the forward pass every rank needs the pooled vectors of ITS samples for ALL
+ * tables (an all-to-all); before the backward pass every rank needs the gradients of ALL samples for ITS tables (the reverse).
+ * The paper names the partitioning only; the exchange below is this library's.  The kernels of different ranks never
+ * wait for one another: the caller orders them (a barrier between "all ranks have run forward" and "a rank reads its buffer").
+ *
+ * mpe_forward_routed: as mpe_forward, but the pooled vector of local table t and sample b is stored by the pooling kernel
+ *   itself at out_ptrs[b / B_local] + ((b % B_local) * tables_global + table_base + t) * dim, B_local = batch / n_ranks.
+ *   out_ptrs: HOST array of n_ranks DEVICE pointers (this GPU's own buffer and peers' buffers mapped into this process),
+ *   each a float [B_local][tables_global * dim] array, 16-byte aligned; the array is read before the call returns.
+ *   Errors: MPE_ERR_ARG when n_ranks is outside 1..72, batch is not a multiple of n_ranks, a pointer is null or unaligned,
+ *   or table_base + (tables of this handle) exceeds tables_global; otherwise as mpe_forward.
+ * mpe_gather_grad: d_grad_local[b][t][:] = grad_ptrs[b / B_local][(b % B_local)][table_base + t][:] for the handle's tables,
+ *   plain loads from the owners' memory; d_grad_local is a DEVICE float [batch][tables * dim] array (caller-owned) that
+ *   mpe_backward then takes.  Same pointer rules and errors as above.
+ * mpe_peer_buffer_*: exchange buffers that other processes can map.  alloc: `bytes` of device memory on `device` plus the
+ *   64-byte handle to send to the peers; open: map a peer's handle (enables peer access on first use); close: unmap;
+ *   free: release an allocated buffer (after every peer has closed it).  Errors: MPE_ERR_ARG, MPE_ERR_NOMEM, MPE_ERR_CUDA. */
+#define MPE_IPC_HANDLE_BYTES 64
+int mpe_forward_routed(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch, int64_t total_indices,
+                       float* const* out_ptrs, int32_t n_ranks, int32_t tables_global, int32_t table_base, void* cuda_stream);
+int mpe_gather_grad(mpe_handle* h, const float* const* grad_ptrs, int32_t n_ranks, int32_t tables_global, int32_t table_base,
+                    int32_t batch, float* d_grad_local, void* cuda_stream);
+int mpe_peer_buffer_alloc(int32_t device, int64_t bytes, void** d_ptr, void* ipc_handle);
+int mpe_peer_buffer_open(int32_t device, const void* ipc_handle, void** d_ptr);
+int mpe_peer_buffer_close(int32_t device, void* d_ptr);
+int mpe_peer_buffer_free(int32_t device, void* d_ptr);
+
 /*
  * Backward of the preceding mpe_forward, on the same stream: update(T, C, i, x) for every distinct
  * row of the batch (Section 3, Algorithm 2).

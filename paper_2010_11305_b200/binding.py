@@ -24,7 +24,9 @@ STATIC_MAX_INDICES, STATIC_MAX_BAGS, STATIC_MAX_TABLES = 32768, 32768, 64
 EXPORTS = [
     "mpe_create", "mpe_create_placed", "mpe_reserve", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_set_rounding", "mpe_step_host", "mpe_flush", "mpe_destroy",
     "mpe_last_error", "mpe_stats", "mpe_memory_bytes", "mpe_cache_geometry", "mpe_step_info", "mpe_export_rows",
-    "mpe_export_cache", "mpe_export_aux", "mpe_use_graphs", "mpe_kernel_launches", "mpe_profile", "mpe_profile_read", "mpe_error_string",
+    "mpe_export_cache", "mpe_export_aux", "mpe_use_graphs", "mpe_kernel_launches", "mpe_profile", "mpe_profile_read",
+    "mpe_forward_routed", "mpe_gather_grad", "mpe_peer_buffer_alloc", "mpe_peer_buffer_open", "mpe_peer_buffer_close", "mpe_peer_buffer_free",
+    "mpe_error_string",
 ]
 
 
@@ -63,6 +65,12 @@ _lib.mpe_set_rounding.argtypes = [_vp, _i32]
 _lib.mpe_kernel_launches.argtypes = [_vp, C.POINTER(_u64)]
 _lib.mpe_profile.argtypes = [_vp, _i32]
 _lib.mpe_profile_read.argtypes = [_vp, _i32, _vp, _vp, _vp, C.POINTER(_i32)]
+_lib.mpe_forward_routed.argtypes = [_vp, _vp, _vp, _i32, _i64, C.POINTER(_vp), _i32, _i32, _i32, _vp]
+_lib.mpe_gather_grad.argtypes = [_vp, C.POINTER(_vp), _i32, _i32, _i32, _i32, _vp, _vp]
+_lib.mpe_peer_buffer_alloc.argtypes = [_i32, _i64, C.POINTER(_vp), _vp]
+_lib.mpe_peer_buffer_open.argtypes = [_i32, _vp, C.POINTER(_vp)]
+_lib.mpe_peer_buffer_close.argtypes = [_i32, _vp]
+_lib.mpe_peer_buffer_free.argtypes = [_i32, _vp]
 _lib.mpe_error_string.argtypes = [C.c_int]
 _lib.mpe_error_string.restype = C.c_char_p
 for _n in EXPORTS[:-1]:
@@ -130,6 +138,18 @@ class Mpe:
         """Evaluation forward for callers that must not allocate: its scratch is a fixed array inside the library."""
         _check(_lib.mpe_forward_static(self._h, _ptr(d_indices), _ptr(d_offsets), batch, d_indices.numel(), _ptr(d_out),
                                        stream), "mpe_forward_static")
+
+    def forward_routed(self, d_indices, d_offsets, batch, out_ptrs, tables_global, table_base, stream=None):
+        """Forward whose pooled vectors go straight to their owners' buffers; out_ptrs: one device address per rank."""
+        arr = (_vp * len(out_ptrs))(*[int(p) for p in out_ptrs])
+        _check(_lib.mpe_forward_routed(self._h, _ptr(d_indices), _ptr(d_offsets), batch, d_indices.numel(), arr, len(out_ptrs),
+                                       tables_global, table_base, stream), "mpe_forward_routed")
+
+    def gather_grad(self, grad_ptrs, tables_global, table_base, batch, d_grad_local, stream=None):
+        """Pull this handle's columns of every rank's gradient buffer into d_grad_local ([batch][tables * dim])."""
+        arr = (_vp * len(grad_ptrs))(*[int(p) for p in grad_ptrs])
+        _check(_lib.mpe_gather_grad(self._h, arr, len(grad_ptrs), tables_global, table_base, batch, _ptr(d_grad_local), stream),
+               "mpe_gather_grad")
 
     def backward(self, d_grad_out, lr, step):
         _check(_lib.mpe_backward(self._h, _ptr(d_grad_out), lr, step), "mpe_backward")
@@ -221,3 +241,27 @@ class Mpe:
             name = names.raw[32 * i:32 * i + 32].split(b"\0")[0].decode()
             out[name] = (float(ms[i]), int(launches[i]))
         return out
+
+
+IPC_HANDLE_BYTES = 64
+
+
+def peer_buffer_alloc(device, nbytes):
+    """(device address, 64-byte handle other processes can open) of a fresh exchange buffer."""
+    p, hd = _vp(), C.create_string_buffer(IPC_HANDLE_BYTES)
+    _check(_lib.mpe_peer_buffer_alloc(device, nbytes, C.byref(p), hd), "mpe_peer_buffer_alloc")
+    return p.value, hd.raw
+
+
+def peer_buffer_open(device, handle):
+    p = _vp()
+    _check(_lib.mpe_peer_buffer_open(device, C.create_string_buffer(handle, IPC_HANDLE_BYTES), C.byref(p)), "mpe_peer_buffer_open")
+    return p.value
+
+
+def peer_buffer_close(device, address):
+    _check(_lib.mpe_peer_buffer_close(device, address), "mpe_peer_buffer_close")
+
+
+def peer_buffer_free(device, address):
+    _check(_lib.mpe_peer_buffer_free(device, address), "mpe_peer_buffer_free")

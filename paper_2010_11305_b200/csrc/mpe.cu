@@ -55,6 +55,7 @@ struct mpe_handle {
     int32_t B = 0; int64_t L = 0;
     const uint32_t *skey = nullptr, *spos = nullptr;
     StepArgs args{};                        // the current call's arguments (passed by value when launching directly)
+    Route* d_route = nullptr;               // destinations of the pooled vectors when the tables are spread over several GPUs
     // CUDA graphs of the two halves of a step (small batches are launch-latency bound)
     bool graphs_enabled = true;
     cudaStream_t cap = nullptr;             // stream the step is captured on
@@ -486,17 +487,9 @@ int capture(mpe_handle* h, cudaGraph_t* graph, cudaGraphExec_t* exec, cudaGraphN
     return *args_node ? MPE_OK : MPE_ERR_CUDA;
 }
 
-}  // namespace
-
-extern "C" {
-
-int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch,
-                int64_t total_indices, float* d_out, void* cuda_stream) {
-    if (!h || !d_offsets || batch < 0 || total_indices < 0 || total_indices > 0x7ffffff0LL) return MPE_ERR_ARG;
-    if ((total_indices > 0 && !d_indices) || (batch > 0 && !d_out)) return MPE_ERR_ARG;
-    DeviceGuard guard(h->device);
-    cudaStream_t stream = (cudaStream_t)cuda_stream;
-    if (stream != h->stream) { CK(h, cudaStreamSynchronize(h->stream)); h->stream = stream; }
+// forward with the pooled vectors going either to d_out (route == nullptr) or to the buffers the route names
+int forward_impl(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch,
+                 int64_t total_indices, float* d_out, const Route* route) {
     h->have_forward = false;
     const int64_t bags = (int64_t)h->T * batch;
     if (total_indices > h->cap_L || bags > h->cap_bags || !h->wk.ctr) {
@@ -507,18 +500,19 @@ int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offset
     uint32_t L = (uint32_t)total_indices;
     h->B = batch; h->L = total_indices; ++h->epoch;
     h->args.indices = d_indices; h->args.offsets = d_offsets; h->args.out = d_out; h->args.B = batch; h->args.L = L; h->args.epoch = h->epoch;
+    h->args.route = route;
     int rc = MPE_OK;
     if (may_use_graph(h)) {
         if (!h->x_fwd) {
             rc = capture(h, &h->g_fwd, &h->x_fwd, &h->n_fwd, &h->k_fwd, (const void*)k_set_args_forward, [&]() {
-                LAUNCH(h, "set_args", k_set_args_forward, 1, 1, 0, w.args, d_indices, d_offsets, d_out, batch, L, h->epoch);
+                LAUNCH(h, "set_args", k_set_args_forward, 1, 1, 0, w.args, d_indices, d_offsets, d_out, batch, L, h->epoch, route);
                 return enqueue_forward(h, h->cap_L, h->cap_bags, true);
             });
             if (rc != MPE_OK) { drop_graphs(h); h->graphs_enabled = false; }      // fall back to plain launches for good
         }
         if (rc == MPE_OK) {
             StepArgs* a = w.args;
-            void* params[] = {&a, &d_indices, &d_offsets, &d_out, &batch, &L, &h->epoch};
+            void* params[] = {&a, &d_indices, &d_offsets, &d_out, &batch, &L, &h->epoch, &route};
             cudaKernelNodeParams kp{};
             kp.func = (void*)k_set_args_forward; kp.gridDim = dim3(1); kp.blockDim = dim3(1); kp.kernelParams = params;
             CK(h, cudaGraphExecKernelNodeSetParams(h->x_fwd, h->n_fwd, &kp));
@@ -532,6 +526,107 @@ int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offset
     if (rc != MPE_OK) return rc;
     h->have_forward = true;
     return MPE_OK;
+}
+
+int check_route(const mpe_handle* h, const void* const* ptrs, int32_t n_ranks, int32_t tables_global, int32_t table_base, int32_t batch) {
+    if (!ptrs || n_ranks < 1 || n_ranks > MAX_RANKS || batch < 0 || batch % n_ranks != 0) return MPE_ERR_ARG;
+    if (table_base < 0 || tables_global < table_base + h->T) return MPE_ERR_ARG;
+    for (int g = 0; g < n_ranks; ++g)
+        if (!ptrs[g] || (reinterpret_cast<uintptr_t>(ptrs[g]) & 15)) return MPE_ERR_ARG;
+    return MPE_OK;
+}
+
+// the route travels to the device as a kernel argument, so the caller's array may be reused at once
+int send_route(mpe_handle* h, const void* const* ptrs, int32_t n_ranks, int32_t tables_global, int32_t table_base, int32_t batch) {
+    if (!h->d_route) CK(h, cudaMalloc(&h->d_route, sizeof(Route)));
+    Route r{};
+    for (int g = 0; g < n_ranks; ++g) r.out[g] = const_cast<float*>(static_cast<const float*>(ptrs[g]));
+    r.B_local = batch / n_ranks > 0 ? batch / n_ranks : 1; r.T_global = tables_global; r.t_base = table_base; r.n_ranks = n_ranks;
+    LAUNCH(h, "set_route", k_set_route, 1, 128, 0, h->d_route, r);
+    return MPE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch,
+                int64_t total_indices, float* d_out, void* cuda_stream) {
+    if (!h || !d_offsets || batch < 0 || total_indices < 0 || total_indices > 0x7ffffff0LL) return MPE_ERR_ARG;
+    if ((total_indices > 0 && !d_indices) || (batch > 0 && !d_out)) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (stream != h->stream) { CK(h, cudaStreamSynchronize(h->stream)); h->stream = stream; }
+    return forward_impl(h, d_indices, d_offsets, batch, total_indices, d_out, nullptr);
+}
+
+int mpe_forward_routed(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch, int64_t total_indices,
+                       float* const* out_ptrs, int32_t n_ranks, int32_t tables_global, int32_t table_base, void* cuda_stream) {
+    if (!h || !d_offsets || batch < 0 || total_indices < 0 || total_indices > 0x7ffffff0LL) return MPE_ERR_ARG;
+    if (total_indices > 0 && !d_indices) return MPE_ERR_ARG;
+    int rc = check_route(h, reinterpret_cast<const void* const*>(out_ptrs), n_ranks, tables_global, table_base, batch);
+    if (rc != MPE_OK) return rc;
+    DeviceGuard guard(h->device);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (stream != h->stream) { CK(h, cudaStreamSynchronize(h->stream)); h->stream = stream; }
+    rc = send_route(h, reinterpret_cast<const void* const*>(out_ptrs), n_ranks, tables_global, table_base, batch);
+    if (rc != MPE_OK) return rc;
+    return forward_impl(h, d_indices, d_offsets, batch, total_indices, nullptr, h->d_route);
+}
+
+int mpe_gather_grad(mpe_handle* h, const float* const* grad_ptrs, int32_t n_ranks, int32_t tables_global, int32_t table_base,
+                    int32_t batch, float* d_grad_local, void* cuda_stream) {
+    if (!h || (batch > 0 && !d_grad_local) || (reinterpret_cast<uintptr_t>(d_grad_local) & 15)) return MPE_ERR_ARG;
+    int rc = check_route(h, reinterpret_cast<const void* const*>(grad_ptrs), n_ranks, tables_global, table_base, batch);
+    if (rc != MPE_OK) return rc;
+    DeviceGuard guard(h->device);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (stream != h->stream) { CK(h, cudaStreamSynchronize(h->stream)); h->stream = stream; }
+    rc = send_route(h, reinterpret_cast<const void* const*>(grad_ptrs), n_ranks, tables_global, table_base, batch);
+    if (rc != MPE_OK) return rc;
+    const int64_t total4 = (int64_t)batch * h->T * h->dim / 4;
+    if (total4 > 0)
+        LAUNCH(h, "gather_grad", k_gather_grad, grid_for(h, total4, 256, 8), 256, 0, (const Route*)h->d_route, d_grad_local,
+               (int64_t)batch, h->T, h->dim);
+    return check_launch(h);
+}
+
+int mpe_peer_buffer_alloc(int32_t device, int64_t bytes, void** d_ptr, void* ipc_handle) {
+    if (!d_ptr || !ipc_handle || bytes <= 0) return MPE_ERR_ARG;
+    static_assert(sizeof(cudaIpcMemHandle_t) == MPE_IPC_HANDLE_BYTES, "handle size");
+    DeviceGuard guard(device);
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, (size_t)bytes);
+    if (e != cudaSuccess) return e == cudaErrorMemoryAllocation ? MPE_ERR_NOMEM : MPE_ERR_CUDA;
+    cudaIpcMemHandle_t hd;
+    e = cudaIpcGetMemHandle(&hd, p);
+    if (e != cudaSuccess) { cudaFree(p); return MPE_ERR_CUDA; }
+    std::memcpy(ipc_handle, &hd, sizeof(hd));
+    *d_ptr = p;
+    return MPE_OK;
+}
+
+int mpe_peer_buffer_open(int32_t device, const void* ipc_handle, void** d_ptr) {
+    if (!d_ptr || !ipc_handle) return MPE_ERR_ARG;
+    DeviceGuard guard(device);
+    cudaIpcMemHandle_t hd;
+    std::memcpy(&hd, ipc_handle, sizeof(hd));
+    void* p = nullptr;
+    if (cudaIpcOpenMemHandle(&p, hd, cudaIpcMemLazyEnablePeerAccess) != cudaSuccess) return MPE_ERR_CUDA;
+    *d_ptr = p;
+    return MPE_OK;
+}
+
+int mpe_peer_buffer_close(int32_t device, void* d_ptr) {
+    if (!d_ptr) return MPE_ERR_ARG;
+    DeviceGuard guard(device);
+    return cudaIpcCloseMemHandle(d_ptr) == cudaSuccess ? MPE_OK : MPE_ERR_CUDA;
+}
+
+int mpe_peer_buffer_free(int32_t device, void* d_ptr) {
+    if (!d_ptr) return MPE_ERR_ARG;
+    DeviceGuard guard(device);
+    return cudaFree(d_ptr) == cudaSuccess ? MPE_OK : MPE_ERR_CUDA;
 }
 
 int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step) {
@@ -663,6 +758,7 @@ int mpe_destroy(mpe_handle* h) {
     free_workspace(h);
     State& s = h->st;
     if (h->table_on_host) { cudaFreeHost(s.codes); cudaFreeHost(s.sb); } else { cudaFree(s.codes); cudaFree(s.sb); }
+    cudaFree(h->d_route);
     cudaFree(h->d_tables); cudaFree(s.cnt); cudaFree(s.G); cudaFree(s.slab);
     cudaFree(s.tags); cudaFree(s.ts); cudaFree(s.hit_epoch); cudaFree(s.hit_k); cudaFree(s.stats);
     cudaFree(h->sh_idx); cudaFree(h->sh_off); cudaFree(h->sh_grad); cudaFree(h->sh_out);

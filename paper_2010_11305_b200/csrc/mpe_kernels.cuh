@@ -56,10 +56,19 @@ struct State {
 
 // What changes from call to call.  It lives in device memory so that a captured CUDA graph of the step stays valid:
 // the kernels read it, one tiny kernel at the head of the graph writes it.
+// Destination of the pooled vectors when the tables are partitioned over several GPUs (Section 1: model parallelism
+// with no replication): sample b belongs to rank b / B_local, whose buffer is [B_local][T_global * dim].
+constexpr int MAX_RANKS = 72;
+struct Route {
+    float* out[MAX_RANKS];
+    int32_t B_local, T_global, t_base, n_ranks;
+};
+
 struct StepArgs {
     const int32_t* indices; const int32_t* offsets; float* out; const float* grad;
     int32_t B; uint32_t L; uint32_t epoch; float lr;
     unsigned long long step;
+    const Route* route;      // null: out is one [B][T * dim] array on this GPU
 };
 
 struct Work {
@@ -82,8 +91,12 @@ struct Work {
 // step prologue
 // ---------------------------------------------------------------------------------------------
 __global__ void k_set_args_forward(StepArgs* a, const int32_t* indices, const int32_t* offsets, float* out, int32_t B, uint32_t L,
-                                   uint32_t epoch) {
-    a->indices = indices; a->offsets = offsets; a->out = out; a->B = B; a->L = L; a->epoch = epoch;
+                                   uint32_t epoch, const Route* route) {
+    a->indices = indices; a->offsets = offsets; a->out = out; a->B = B; a->L = L; a->epoch = epoch; a->route = route;
+}
+__global__ void k_set_route(Route* dst, Route r) {
+    for (int g = threadIdx.x; g < MAX_RANKS; g += blockDim.x) dst->out[g] = r.out[g];
+    if (threadIdx.x == 0) { dst->B_local = r.B_local; dst->T_global = r.T_global; dst->t_base = r.t_base; dst->n_ranks = r.n_ranks; }
 }
 __global__ void k_set_args_backward(StepArgs* a, const float* grad, float lr, unsigned long long step) {
     a->grad = grad; a->lr = lr; a->step = step;
@@ -415,7 +428,13 @@ k_pool(State s, Work w, StepArgs av) {
                 }
             }
         }
-        reinterpret_cast<float4*>(out + (b * s.T + t) * dim)[sub] = acc;
+        float* dst = out + (b * s.T + t) * dim;
+        if (a.route) {                                // the owner of sample b gets the vector, straight into its buffer
+            const Route* __restrict__ r = a.route;
+            const int g = (int)(b / r->B_local);
+            dst = r->out[g] + ((b - (int64_t)g * r->B_local) * r->T_global + r->t_base + t) * dim;
+        }
+        reinterpret_cast<float4*>(dst)[sub] = acc;
         b += ng;
         while (b >= B) { b -= B; ++t; }
     }
@@ -1020,6 +1039,20 @@ __global__ void k_gather_rows(State s, int t, const int64_t* __restrict__ rows, 
         }
         if (cnt) cnt[i] = s.cnt ? s.cnt[g] : 0u;
         if (G) G[i] = s.G ? s.G[g] : 0.0f;
+    }
+}
+
+// The reverse exchange before backward: this rank's columns of every rank's [B_local][T_global * dim] gradient buffer are
+// pulled into one local [B][T * dim] array (plain loads from the owners' memory, 16 bytes per thread).
+__global__ void __launch_bounds__(256)
+k_gather_grad(const Route* __restrict__ r, float* __restrict__ dst, int64_t B, int T, int dim) {
+    const int64_t row4 = (int64_t)T * dim / 4;
+    const int64_t total = B * row4;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t b = i / row4, c = i - b * row4;
+        const int g = (int)(b / r->B_local);
+        const float4* src = reinterpret_cast<const float4*>(r->out[g] + ((b - (int64_t)g * r->B_local) * r->T_global + r->t_base) * dim);
+        reinterpret_cast<float4*>(dst)[i] = src[c];
     }
 }
 

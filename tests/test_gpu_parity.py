@@ -38,6 +38,18 @@ def test_config2_lfu_many_tables():
     run_parity(cfg, 12, check_every=4)
 
 
+def test_config2_with_the_table_sizes_the_paper_prints():
+    """Configuration 2 on the 26 row counts of the paper's Table 1 (tables of 3 rows up to 10 M rows, some smaller than one cache set)."""
+    import os
+    from dataclasses import replace
+    from parity_util import run_parity
+    path = os.path.join(os.path.dirname(__file__), "golden", "kaggle_table_sizes.txt")
+    sizes = [int(x) for l in open(path) if not l.startswith("#") for x in l.split()]
+    base = wl.config(2)
+    cfg = replace(base, name="cfg2b", num_rows=sizes, zipf=[base.zipf[0]] * len(sizes))
+    run_parity(cfg, 8, check_every=4)
+
+
 @pytest.mark.parametrize("bits,policy,opt,ways,dim", [
     (8, wl.LRU, wl.SGD, 8, 16), (4, wl.LRU, wl.ROWWISE_ADAGRAD, 16, 64), (4, wl.LFU, wl.SGD, 32, 128),
     (8, wl.LFU, wl.ROWWISE_ADAGRAD, 32, 64), (4, wl.LFU, wl.SGD, 2, 32), (8, wl.LRU, wl.SGD, 1, 8),
