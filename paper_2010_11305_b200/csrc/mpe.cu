@@ -428,12 +428,6 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
         constexpr int BITS = decltype(bc)::value, LANES = decltype(lc)::value;
         auto upd = ind ? k_update<BITS, LANES, true> : k_update<BITS, LANES, false>;
         auto lst = ind ? k_update_list<BITS, LANES, true> : k_update_list<BITS, LANES, false>;
-        static bool smem_set = false;     // one flag per instantiation of this lambda
-        if (!smem_set) {
-            cudaFuncSetAttribute(k_update<BITS, LANES, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, UPD_SMEM);
-            cudaFuncSetAttribute(k_update<BITS, LANES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, UPD_SMEM);
-            smem_set = true;
-        }
         LAUNCH(h, "update", upd, gu, UPD_WARPS * 32, UPD_SMEM, s, w, av);
         cudaStreamWaitEvent(h->stream, h->ev_join, 0);
         LAUNCH(h, "update_hot", lst, gh, 256, 0, s, w, (const int32_t*)w.hot_k, (const uint32_t*)&w.ctr->hot_rows, 0, av);

@@ -70,6 +70,30 @@ __device__ __forceinline__ void store_codes4(uint8_t* codes, int64_t grow, int d
     else row[sub] = (uint8_t)q;
 }
 
+// Element-wise IEEE additions / fused multiply-adds, two FP32 values per instruction (the packed f32x2 forms of sm_100):
+// every component is rounded to nearest exactly as the scalar instruction would round it.
+__device__ __forceinline__ float4 add4(float4 a, float4 b) {
+    return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
+}
+__device__ __forceinline__ float4 add4p(float4 a, float4 b) {
+    const float2 lo = __fadd2_rn(make_float2(a.x, a.y), make_float2(b.x, b.y));
+    const float2 hi = __fadd2_rn(make_float2(a.z, a.w), make_float2(b.z, b.w));
+    return make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+__device__ __forceinline__ float4 fma4(float m, float4 g, float4 x) {       // m * g + x, fused, per component
+    const float2 mm = make_float2(m, m);
+    const float2 lo = __ffma2_rn(mm, make_float2(g.x, g.y), make_float2(x.x, x.y));
+    const float2 hi = __ffma2_rn(mm, make_float2(g.z, g.w), make_float2(x.z, x.w));
+    return make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+// minimum / maximum over the lanes of `mask` in one instruction (floating-point warp reduction of sm_100a)
+__device__ __forceinline__ float group_min(float v, uint32_t mask) {
+    float r; asm volatile("redux.sync.min.f32 %0, %1, %2;" : "=f"(r) : "f"(v), "r"(mask)); return r;
+}
+__device__ __forceinline__ float group_max(float v, uint32_t mask) {
+    float r; asm volatile("redux.sync.max.f32 %0, %1, %2;" : "=f"(r) : "f"(v), "r"(mask)); return r;
+}
+
 // four stored values -> FP32: q*scale + bias for integer codes (Algorithm 1, up-conversion), exact for FP16
 template <int BITS>
 __device__ __forceinline__ float4 decode4(uint2 qq, float2 p) {
@@ -83,11 +107,11 @@ __device__ __forceinline__ float4 decode4(uint2 qq, float2 p) {
     }
     constexpr uint32_t M = (1u << (BITS & 15)) - 1u;
     const uint32_t q = qq.x;
-    x.x = __fmaf_rn(__uint2float_rn(q & M), p.x, p.y);
-    x.y = __fmaf_rn(__uint2float_rn((q >> (BITS & 15)) & M), p.x, p.y);
-    x.z = __fmaf_rn(__uint2float_rn((q >> ((2 * BITS) & 31)) & M), p.x, p.y);
-    x.w = __fmaf_rn(__uint2float_rn((q >> ((3 * BITS) & 31)) & M), p.x, p.y);
-    return x;
+    x.x = __uint2float_rn(q & M);
+    x.y = __uint2float_rn((q >> (BITS & 15)) & M);
+    x.z = __uint2float_rn((q >> ((2 * BITS) & 31)) & M);
+    x.w = __uint2float_rn((q >> ((3 * BITS) & 31)) & M);
+    return fma4(p.x, x, make_float4(p.y, p.y, p.y, p.y));      // q * s + b
 }
 
 // RO = the table is not written by the running kernel, so the read-only data path may serve the loads
@@ -98,21 +122,37 @@ __device__ __forceinline__ float4 dequant4(const uint8_t* codes, const float2* s
     return decode4<BITS>(load_codes4<BITS, RO>(codes, grow, dim, sub), p);
 }
 
-__device__ __forceinline__ float4 add4(float4 a, float4 b) {
-    return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
+__device__ __forceinline__ float4 mul4(float4 a, float4 b) {
+    const float2 lo = __fmul2_rn(make_float2(a.x, a.y), make_float2(b.x, b.y));
+    const float2 hi = __fmul2_rn(make_float2(a.z, a.w), make_float2(b.z, b.w));
+    return make_float4(lo.x, lo.y, hi.x, hi.y);
 }
 
-// one value -> its code; `stochastic` picks the rounding of Section 3 "Rounding" (it is the same for a whole kernel)
-__device__ __forceinline__ uint32_t quant1(float x, float mn, float inv, float qmax, uint32_t key, uint32_t column, bool stochastic) {
-    float y = __fmul_rn(__fsub_rn(x, mn), inv);           // (x - b)/s as (x - b) * (1/s)
-    y = fminf(fmaxf(y, 0.0f), qmax);
+// four values -> their codes; `stochastic` picks the rounding of Section 3 "Rounding" (it is the same for a whole kernel)
+struct Codes4 { uint32_t q0, q1, q2, q3; };
+__device__ __forceinline__ Codes4 quant4(float4 x, float mn, float inv, float qmax, uint32_t key, uint32_t column, bool stochastic) {
+    // (x - b)/s as (x - b) * (1/s); x - b is formed as x + (-b), which rounds identically
+    float4 y = mul4(add4p(x, make_float4(-mn, -mn, -mn, -mn)), make_float4(inv, inv, inv, inv));
+    y.x = fminf(fmaxf(y.x, 0.0f), qmax); y.y = fminf(fmaxf(y.y, 0.0f), qmax);
+    y.z = fminf(fmaxf(y.z, 0.0f), qmax); y.w = fminf(fmaxf(y.w, 0.0f), qmax);
+    Codes4 q;
     if (stochastic) {
-        const float f = floorf(y);
-        const float p = __fsub_rn(y, f);                   // exact
-        const float u = uniform01(key, column);
-        return (uint32_t)f + (u < p ? 1u : 0u);            // x+ with probability p: expectation y
+        const float4 f = make_float4(floorf(y.x), floorf(y.y), floorf(y.z), floorf(y.w));
+        const float4 p = add4p(y, make_float4(-f.x, -f.y, -f.z, -f.w));          // y - floor(y), exact
+        float4 u;                                                                // 24 random bits each, scaled to [0, 1): exact
+        u.x = __uint2float_rn(mix32(key ^ (column * 0x9E3779B9U + 0x7F4A7C15U)) >> 8);
+        u.y = __uint2float_rn(mix32(key ^ ((column + 1u) * 0x9E3779B9U + 0x7F4A7C15U)) >> 8);
+        u.z = __uint2float_rn(mix32(key ^ ((column + 2u) * 0x9E3779B9U + 0x7F4A7C15U)) >> 8);
+        u.w = __uint2float_rn(mix32(key ^ ((column + 3u) * 0x9E3779B9U + 0x7F4A7C15U)) >> 8);
+        u = mul4(u, make_float4(0x1p-24f, 0x1p-24f, 0x1p-24f, 0x1p-24f));
+        q.q0 = (uint32_t)f.x + (u.x < p.x ? 1u : 0u);                            // x+ with probability p: expectation y
+        q.q1 = (uint32_t)f.y + (u.y < p.y ? 1u : 0u);
+        q.q2 = (uint32_t)f.z + (u.z < p.z ? 1u : 0u);
+        q.q3 = (uint32_t)f.w + (u.w < p.w ? 1u : 0u);
+    } else {                                                                     // nearest, ties to even
+        q.q0 = (uint32_t)rintf(y.x); q.q1 = (uint32_t)rintf(y.y); q.q2 = (uint32_t)rintf(y.z); q.q3 = (uint32_t)rintf(y.w);
     }
-    return (uint32_t)rintf(y);                             // nearest, ties to even
+    return q;
 }
 
 // one value -> FP16 bits: the nearer neighbour, or one of the two neighbours x- <= x <= x+ (one unit in the last
@@ -141,9 +181,9 @@ __device__ __forceinline__ void quantize_store(float4 x, uint8_t* __restrict__ c
     const uint32_t mask = group_mask(lanes_per_row);
     float mn = fminf(fminf(x.x, x.y), fminf(x.z, x.w));
     float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
-    for (int o = lanes_per_row >> 1; o > 0; o >>= 1) {
-        mn = fminf(mn, __shfl_xor_sync(mask, mn, o));
-        mx = fmaxf(mx, __shfl_xor_sync(mask, mx, o));
+    if (lanes_per_row > 1) {                               // which zero a tie between -0 and +0 yields does not matter below
+        mn = group_min(mn, mask);
+        mx = group_max(mx, mask);
     }
     mn = __fadd_rn(mn, 0.0f);                              // -0 -> +0
     const float qmax = (float)((1 << (BITS & 15)) - 1);
@@ -152,11 +192,8 @@ __device__ __forceinline__ void quantize_store(float4 x, uint8_t* __restrict__ c
     if (s >= 1.17549435e-38f) inv = __fdiv_rn(1.0f, s);
     if (inv == 0.0f) s = 0.0f;
     const uint32_t c = 4u * (uint32_t)sub;
-    const uint32_t q0 = quant1(x.x, mn, inv, qmax, key, c, stochastic);
-    const uint32_t q1 = quant1(x.y, mn, inv, qmax, key, c + 1, stochastic);
-    const uint32_t q2 = quant1(x.z, mn, inv, qmax, key, c + 2, stochastic);
-    const uint32_t q3 = quant1(x.w, mn, inv, qmax, key, c + 3, stochastic);
-    store_codes4<BITS>(codes, grow, dim, sub, q0, q1, q2, q3);
+    const Codes4 q = quant4(x, mn, inv, qmax, key, c, stochastic);
+    store_codes4<BITS>(codes, grow, dim, sub, q.q0, q.q1, q.q2, q.q3);
     if (sub == 0) sb[grow] = make_float2(s, mn);
 }
 

@@ -750,9 +750,7 @@ __device__ __forceinline__ void apply_update(const State& s, const TableDev& tb,
         if (sub == 0) s.G[grow] = Gn;
         mult = __fdiv_rn(lr, __fadd_rn(__fsqrt_rn(Gn), s.eps));
     }
-    float4 xn;
-    xn.x = __fmaf_rn(-mult, g.x, x.x); xn.y = __fmaf_rn(-mult, g.y, x.y);
-    xn.z = __fmaf_rn(-mult, g.z, x.z); xn.w = __fmaf_rn(-mult, g.w, x.w);
+    const float4 xn = fma4(-mult, g, x);
     if (floc >= 0) {
         float4* dst = reinterpret_cast<float4*>(s.slab + (int64_t)floc * dim) + sub;
         if (loc < 0 && victim >= 0)     // the row this newcomer displaces is down-converted and placed back in T
@@ -770,19 +768,18 @@ __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefe
 struct RawRow { float4 f; uint2 q; float2 sb; };
 
 constexpr int UPD_WARPS = 4;     // warps per block of k_update
-constexpr int UPD_RING = 8;      // gradient rows a group can have in shared memory
-constexpr int UPD_GROUPS = 2;    // copy groups a group keeps in flight (each up to 4 rows)
-constexpr int UPD_NB = 4;        // rows per copy group
-constexpr int UPD_META = 16;     // ints of bookkeeping per staged row
-constexpr int UPD_SMEM = UPD_WARPS * (UPD_RING * 32 * 16 + 32 * UPD_META * 4);
+constexpr int UPD_NB = 4;        // gradient rows per batch of asynchronous copies
+constexpr int UPD_DEPTH = 2;     // batches in flight per group
+constexpr int UPD_SMEM = UPD_WARPS * (UPD_DEPTH * UPD_NB * 32 * 16 + 32 * 3 * 16);
 
-// Every distinct row with at most HOT_SPAN occurrences, except newcomers that wait for a write-back.
-// A warp stages the bookkeeping of 32 consecutive rows in shared memory, one row per lane (coalesced
-// loads; the per-row scalar work -- addresses, the stochastic-rounding key -- is done there once, 32
-// rows at a time).  Each group of LANES lanes then streams through the gradient rows of its rows:
-// asynchronous 16-byte copies bring up to UPD_GROUPS x UPD_NB gradient rows into a shared-memory ring
-// while earlier ones are being added (in index order, radix-32 tree), independent of where one
-// embedding row ends and the next begins.
+// Every distinct row with at most HOT_MIN occurrences, except newcomers that wait for a write-back.  A warp stages the
+// bookkeeping of 32 consecutive rows in shared memory, one row per lane (coalesced loads; the per-row scalar work --
+// addresses, the stochastic-rounding key -- is done there once, 32 rows at a time).  The distinct rows of a block are
+// consecutive in the sorted batch, so the gradient rows they need are one contiguous run of the sorted occurrence list
+// (broken only where a row is not this kernel's, or where the table changes).  Each group of LANES lanes walks such a
+// run four occurrences at a time: a batch of asynchronous 16-byte copies brings four gradient rows into shared memory
+// while the batch before it is added, and a row is finished (FP32 update, commit) the moment its last term has been added.
+
 template <int BITS, int LANES, bool IND>
 __global__ void __launch_bounds__(UPD_WARPS * 32, 8)
 k_update(State s, Work w, StepArgs av) {
@@ -792,16 +789,19 @@ k_update(State s, Work w, StepArgs av) {
     const float* __restrict__ grad = a.grad;
     const float lr = a.lr;
     const uint64_t step = a.step;
-    constexpr int dim = 4 * LANES, G = 32 / LANES, NB = LANES < UPD_NB ? LANES : UPD_NB;
-    enum { M_LOC, M_FLOC, M_COL, M_ROW, M_FIRST, M_CNT, M_SKIP, M_VICTIM, M_KEY, M_VKEY, M_GROW_LO, M_GROW_HI, M_VROW_LO, M_VROW_HI };
+    constexpr int dim = 4 * LANES, G = 32 / LANES, RPG = LANES, NB = LANES < UPD_NB ? LANES : UPD_NB, BPW = LANES / NB;
+    constexpr int SLOTS = UPD_DEPTH * NB;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int sub = lane & (LANES - 1), grp = lane / LANES, gbase = lane & ~(LANES - 1);
     const uint32_t gmask = group_mask(LANES);
-    float4* ring = reinterpret_cast<float4*>(upd_smem) + ((warp * G + grp) * UPD_RING) * LANES + sub;   // slot i: ring[i * LANES]
-    int32_t(*meta)[UPD_META] = reinterpret_cast<int32_t(*)[UPD_META]>(upd_smem + UPD_WARPS * UPD_RING * 32 * 16) + warp * 32;
+    float4* ring = reinterpret_cast<float4*>(upd_smem) + ((warp * G + grp) * SLOTS) * LANES + sub;       // slot i: ring[i * LANES]
+    // per staged row: A = {loc, final loc, global row lo, hi}, B = {rounding key, occurrences, first occurrence, victim},
+    // C = {victim's key, victim's global row lo, hi, gradient column}
+    int4* recs = reinterpret_cast<int4*>(upd_smem + UPD_WARPS * UPD_DEPTH * UPD_NB * 32 * 16) + warp * 96;
     const int64_t U = w.ctr->U;
     const uint32_t stride_bytes = (uint32_t)s.T * (uint32_t)dim * 4u;
     const char* gcol = reinterpret_cast<const char*>(grad + 4 * sub);
+    const float NZ = __int_as_float(0x80000000);          // -0: adding it changes no value, not even a zero's sign
     for (;;) {
         // blocks of 32 rows are handed out on demand: their cost varies with the rows' multiplicities
         uint32_t blk = 0;
@@ -809,21 +809,20 @@ k_update(State s, Work w, StepArgs av) {
         const int64_t k0 = (int64_t)__shfl_sync(0xffffffffU, blk, 0) * 32;
         if (k0 >= U) break;
         const int64_t k = k0 + lane;
+        bool skip = true; int myt = -1;
         if (k < U) {
             const int32_t first = w.seg[k], row = w.uniq_row[k];
             const int loc = w.loc[k], floc = w.final_loc[k], hb = w.hot_base[k], victim = w.victim[k], t = w.uniq_t[k];
-            int32_t* mrow = meta[lane];
-            mrow[M_LOC] = loc; mrow[M_FLOC] = floc; mrow[M_COL] = t * dim; mrow[M_ROW] = row;
-            mrow[M_FIRST] = first; mrow[M_CNT] = w.seg[k + 1] - first; mrow[M_VICTIM] = victim;
+            myt = t;
             // pseudo rows, hot rows (own kernel) and newcomers that wait for a write-back are not ours
             const bool newcomer = loc < 0 && floc >= 0;
-            const bool skip = loc == LOC_INVALID || hb >= 0 || (newcomer && victim == VICTIM_DEFER);
-            mrow[M_SKIP] = skip ? 1 : 0;
+            skip = loc == LOC_INVALID || hb >= 0 || (newcomer && victim == VICTIM_DEFER);
+            int4 A = make_int4(loc, floc, 0, 0), Bq = make_int4(0, w.seg[k + 1] - first, first, victim), C = make_int4(0, 0, 0, t * dim);
             if (!skip) {
                 const int64_t rb = s.tables[t].row_base;
                 const int64_t grow = rb + row;
-                mrow[M_GROW_LO] = (int32_t)(uint32_t)grow; mrow[M_GROW_HI] = (int32_t)(grow >> 32);
-                mrow[M_KEY] = (int32_t)rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)row, step);
+                A.z = (int32_t)(uint32_t)grow; A.w = (int32_t)(grow >> 32);
+                Bq.x = (int32_t)rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)row, step);
                 // pull this row's current value towards L2 now; it is needed when its gradient has been summed
                 if (loc >= 0) {
                     const char* src = reinterpret_cast<const char*>(s.slab + (int64_t)loc * dim);
@@ -835,111 +834,116 @@ k_update(State s, Work w, StepArgs av) {
                 }
                 if (newcomer && victim >= 0) {
                     const int64_t vrow = rb + victim;
-                    mrow[M_VROW_LO] = (int32_t)(uint32_t)vrow; mrow[M_VROW_HI] = (int32_t)(vrow >> 32);
-                    mrow[M_VKEY] = (int32_t)rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)victim, step);
+                    C.x = (int32_t)rowkey(s.seed, DOMAIN_SR, (uint32_t)t, (uint32_t)victim, step);
+                    C.y = (int32_t)(uint32_t)vrow; C.z = (int32_t)(vrow >> 32);
                     const char* src = reinterpret_cast<const char*>(s.slab + (int64_t)floc * dim);
 #pragma unroll
                     for (int o = 0; o < dim * 4; o += 128) prefetch_l2(src + o);
                 }
             }
+            recs[lane * 3] = A; recs[lane * 3 + 1] = Bq; recs[lane * 3 + 2] = C;
         }
+        const int tprev = __shfl_up_sync(0xffffffffU, myt, 1);
+        const uint32_t skipmask = __ballot_sync(0xffffffffU, skip);                       // rows that are not ours (or past the end)
+        const uint32_t stopmask = skipmask | __ballot_sync(0xffffffffU, lane > 0 && myt != tprev);   // a run ends before these rows
         __syncwarp();
-        const int nrow = (int)min((int64_t)32, U - k0);
-        {   // and the sample ids of the warp's occurrences (one contiguous range of the sorted batch)
-            const int32_t o0 = meta[0][M_FIRST], o1 = meta[nrow - 1][M_FIRST] + meta[nrow - 1][M_CNT];
-            for (int32_t o = o0 + 32 * lane; o < o1 && o < o0 + 4096; o += 1024) prefetch_l2(w.occ_b + o);
-        }
-        auto valid_from = [&](int r) { while (r < nrow && meta[r][M_SKIP]) r += G; return r; };
-        int pr = valid_from(grp), po = 0;          // producer: next gradient row to request
-        int cr = pr, co = 0;                        // consumer: next gradient row to add
-        int head = 0, tail = 0, inflight = 0;
-        int ncnt = 0; int32_t nb = 0;               // the next copy group: how many rows, and their sample ids (one per lane)
-        auto describe_next = [&]() {
-            if (pr < nrow) {
-                ncnt = min(NB, meta[pr][M_CNT] - po);
-                nb = sub < ncnt ? w.occ_b[meta[pr][M_FIRST] + po + sub] : 0;
-            }
-        };
-        describe_next();
-        RawRow xr;
-        auto load_x = [&]() {
-            const int loc = meta[cr][M_LOC];
-            if (loc >= 0) {
-                xr.f = reinterpret_cast<const float4*>(s.slab + (int64_t)loc * dim)[sub];
-            } else {
-                const int64_t grow = ((int64_t)meta[cr][M_GROW_HI] << 32) | (uint32_t)meta[cr][M_GROW_LO];
-                if (BITS != 16) xr.sb = s.sb[grow];
-                xr.q = load_codes4<BITS, false>(s.codes, grow, dim, sub);
-            }
-        };
-        if (cr < nrow) load_x();
-        float4 chunkacc = make_float4(0.f, 0.f, 0.f, 0.f), rowacc = chunkacc;
-        while (cr < nrow) {
-            while (inflight < UPD_GROUPS && pr < nrow) {
-                const char* src = gcol + (size_t)(uint32_t)meta[pr][M_COL] * 4u;
+        // this group's rows: RPG consecutive ones; their runs
+        const int gr0 = grp * RPG, gr1 = gr0 + RPG;
+        uint32_t avail = ~skipmask & (RPG == 32 ? 0xffffffffU : (((1U << RPG) - 1U) << gr0));
+        while (avail) {
+            const int rs = __ffs(avail) - 1;
+            const uint32_t above = stopmask & (rs == 31 ? 0u : (0xfffffffeU << rs));
+            int re = above ? __ffs(above) - 1 : 32;
+            re = min(re, gr1);
+            avail = re >= 32 ? 0u : (avail & (0xffffffffU << re));
+            // the run's occurrences and gradient column
+            const int4 Bs = recs[rs * 3 + 1], Be = recs[(re - 1) * 3 + 1];
+            const int32_t os = Bs.z, oe = Be.z + Be.y;
+            const char* src = gcol + (size_t)(uint32_t)recs[rs * 3 + 2].w * 4u;
+            const int nbatch = (oe - os + NB - 1) / NB;
+            uint32_t wb = 0;                                   // sample ids of LANES consecutive occurrences, one per lane
+            auto issue = [&](int j) {                          // copies of batch j (none when j is past the end); always one group
+                if (j < nbatch) {
+                    const int jw = j % BPW;
+                    if (jw == 0) { const int32_t o = os + j * NB + sub; wb = o < oe ? (uint32_t)w.occ_b[o] : 0u; }
+                    const int32_t left = oe - (os + j * NB);
+                    float4* dst = ring + ((j % UPD_DEPTH) * NB) * LANES;
 #pragma unroll
-                for (int u = 0; u < NB; ++u) {
-                    const uint32_t b = (uint32_t)__shfl_sync(gmask, nb, gbase + u);
-                    if (u < ncnt) cp_async16(ring + ((head + u) & (UPD_RING - 1)) * LANES, src + (size_t)b * stride_bytes);
+                    for (int u = 0; u < NB; ++u) {
+                        const uint32_t b = __shfl_sync(gmask, wb, gbase + jw * NB + u);
+                        if (u < left) cp_async16(dst + u * LANES, src + (size_t)b * stride_bytes);
+                    }
                 }
                 cp_async_commit();
-                head += ncnt; ++inflight; po += ncnt;
-                if (po == meta[pr][M_CNT]) { pr = valid_from(pr + G); po = 0; }
-                describe_next();
-            }
-            switch (inflight) {                     // the oldest group has landed when at most inflight-1 are pending
-                case 1: cp_async_wait<0>(); break;
-                case 2: cp_async_wait<1>(); break;
-                case 3: cp_async_wait<2>(); break;
-                default: cp_async_wait<3>(); break;
-            }
-            const int m = meta[cr][M_CNT];
-            const int cnt = min(NB, m - co);
-            // a copy group never straddles a chunk of 32 terms: add its rows left to right ...
-            float4 acc = ring[(tail & (UPD_RING - 1)) * LANES];
-            if (co & 31) acc = add4(chunkacc, acc);
-#pragma unroll
-            for (int u = 1; u < NB; ++u)
-                if (u < cnt) acc = add4(acc, ring[((tail + u) & (UPD_RING - 1)) * LANES]);
-            chunkacc = acc;
-            tail += cnt; co += cnt; --inflight;
-            // ... and fold a finished chunk into the sum of chunk sums
-            if ((co & 31) == 0 || co == m) rowacc = co <= 32 ? chunkacc : add4(rowacc, chunkacc);
-            if (co == m) {
-                const int32_t* mc = meta[cr];
-                const int loc = mc[M_LOC], floc = mc[M_FLOC];
-                float4 x = xr.f;
-                if (loc < 0) x = decode4<BITS>(xr.q, xr.sb);
-                const int64_t grow = ((int64_t)mc[M_GROW_HI] << 32) | (uint32_t)mc[M_GROW_LO];
-                float mult = lr;                                         // SGD: x <- x - lr * g
-                if (s.optimizer == 1) {                                  // row-wise Adagrad
-                    float a = __fmul_rn(rowacc.x, rowacc.x);
-                    a = __fmaf_rn(rowacc.y, rowacc.y, a); a = __fmaf_rn(rowacc.z, rowacc.z, a); a = __fmaf_rn(rowacc.w, rowacc.w, a);
-#pragma unroll
-                    for (int o = LANES >> 1; o > 0; o >>= 1) a = __fadd_rn(a, __shfl_xor_sync(gmask, a, o));
-                    const float Gold = s.G[grow];
-                    __syncwarp(gmask);                                   // every lane has read G before lane 0 replaces it
-                    const float Gn = __fadd_rn(Gold, __fmul_rn(a, __fdiv_rn(1.0f, (float)dim)));
-                    if (sub == 0) s.G[grow] = Gn;
-                    mult = __fdiv_rn(lr, __fadd_rn(__fsqrt_rn(Gn), s.eps));
-                }
-                float4 xn;
-                xn.x = __fmaf_rn(-mult, rowacc.x, x.x); xn.y = __fmaf_rn(-mult, rowacc.y, x.y);
-                xn.z = __fmaf_rn(-mult, rowacc.z, x.z); xn.w = __fmaf_rn(-mult, rowacc.w, x.w);
-                if (floc >= 0) {
-                    float4* dst = reinterpret_cast<float4*>(s.slab + (int64_t)floc * dim) + sub;
-                    if (loc < 0 && mc[M_VICTIM] >= 0) {  // the row this newcomer displaces is down-converted and placed back in T
-                        const int64_t vrow = ((int64_t)mc[M_VROW_HI] << 32) | (uint32_t)mc[M_VROW_LO];
-                        quantize_store<BITS>(*dst, s.codes, s.sb, vrow, dim, sub, LANES, (uint32_t)mc[M_VKEY], s.rounding != 0);
-                    }
-                    *dst = xn;                           // cached rows keep full precision, a newcomer enters verbatim
+            };
+            // current row: its records, its stored value, how many terms are still to come
+            int r = rs;
+            int4 A, Bq; RawRow xr; int rem = 0;
+            auto open_row = [&]() {
+                A = recs[r * 3]; Bq = recs[r * 3 + 1]; rem = Bq.y;
+                if (A.x >= 0) {
+                    xr.f = reinterpret_cast<const float4*>(s.slab + (int64_t)A.x * dim)[sub];
                 } else {
-                    quantize_store<BITS>(xn, s.codes, s.sb, grow, dim, sub, LANES, (uint32_t)mc[M_KEY], s.rounding != 0);
+                    const int64_t grow = ((int64_t)A.w << 32) | (uint32_t)A.z;
+                    if (BITS != 16) xr.sb = s.sb[grow];
+                    xr.q = load_codes4<BITS, false>(s.codes, grow, dim, sub);
                 }
-                cr = valid_from(cr + G); co = 0;
-                if (cr < nrow) load_x();
+            };
+            open_row();
+#pragma unroll
+            for (int j = 0; j < UPD_DEPTH; ++j) issue(j);
+            float4 chunkacc = make_float4(NZ, NZ, NZ, NZ), rowacc = chunkacc;
+            int c = 0;                                         // terms in the current chunk of 32
+            for (int j = 0; j < nbatch; ++j) {
+                cp_async_wait<UPD_DEPTH - 1>();               // batch j has landed
+                const int cnt = min(NB, oe - (os + j * NB));
+                const float4* slot = ring + ((j % UPD_DEPTH) * NB) * LANES;
+#pragma unroll 1
+                for (int u = 0; u < cnt; ++u) {
+                    chunkacc = add4(chunkacc, slot[u * LANES]);
+                    ++c; --rem;
+                    if (c == 32 || rem == 0) {                 // a finished chunk joins the sum of chunk sums
+                        rowacc = add4(rowacc, chunkacc);
+                        chunkacc = make_float4(NZ, NZ, NZ, NZ); c = 0;
+                    }
+                    if (rem == 0) {
+                        const int loc = A.x, floc = A.y;
+                        float4 x = xr.f;
+                        if (loc < 0) x = decode4<BITS>(xr.q, xr.sb);
+                        const int64_t grow = ((int64_t)A.w << 32) | (uint32_t)A.z;
+                        float mult = lr;                                         // SGD: x <- x - lr * g
+                        if (s.optimizer == 1) {                                  // row-wise Adagrad
+                            float q = __fmul_rn(rowacc.x, rowacc.x);
+                            q = __fmaf_rn(rowacc.y, rowacc.y, q); q = __fmaf_rn(rowacc.z, rowacc.z, q); q = __fmaf_rn(rowacc.w, rowacc.w, q);
+#pragma unroll
+                            for (int o = LANES >> 1; o > 0; o >>= 1) q = __fadd_rn(q, __shfl_xor_sync(gmask, q, o));
+                            const float Gold = s.G[grow];
+                            __syncwarp(gmask);                                   // every lane has read G before lane 0 replaces it
+                            const float Gn = __fadd_rn(Gold, __fmul_rn(q, __fdiv_rn(1.0f, (float)dim)));
+                            if (sub == 0) s.G[grow] = Gn;
+                            mult = __fdiv_rn(lr, __fadd_rn(__fsqrt_rn(Gn), s.eps));
+                        }
+                        const float4 xn = fma4(-mult, rowacc, x);
+                        if (floc >= 0) {
+                            float4* dst = reinterpret_cast<float4*>(s.slab + (int64_t)floc * dim) + sub;
+                            if (loc < 0 && Bq.w >= 0) {          // the row this newcomer displaces is down-converted and placed back in T
+                                const int4 C = recs[r * 3 + 2];
+                                const int64_t vrow = ((int64_t)C.z << 32) | (uint32_t)C.y;
+                                quantize_store<BITS>(*dst, s.codes, s.sb, vrow, dim, sub, LANES, (uint32_t)C.x, s.rounding != 0);
+                            }
+                            *dst = xn;                           // cached rows keep full precision, a newcomer enters verbatim
+                        } else {
+                            quantize_store<BITS>(xn, s.codes, s.sb, grow, dim, sub, LANES, (uint32_t)Bq.x, s.rounding != 0);
+                        }
+                        rowacc = make_float4(NZ, NZ, NZ, NZ);
+                        if (++r < re) open_row();
+                    }
+                }
+                issue(j + UPD_DEPTH);
             }
+            cp_async_wait<0>();
         }
+        __syncwarp();                                          // the records are rewritten by the next block
     }
 }
 
