@@ -269,22 +269,32 @@ k_probe(State s, Work w, StepArgs av) {
             if (row >= tb.N) myloc = LOC_INVALID;
             else if (tb.n_sets > 0) { set = set_of((uint32_t)row, tb.salt, tb.n_sets); gset = (int32_t)(tb.set_base + set); }
         }
-#pragma unroll 4
-        for (int it = 0; it < ways; ++it) {            // 32 / G rounds
-            const int r = it * G + grp;               // the row this group looks at
-            const int32_t rgset = __shfl_sync(0xffffffffU, gset, r);
-            const int32_t rrow = __shfl_sync(0xffffffffU, row, r);
-            bool match = false;
-            int64_t slot = 0;
-            if (rgset >= 0) { slot = (int64_t)rgset * ways + way; match = s.tags[slot] == rrow; }
-            const uint32_t hit = __ballot_sync(0xffffffffU, match) & gmask;
-            int rloc = LOC_MISS;
-            if (hit) {
-                rloc = (int)((int64_t)rgset * ways + (__ffs(hit) - 1 - (lane & ~(ways - 1))));
-                if (match) { s.hit_epoch[slot] = epoch; s.hit_k[slot] = (int32_t)(k0 + r); }
+        // 32 / G rounds, eight at a time (eight tag loads in flight).  In round `it` group g looks at row it*G + g; every
+        // lane sees the whole ballot, and lane l keeps the one of the round that handled its own row (l / G).
+        uint32_t myhit = 0;
+        for (int it0 = 0; it0 < ways; it0 += 8) {
+            int32_t tg[8], rg[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int r = ((it0 + j) * G + grp) & 31;
+                rg[j] = __shfl_sync(0xffffffffU, gset, r);
+                tg[j] = -1;
+                if (it0 + j < ways && rg[j] >= 0) tg[j] = s.tags[(int64_t)rg[j] * ways + way];
             }
-            const int got = __shfl_sync(0xffffffffU, rloc, (lane % G) * ways);   // result of the group that handled my row
-            if (lane / G == it && gset >= 0) myloc = got;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int it = it0 + j;
+                const int r = (it * G + grp) & 31;
+                const int32_t rrow = __shfl_sync(0xffffffffU, row, r);
+                const bool match = it < ways && rg[j] >= 0 && tg[j] == rrow;
+                const uint32_t hit = __ballot_sync(0xffffffffU, match);
+                if (match) { const int64_t slot = (int64_t)rg[j] * ways + way; s.hit_epoch[slot] = epoch; s.hit_k[slot] = (int32_t)(k0 + r); }
+                if (lane / G == it) myhit = hit;
+            }
+        }
+        if (gset >= 0) {
+            const uint32_t mine = (myhit >> ((lane % G) * ways)) & (ways == 32 ? 0xffffffffU : ((1u << ways) - 1u));
+            if (mine) myloc = (int)((int64_t)gset * ways + (__ffs(mine) - 1));
         }
         if (k < U) {
             w.loc[k] = myloc; w.final_loc[k] = myloc; w.uset[k] = set;
