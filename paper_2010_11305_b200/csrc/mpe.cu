@@ -409,7 +409,7 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
     dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
         constexpr int LANES = decltype(lc)::value;
         auto hot = ind ? k_hot_partial<LANES, true> : k_hot_partial<LANES, false>;
-        LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, L / HOT_MIN + 1, 1, 1), 8 * LANES, 32 * s.dim * sizeof(float), s, w, av);
+        LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, L / HOT_MIN + 1, 1, 2), 8 * LANES, 32 * s.dim * sizeof(float), s, w, av);
     });
     CK(h, cudaEventRecord(h->ev_join, h->side));
     LAUNCH(h, "priority", (ind ? k_priority<true> : k_priority<false>), grid_for(h, L, 1024, 8), 256, 0, s, w, h->ckeyA, av);

@@ -202,6 +202,11 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
     const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
 }
+// same with the shared-memory address already converted; `take` false copies nothing (the source is not read)
+__device__ __forceinline__ void cp_async16_if(uint32_t smem_addr, const void* gsrc, bool take) {
+    const uint32_t n = take ? 16u : 0u;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr), "l"(gsrc), "r"(n) : "memory");
+}
 // same, but the line is also kept in L1 (rows that many bags of one SM share)
 __device__ __forceinline__ void cp_async16_l1(void* smem_dst, const void* gsrc) {
     const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);

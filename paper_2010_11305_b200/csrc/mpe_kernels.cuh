@@ -645,27 +645,30 @@ __device__ __forceinline__ float4 sum_chunk(const int32_t* __restrict__ occ_b, c
                                             int32_t first, int len, uint32_t gmask, int gbase, int sub) {
     constexpr int NB = LANES < 8 ? LANES : 8;
     float4 acc;
-    if (LANES == 32 && len == 32) {       // a full chunk handled by a whole warp: no bounds to check, 16 rows in flight
+    if (LANES == 32 && len == 32) {       // a full chunk handled by a whole warp: no bounds to check, 8 rows in flight
         const uint32_t myb = (uint32_t)occ_b[first + sub];
-        float4 va[8], vb[8];
+        float4 va[4], vb[4];
         auto row = [&](int u) { return __ldg(reinterpret_cast<const float4*>(gcol + (size_t)__shfl_sync(0xffffffffU, myb, u) * stride_bytes)); };
 #pragma unroll
-        for (int u = 0; u < 8; ++u) va[u] = row(u);
+        for (int u = 0; u < 4; ++u) va[u] = row(u);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) vb[u] = row(8 + u);
+        for (int u = 0; u < 4; ++u) vb[u] = row(4 + u);
         acc = va[0];
 #pragma unroll
-        for (int u = 1; u < 8; ++u) acc = add4(acc, va[u]);
+        for (int u = 1; u < 4; ++u) acc = add4(acc, va[u]);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) va[u] = row(16 + u);
+        for (int g = 1; g < 4; ++g) {
 #pragma unroll
-        for (int u = 0; u < 8; ++u) acc = add4(acc, vb[u]);
+            for (int u = 0; u < 4; ++u) va[u] = row(8 * g + u);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) vb[u] = row(24 + u);
+            for (int u = 0; u < 4; ++u) acc = add4(acc, vb[u]);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) acc = add4(acc, va[u]);
+            for (int u = 0; u < 4; ++u) vb[u] = row(8 * g + 4 + u);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) acc = add4(acc, vb[u]);
+            for (int u = 0; u < 4; ++u) acc = add4(acc, va[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) acc = add4(acc, vb[u]);
         return acc;
     }
     acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -707,7 +710,7 @@ __device__ __forceinline__ float4 tree_reduce(const Term& term, int64_t first, i
 // rows with more than HOT_SPAN occurrences: one block per HOT_SPAN occurrences computes two tree levels
 // (8 groups of LANES lanes share the 32 chunks of a task)
 template <int LANES, bool IND>
-__global__ void __launch_bounds__(8 * LANES)
+__global__ void __launch_bounds__(8 * LANES, LANES == 32 ? 3 : 1)
 k_hot_partial(State s, Work w, StepArgs av) {
     StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
     extern __shared__ float chunk_sums[];     // [32][dim]
@@ -805,6 +808,7 @@ k_update(State s, Work w, StepArgs av) {
     const int sub = lane & (LANES - 1), grp = lane / LANES, gbase = lane & ~(LANES - 1);
     const uint32_t gmask = group_mask(LANES);
     float4* ring = reinterpret_cast<float4*>(upd_smem) + ((warp * G + grp) * SLOTS) * LANES + sub;       // slot i: ring[i * LANES]
+    const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
     // per staged row: A = {loc, final loc, global row lo, hi}, B = {rounding key, occurrences, first occurrence, victim},
     // C = {victim's key, victim's global row lo, hi, gradient column}
     int4* recs = reinterpret_cast<int4*>(upd_smem + UPD_WARPS * UPD_DEPTH * UPD_NB * 32 * 16) + warp * 96;
@@ -877,11 +881,11 @@ k_update(State s, Work w, StepArgs av) {
                     const int jw = j % BPW;
                     if (jw == 0) { const int32_t o = os + j * NB + sub; wb = o < oe ? (uint32_t)w.occ_b[o] : 0u; }
                     const int32_t left = oe - (os + j * NB);
-                    float4* dst = ring + ((j % UPD_DEPTH) * NB) * LANES;
+                    const uint32_t dst = ring_s + (uint32_t)(((j % UPD_DEPTH) * NB) * LANES * 16);
 #pragma unroll
                     for (int u = 0; u < NB; ++u) {
-                        const uint32_t b = __shfl_sync(gmask, wb, gbase + jw * NB + u);
-                        if (u < left) cp_async16(dst + u * LANES, src + (size_t)b * stride_bytes);
+                        const uint32_t b = __shfl_sync(gmask, wb, gbase + jw * NB + u);          // 0 (a valid sample) past the end
+                        cp_async16_if(dst + (uint32_t)(u * LANES * 16), src + (size_t)b * stride_bytes, u < left);
                     }
                 }
                 cp_async_commit();
@@ -904,13 +908,15 @@ k_update(State s, Work w, StepArgs av) {
             for (int j = 0; j < UPD_DEPTH; ++j) issue(j);
             float4 chunkacc = make_float4(NZ, NZ, NZ, NZ), rowacc = chunkacc;
             int c = 0;                                         // terms in the current chunk of 32
-            for (int j = 0; j < nbatch; ++j) {
-                cp_async_wait<UPD_DEPTH - 1>();               // batch j has landed
-                const int cnt = min(NB, oe - (os + j * NB));
-                const float4* slot = ring + ((j % UPD_DEPTH) * NB) * LANES;
+            const int nocc = oe - os;
 #pragma unroll 1
-                for (int u = 0; u < cnt; ++u) {
-                    chunkacc = add4(chunkacc, slot[u * LANES]);
+            for (int jo = 0; jo < nocc; ++jo) {
+                if ((jo & (NB - 1)) == 0) {                    // a batch boundary: refill the slots just drained, then wait for this batch
+                    if (jo) issue(jo / NB - 1 + UPD_DEPTH);
+                    cp_async_wait<UPD_DEPTH - 1>();
+                }
+                {
+                    chunkacc = add4(chunkacc, ring[(jo & (SLOTS - 1)) * LANES]);
                     ++c; --rem;
                     if (c == 32 || rem == 0) {                 // a finished chunk joins the sum of chunk sums
                         rowacc = add4(rowacc, chunkacc);
@@ -949,7 +955,6 @@ k_update(State s, Work w, StepArgs av) {
                         if (++r < re) open_row();
                     }
                 }
-                issue(j + UPD_DEPTH);
             }
             cp_async_wait<0>();
         }

@@ -109,8 +109,7 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict_
                const uint32_t* __restrict__ hist_scanned) {
     constexpr int WARPS = SORT_THREADS / 32;
     __shared__ uint32_t wcnt[WARPS][256];      // per-warp digit counters, then per-warp digit bases
-    __shared__ uint32_t dstart[256];           // first tile-local position of each digit
-    __shared__ uint32_t gbase[256];            // first global position of each digit of this tile
+    __shared__ uint32_t gbase[256];            // first global position of each digit of this tile, later minus its tile-local start
     __shared__ uint32_t skey[SORT_TILE];
     __shared__ uint32_t sval[SORT_TILE];
     __shared__ uint32_t scan_tmp[SORT_THREADS / 32 + 1];
@@ -145,18 +144,20 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict_
         }
         __syncthreads();
         // digit d (= threadIdx.x): exclusive sum over warps, then over digits
-        uint32_t tot = 0;
+        uint32_t cw[WARPS], tot = 0;
 #pragma unroll
-        for (int w = 0; w < WARPS; ++w) { uint32_t c = wcnt[w][threadIdx.x]; wcnt[w][threadIdx.x] = tot; tot += c; }
+        for (int w = 0; w < WARPS; ++w) { cw[w] = tot; tot += wcnt[w][threadIdx.x]; }
         uint32_t all;
         const uint32_t ds = block_exclusive_scan<SORT_THREADS>(tot, &all, scan_tmp);
-        dstart[threadIdx.x] = ds;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) wcnt[w][threadIdx.x] = ds + cw[w];     // tile-local position of warp w's first key with this digit
+        gbase[threadIdx.x] -= ds;                                              // global position = gbase + tile-local position
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < SORT_ITEMS; ++i) {
             const int e = warp * (32 * SORT_ITEMS) + i * 32 + lane;
             const uint32_t dg = (key[i] >> shift) & 255u;
-            const uint32_t pos = dstart[dg] + wcnt[warp][dg] + rank[i];
+            const uint32_t pos = wcnt[warp][dg] + rank[i];
             skey[pos] = key[i];
             sval[pos] = e < count ? (vals_in ? vals_in[start + e] : (uint32_t)(start + e)) : 0u;
         }
@@ -165,7 +166,7 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict_
         for (int j = threadIdx.x; j < count; j += SORT_THREADS) {
             const uint32_t k = skey[j];
             const uint32_t dg = (k >> shift) & 255u;
-            const uint32_t dst = gbase[dg] + ((uint32_t)j - dstart[dg]);
+            const uint32_t dst = gbase[dg] + (uint32_t)j;
             keys_out[dst] = k;
             vals_out[dst] = sval[j];
         }
