@@ -328,6 +328,7 @@ int mpe_create_placed(mpe_handle** out, const mpe_table_spec* tables, int32_t nu
     if (policy == MPE_LRU && (rc = dmalloc(h, &s.ts, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
     if ((rc = dmalloc(h, &s.hit_epoch, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
     if ((rc = dmalloc(h, &s.hit_k, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
+    if ((rc = dmalloc(h, &s.floor, std::max<int64_t>(1, h->total_sets), nullptr)) != MPE_OK) return fail(rc);
     if ((rc = dmalloc(h, &s.stats, (int64_t)num_tables * 8, nullptr)) != MPE_OK) return fail(rc);
 #define CKC(expr) do { cudaError_t e_ = (expr); if (e_ != cudaSuccess) { h->last_cuda_error = (int)e_; return fail(MPE_ERR_CUDA); } } while (0)
     CKC(cudaMemcpy(h->d_tables, h->tables.data(), sizeof(TableDev) * num_tables, cudaMemcpyHostToDevice));
@@ -336,6 +337,7 @@ int mpe_create_placed(mpe_handle** out, const mpe_table_spec* tables, int32_t nu
     CKC(cudaMemset(s.slab, 0, sizeof(float) * std::max<int64_t>(1, h->total_slots * dim)));
     if (s.ts) CKC(cudaMemset(s.ts, 0, sizeof(uint32_t) * std::max<int64_t>(1, h->total_slots)));
     CKC(cudaMemset(s.hit_epoch, 0, sizeof(uint32_t) * std::max<int64_t>(1, h->total_slots)));
+    CKC(cudaMemset(s.floor, 0, sizeof(uint32_t) * std::max<int64_t>(1, h->total_sets)));
     CKC(cudaMemset(s.stats, 0, sizeof(unsigned long long) * 8 * num_tables));
     LAUNCH(h, "fill_tags", k_fill_i32, grid_for(h, h->total_slots, 256, 8), 256, 0, s.tags, h->total_slots, -1);
     for (int t = 0; t < num_tables; ++t) {
@@ -754,7 +756,7 @@ int mpe_destroy(mpe_handle* h) {
     if (h->table_on_host) { cudaFreeHost(s.codes); cudaFreeHost(s.sb); } else { cudaFree(s.codes); cudaFree(s.sb); }
     cudaFree(h->d_route);
     cudaFree(h->d_tables); cudaFree(s.cnt); cudaFree(s.G); cudaFree(s.slab);
-    cudaFree(s.tags); cudaFree(s.ts); cudaFree(s.hit_epoch); cudaFree(s.hit_k); cudaFree(s.stats);
+    cudaFree(s.tags); cudaFree(s.ts); cudaFree(s.hit_epoch); cudaFree(s.hit_k); cudaFree(s.floor); cudaFree(s.stats);
     cudaFree(h->sh_idx); cudaFree(h->sh_off); cudaFree(h->sh_grad); cudaFree(h->sh_out);
     for (auto& r : h->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto e : h->event_pool) cudaEventDestroy(e);

@@ -51,6 +51,7 @@ struct State {
     uint32_t* ts;          // LRU: [slots]
     uint32_t* hit_epoch;   // [slots] forward call in which the slot was last hit
     int32_t* hit_k;        // [slots] unique-row index of that hit
+    uint32_t* floor;       // [sets] a lower bound of the lowest priority value among the set's residents (0: none known)
     unsigned long long* stats;   // [T][8]
 };
 
@@ -464,7 +465,7 @@ k_priority(State s, Work w, uint32_t* __restrict__ ckey, StepArgs av) {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int64_t U32 = (U + 31) & ~31LL;
     for (int64_t k0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k0 < U32; k0 += Q * stride) {
-        int t[Q], loc[Q]; int32_t row[Q]; uint32_t mult[Q], old[Q]; int64_t rb[Q]; int32_t nsets[Q];
+        int t[Q], loc[Q]; int32_t row[Q]; uint32_t mult[Q], old[Q]; int64_t rb[Q], sbase[Q]; int32_t nsets[Q];
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
             const int64_t k = k0 + q * stride;
@@ -476,25 +477,35 @@ k_priority(State s, Work w, uint32_t* __restrict__ ckey, StepArgs av) {
             old[q] = 0;
             if (t[q] >= 0) {
                 const TableDev tb = s.tables[t[q]];
-                rb[q] = tb.row_base; nsets[q] = tb.n_sets;
+                rb[q] = tb.row_base; nsets[q] = tb.n_sets; sbase[q] = tb.set_base;
                 if (s.policy == 1 && loc[q] != LOC_INVALID) old[q] = s.cnt[rb[q] + row[q]];
             }
         }
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
             const int64_t k = k0 + q * stride;
-            unsigned long long m = 0, hitm = 0, uh = 0, un = 0;
+            unsigned long long m = 0, hitm = 0, uh = 0, un = 0, byp = 0;
             if (t[q] >= 0) {
                 uint32_t key = (uint32_t)nsets[q];           // sorts behind every real set: not a candidate
                 if (loc[q] != LOC_INVALID) {
                     m = mult[q]; un = 1;
+                    uint32_t pv = step;                      // the priority value the row has from now on
                     if (s.policy == 1) {                     // LFU: access count of the row, saturating
-                        s.cnt[rb[q] + row[q]] = old[q] + mult[q] < old[q] ? 0xffffffffU : old[q] + mult[q];
+                        pv = old[q] + mult[q] < old[q] ? 0xffffffffU : old[q] + mult[q];
+                        s.cnt[rb[q] + row[q]] = pv;
                     } else if (loc[q] >= 0) {
                         s.ts[loc[q]] = step;                 // LRU: time stamp of the cached row
                     }
                     if (loc[q] >= 0) { hitm = mult[q]; uh = 1; }
-                    else if (nsets[q] > 0) key = (uint32_t)w.uset[k];
+                    else if (nsets[q] > 0) {
+                        // The lowest priority value in a set never falls (counts and time stamps only grow, a replacement
+                        // puts a larger value in the place of the lowest, no way is ever emptied), so a row that does not
+                        // beat a bound recorded earlier is bypassed whatever happens in this step (Algorithm 2: PV[i] <= PV[j]).
+                        const int32_t set = w.uset[k];
+                        const bool always = s.ways == 1 && s.policy == 0;
+                        if (!always && pv <= s.floor[sbase[q] + set]) byp = 1;
+                        else key = (uint32_t)set;
+                    }
                 }
                 ckey[k] = key;
             }
@@ -506,14 +517,17 @@ k_priority(State s, Work w, uint32_t* __restrict__ ckey, StepArgs av) {
                 for (int o = 16; o > 0; o >>= 1) {
                     m += __shfl_xor_sync(0xffffffffU, m, o); hitm += __shfl_xor_sync(0xffffffffU, hitm, o);
                     uh += __shfl_xor_sync(0xffffffffU, uh, o); un += __shfl_xor_sync(0xffffffffU, un, o);
+                    byp += __shfl_xor_sync(0xffffffffU, byp, o);
                 }
                 if ((threadIdx.x & 31) == 0) {
                     unsigned long long* st = s.stats + (int64_t)t0 * 8;
                     atomicAdd(st + 0, m); atomicAdd(st + 1, hitm); atomicAdd(st + 2, un); atomicAdd(st + 3, uh);
+                    if (byp) atomicAdd(st + 6, byp);
                 }
             } else if (t[q] >= 0) {
                 unsigned long long* st = s.stats + (int64_t)t[q] * 8;
                 atomicAdd(st + 0, m); atomicAdd(st + 1, hitm); atomicAdd(st + 2, un); atomicAdd(st + 3, uh);
+                if (byp) atomicAdd(st + 6, byp);
             }
         }
     }
@@ -618,6 +632,11 @@ k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __r
                 u = f + 1;
             }
             if (n < ways) break;
+        }
+        {   // what the set's lowest priority value is now bounds it from below for good
+            const bool any_empty = (__ballot_sync(gmask, tag < 0) & gmask) != 0;
+            const uint32_t low = __reduce_min_sync(gmask, tag < 0 ? 0u : pri);
+            if (way == 0) s.floor[tb.set_base + key] = any_empty ? 0u : low;
         }
         if (cand >= 0) {
             s.tags[slot] = tag;
