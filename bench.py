@@ -33,7 +33,7 @@ METRIC = "embedding rows/sec per training step (fwd+bwd+cache) and % of 8 TB/s H
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per index of the batch, from the ncu capture summarised in
 # profiles/k_update_cfg4_8tables.md (8 of the 64 tables; traffic grows in proportion to the indices processed)
-NCU_DRAM_BYTES_PER_INDEX = {"update": 113.6}
+NCU_DRAM_BYTES_PER_INDEX = {"update": 112.2, "pool": 75.0}
 
 
 def measured_peaks():
