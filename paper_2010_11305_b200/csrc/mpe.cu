@@ -157,8 +157,8 @@ int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
     A(w.bag_of, n); A(w.kidx, n); A(w.occ_loc, n); A(w.occ_b, n);
     A(w.uniq_row, n); A(w.uniq_t, n); A(w.seg, n + 1); A(w.loc, n); A(w.final_loc, n); A(w.victim, n);
     A(w.hot_base, n); A(w.uset, n);
-    const int64_t max_tasks = L / HOT_MIN + 2;
-    A(w.task_k, max_tasks); A(w.partial, max_tasks * h->dim); A(w.hot_k, L / HOT_MIN + 2); A(w.defer_k, n); A(w.heads, n);
+    const int64_t max_tasks = hot_capacity(L);
+    A(w.task_k, max_tasks); A(w.partial, max_tasks * h->dim); A(w.hot_k, max_tasks); A(w.defer_k, n); A(w.heads, n);
 #undef A
     CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), h->stream));
     h->cap_L = L; h->cap_bags = bags;
@@ -167,6 +167,10 @@ int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
 
 // device-wide exclusive prefix sum of data[0 .. *n_ptr) in place
 void scan_u32(mpe_handle* h, uint32_t* data, const uint32_t* n_ptr, int64_t n_upper) {
+    if (n_upper <= SCAN1_MAX) {      // small steps are bound by the number of launches
+        LAUNCH(h, "scan_single", k_scan_single, 1, SCAN1_THREADS, 0, data, n_ptr);
+        return;
+    }
     const int g = grid_for(h, n_upper, SCAN_TILE, 8);
     LAUNCH(h, "scan_reduce", k_scan_reduce, g, SCAN_THREADS, 0, data, n_ptr, h->block_sums);
     LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, n_ptr, (uint32_t)SCAN_TILE, (uint32_t*)nullptr);
@@ -411,7 +415,7 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
     dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
         constexpr int LANES = decltype(lc)::value;
         auto hot = ind ? k_hot_partial<LANES, true> : k_hot_partial<LANES, false>;
-        LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, L / HOT_MIN + 1, 1, 2), 8 * LANES, 32 * s.dim * sizeof(float), s, w, av);
+        LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, hot_capacity(L), 1, 2), 8 * LANES, 32 * s.dim * sizeof(float), s, w, av);
     });
     CK(h, cudaEventRecord(h->ev_join, h->side));
     LAUNCH(h, "priority", (ind ? k_priority<true> : k_priority<false>), grid_for(h, L, 1024, 8), 256, 0, s, w, h->ckeyA, av);
@@ -425,7 +429,7 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
         LAUNCH(h, "policy", (ind ? k_policy<true> : k_policy<false>), grid_for(h, std::min<int64_t>(L, h->total_sets), 256 / s.ways, 8), 256, 0, s, w, ck, cv, av);
     }
     const int gu = grid_for(h, (L + 31) / 32, UPD_WARPS, 8);
-    const int gh = grid_for(h, L / HOT_MIN + 1, 256 / s.lanes, 4);
+    const int gh = grid_for(h, hot_capacity(L), 256 / s.lanes, 4);
     dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
         constexpr int BITS = decltype(bc)::value, LANES = decltype(lc)::value;
         auto upd = ind ? k_update<BITS, LANES, true> : k_update<BITS, LANES, false>;
@@ -956,7 +960,7 @@ constexpr size_t STATIC_SCRATCH_BYTES =
     align256((256 * ((STATIC_MAX_INDICES + SORT_TILE - 1) / SORT_TILE + STATIC_MAX_TABLES + 1) / SCAN_TILE + 2 +
               STATIC_MAX_INDICES / SCAN_TILE + 2) * 4) +                                               // block sums
     4 * align256((STATIC_MAX_TABLES + 1) * 4) +                                                        // per-table starts
-    2 * align256((STATIC_MAX_INDICES / HOT_MIN + 2) * 4) +                                             // hot-row lists
+    2 * align256(hot_capacity(STATIC_MAX_INDICES) * 4) +                                             // hot-row lists
     align256(sizeof(Counters)) + align256(sizeof(StepArgs));
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress; it is not a device address.
@@ -1003,7 +1007,7 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     uint32_t* block_sums = c.take<uint32_t>(256 * max_tiles / SCAN_TILE + 2 + STATIC_MAX_INDICES / SCAN_TILE + 2);
     w.table_start = c.take<int32_t>(STATIC_MAX_TABLES + 1); w.tile_base = c.take<int32_t>(STATIC_MAX_TABLES + 1);
     w.ustart = c.take<int32_t>(STATIC_MAX_TABLES + 1); w.ctile_base = c.take<int32_t>(STATIC_MAX_TABLES + 1);
-    w.hot_k = c.take<int32_t>(STATIC_MAX_INDICES / HOT_MIN + 2); w.task_k = c.take<int32_t>(STATIC_MAX_INDICES / HOT_MIN + 2);
+    w.hot_k = c.take<int32_t>(hot_capacity(STATIC_MAX_INDICES)); w.task_k = c.take<int32_t>(hot_capacity(STATIC_MAX_INDICES));
     w.ctr = c.take<Counters>(1);
     w.args = c.take<StepArgs>(1);
     if (c.used > STATIC_SCRATCH_BYTES) return MPE_ERR_ARG;      // cannot happen: the size formula above mirrors this list

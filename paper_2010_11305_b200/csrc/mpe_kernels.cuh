@@ -9,6 +9,14 @@ namespace mpe {
 
 constexpr int HOT_SPAN = 1024;        // occurrences covered by one multi-block gradient task (two tree levels)
 constexpr int HOT_MIN = 256;          // rows with more occurrences than this take the multi-block path
+// A step with few distinct rows has few warps' worth of work in k_update, and its duration is that of the warp with the
+// longest rows: there the multi-block path starts earlier.
+constexpr int HOT_MIN_SMALL = 64;
+constexpr int HOT_SMALL_U = 131072;   // "few": at most this many distinct rows
+// upper bound of the number of hot rows, and of their tasks, in a step of L indices (either threshold)
+__host__ __device__ constexpr int64_t hot_capacity(int64_t L) {
+    return (L / HOT_MIN_SMALL < HOT_SMALL_U ? L / HOT_MIN_SMALL : HOT_SMALL_U) + L / HOT_MIN + L / HOT_SPAN + 4;
+}
 constexpr int ERR_INDEX = 0, ERR_OFFSETS = 1;
 
 struct TableDev {
@@ -259,6 +267,7 @@ k_probe(State s, Work w, StepArgs av) {
     const int lane = threadIdx.x & 31, way = lane & (ways - 1), grp = lane / ways;
     const uint32_t gmask = group_mask(ways);
     const int64_t U = w.ctr->U;
+    const uint32_t hot_min = U <= HOT_SMALL_U ? (uint32_t)HOT_MIN_SMALL : (uint32_t)HOT_MIN;
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
     for (int64_t k0 = ((int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 32; k0 < U; k0 += nwarps * 32) {
         const int64_t k = k0 + lane;
@@ -302,7 +311,7 @@ k_probe(State s, Work w, StepArgs av) {
             // rows with very many occurrences get their gradient summed by whole blocks, HOT_SPAN occurrences per task
             int hb = -1;
             const uint32_t mult = (uint32_t)(w.seg[k + 1] - w.seg[k]);
-            if (myloc != LOC_INVALID && mult > (uint32_t)HOT_MIN) {
+            if (myloc != LOC_INVALID && mult > hot_min) {
                 const uint32_t nt = (mult + HOT_SPAN - 1) / HOT_SPAN;
                 hb = (int)atomicAdd(&w.ctr->hot_tasks, nt);
                 w.hot_k[atomicAdd(&w.ctr->hot_rows, 1u)] = (int32_t)k;
@@ -804,7 +813,7 @@ constexpr int UPD_NB = 4;        // gradient rows per batch of asynchronous copi
 constexpr int UPD_DEPTH = 2;     // batches in flight per group
 constexpr int UPD_SMEM = UPD_WARPS * (UPD_DEPTH * UPD_NB * 32 * 16 + 32 * 3 * 16);
 
-// Every distinct row with at most HOT_MIN occurrences, except newcomers that wait for a write-back.  A warp stages the
+// Every distinct row that is not on the multi-block path, except newcomers that wait for a write-back.  A warp stages the
 // bookkeeping of 32 consecutive rows in shared memory, one row per lane (coalesced loads; the per-row scalar work --
 // addresses, the stochastic-rounding key -- is done there once, 32 rows at a time).  The distinct rows of a block are
 // consecutive in the sorted batch, so the gradient rows they need are one contiguous run of the sorted occurrence list

@@ -233,4 +233,26 @@ k_scan_apply(uint32_t* __restrict__ data, const uint32_t* __restrict__ n_ptr, co
     }
 }
 
+// short arrays: the whole exclusive scan in one block and one launch (in place)
+constexpr int SCAN1_THREADS = 512;
+constexpr int SCAN1_ITEMS = 8;
+constexpr int64_t SCAN1_MAX = 32768;
+__global__ void __launch_bounds__(SCAN1_THREADS)
+k_scan_single(uint32_t* __restrict__ data, const uint32_t* __restrict__ n_ptr) {
+    __shared__ uint32_t tmp[SCAN1_THREADS / 32 + 1];
+    const uint32_t n = *n_ptr;
+    uint32_t carry = 0;
+    for (uint32_t base = 0; base < n; base += SCAN1_THREADS * SCAN1_ITEMS) {
+        const uint32_t i = base + threadIdx.x * SCAN1_ITEMS;
+        uint32_t v[SCAN1_ITEMS], sum = 0;
+#pragma unroll
+        for (int q = 0; q < SCAN1_ITEMS; ++q) { v[q] = i + q < n ? data[i + q] : 0; sum += v[q]; }
+        uint32_t total;
+        uint32_t ex = carry + block_exclusive_scan<SCAN1_THREADS>(sum, &total, tmp);
+#pragma unroll
+        for (int q = 0; q < SCAN1_ITEMS; ++q) { if (i + q < n) data[i + q] = ex; ex += v[q]; }
+        carry += total;
+    }
+}
+
 }  // namespace mpe
