@@ -428,7 +428,7 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
         LAUNCH(h, "policy_heads", k_policy_heads, grid_for(h, L, 256, 8), 256, 0, s, w, ck);
         LAUNCH(h, "policy", (ind ? k_policy<true> : k_policy<false>), grid_for(h, std::min<int64_t>(L, h->total_sets), 256 / s.ways, 8), 256, 0, s, w, ck, cv, av);
     }
-    const int gu = grid_for(h, (L + 31) / 32, UPD_WARPS, 8);
+    const int gu = grid_for(h, (L + 7) / 8, UPD_WARPS, 8);
     const int gh = grid_for(h, hot_capacity(L), 256 / s.lanes, 4);
     dispatch(h->bits, s.lanes, [&](auto bc, auto lc) {
         constexpr int BITS = decltype(bc)::value, LANES = decltype(lc)::value;

@@ -811,6 +811,7 @@ struct RawRow { float4 f; uint2 q; float2 sb; };
 constexpr int UPD_WARPS = 4;     // warps per block of k_update
 constexpr int UPD_NB = 4;        // gradient rows per batch of asynchronous copies
 constexpr int UPD_DEPTH = 2;     // batches in flight per group
+constexpr int UPD_SMALL_U = 524288;   // at most this many distinct rows: blocks of 8 rows instead of 32
 constexpr int UPD_SMEM = UPD_WARPS * (UPD_DEPTH * UPD_NB * 32 * 16 + 32 * 3 * 16);
 
 // Every distinct row that is not on the multi-block path, except newcomers that wait for a write-back.  A warp stages the
@@ -830,7 +831,7 @@ k_update(State s, Work w, StepArgs av) {
     const float* __restrict__ grad = a.grad;
     const float lr = a.lr;
     const uint64_t step = a.step;
-    constexpr int dim = 4 * LANES, G = 32 / LANES, RPG = LANES, NB = LANES < UPD_NB ? LANES : UPD_NB, BPW = LANES / NB;
+    constexpr int dim = 4 * LANES, G = 32 / LANES, NB = LANES < UPD_NB ? LANES : UPD_NB, BPW = LANES / NB;
     constexpr int SLOTS = UPD_DEPTH * NB;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int sub = lane & (LANES - 1), grp = lane / LANES, gbase = lane & ~(LANES - 1);
@@ -841,6 +842,10 @@ k_update(State s, Work w, StepArgs av) {
     // C = {victim's key, victim's global row lo, hi, gradient column}
     int4* recs = reinterpret_cast<int4*>(upd_smem + UPD_WARPS * UPD_DEPTH * UPD_NB * 32 * 16) + warp * 96;
     const int64_t U = w.ctr->U;
+    // rows per hand-out and per group: 32 per warp when there is plenty of work; a step with few distinct rows is cut
+    // finer, because there the kernel lasts as long as its longest chain of rows (each row ends in dependent loads)
+    const int rpt = U > UPD_SMALL_U ? 32 : (G > 8 ? G : 8);
+    const int rpg = rpt / G;
     const uint32_t stride_bytes = (uint32_t)s.T * (uint32_t)dim * 4u;
     const char* gcol = reinterpret_cast<const char*>(grad + 4 * sub);
     const float NZ = __int_as_float(0x80000000);          // -0: adding it changes no value, not even a zero's sign
@@ -848,11 +853,11 @@ k_update(State s, Work w, StepArgs av) {
         // blocks of 32 rows are handed out on demand: their cost varies with the rows' multiplicities
         uint32_t blk = 0;
         if (lane == 0) blk = atomicAdd(&w.ctr->upd_next, 1u);
-        const int64_t k0 = (int64_t)__shfl_sync(0xffffffffU, blk, 0) * 32;
+        const int64_t k0 = (int64_t)__shfl_sync(0xffffffffU, blk, 0) * rpt;
         if (k0 >= U) break;
         const int64_t k = k0 + lane;
         bool skip = true; int myt = -1;
-        if (k < U) {
+        if (lane < rpt && k < U) {
             const int32_t first = w.seg[k], row = w.uniq_row[k];
             const int loc = w.loc[k], floc = w.final_loc[k], hb = w.hot_base[k], victim = w.victim[k], t = w.uniq_t[k];
             myt = t;
@@ -889,9 +894,9 @@ k_update(State s, Work w, StepArgs av) {
         const uint32_t skipmask = __ballot_sync(0xffffffffU, skip);                       // rows that are not ours (or past the end)
         const uint32_t stopmask = skipmask | __ballot_sync(0xffffffffU, lane > 0 && myt != tprev);   // a run ends before these rows
         __syncwarp();
-        // this group's rows: RPG consecutive ones; their runs
-        const int gr0 = grp * RPG, gr1 = gr0 + RPG;
-        uint32_t avail = ~skipmask & (RPG == 32 ? 0xffffffffU : (((1U << RPG) - 1U) << gr0));
+        // this group's rows: rpg consecutive ones; their runs
+        const int gr0 = grp * rpg, gr1 = gr0 + rpg;
+        uint32_t avail = ~skipmask & (rpg == 32 ? 0xffffffffU : (((1U << rpg) - 1U) << gr0));
         while (avail) {
             const int rs = __ffs(avail) - 1;
             const uint32_t above = stopmask & (rs == 31 ? 0u : (0xfffffffeU << rs));
