@@ -408,3 +408,26 @@ def test_table_in_host_memory_gives_the_same_results(bits, policy):
     h.flush()
     o.flush()
     compare_state(h, o, cfg, [0, 1], rng)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_configurations(seed):
+    """Configurations drawn at random: table counts and sizes (down to a few rows), every code width, both policies and
+    optimizers, every associativity, bag shapes from one-hot to long ragged bags, cache sizes from none to most of a table.
+    Rows with 65..1024 occurrences (the boundary between the per-warp and the multi-block gradient paths) and tables
+    that end inside a block of distinct rows come up by construction."""
+    from parity_util import run_parity
+    rng = np.random.default_rng(1000 + seed)
+    T = int(rng.integers(1, 7))
+    num_rows = [int(rng.choice([3, 17, 200, 2000, 30000, 400000])) for _ in range(T)]
+    dim = int(rng.choice([4, 8, 16, 32, 64, 128]))
+    bits = int(rng.choice([2, 4, 8, 16]))
+    ways = int(rng.choice([1, 2, 4, 8, 16, 32]))
+    policy = int(rng.choice([wl.LRU, wl.LFU]))
+    opt = int(rng.choice([wl.SGD, wl.ROWWISE_ADAGRAD]))
+    bag = [("fixed", 1), ("fixed", 7), ("poisson", 3.0), ("poisson_cap", 25.0, 60), ("poisson", 0.4)][int(rng.integers(0, 5))]
+    zipf = [[None, 0.7, 1.05, 1.3, 2.0][int(rng.integers(0, 5))] for _ in range(T)]
+    cfg = _cfg(name=f"rnd{seed}", num_rows=num_rows, dim=dim, bits=bits, ways=ways, policy=policy, optimizer=opt,
+               cache_fraction=float(rng.choice([0.0, 0.01, 0.1, 0.6])), batch=int(rng.choice([1, 33, 256, 1500])), bag=bag, zipf=zipf,
+               lr=0.05, steps=5, seed=seed)
+    run_parity(cfg, 5, check_every=2)
