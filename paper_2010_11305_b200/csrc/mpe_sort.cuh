@@ -110,8 +110,7 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict_
     constexpr int WARPS = SORT_THREADS / 32;
     __shared__ uint32_t wcnt[WARPS][256];      // per-warp digit counters, then per-warp digit bases
     __shared__ uint32_t gbase[256];            // first global position of each digit of this tile, later minus its tile-local start
-    __shared__ uint32_t skey[SORT_TILE];
-    __shared__ uint32_t sval[SORT_TILE];
+    __shared__ uint2 skv[SORT_TILE];
     __shared__ uint32_t scan_tmp[SORT_THREADS / 32 + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int ntiles = tile_base[T];
@@ -158,17 +157,16 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict_
             const int e = warp * (32 * SORT_ITEMS) + i * 32 + lane;
             const uint32_t dg = (key[i] >> shift) & 255u;
             const uint32_t pos = wcnt[warp][dg] + rank[i];
-            skey[pos] = key[i];
-            sval[pos] = e < count ? (vals_in ? vals_in[start + e] : (uint32_t)(start + e)) : 0u;
+            skv[pos] = make_uint2(key[i], e < count ? (vals_in ? vals_in[start + e] : (uint32_t)(start + e)) : 0u);
         }
         __syncthreads();
         // padding keys (0xffffffff, digit 255) follow every real key of the tile, so positions [0,count) are real
         for (int j = threadIdx.x; j < count; j += SORT_THREADS) {
-            const uint32_t k = skey[j];
-            const uint32_t dg = (k >> shift) & 255u;
+            const uint2 kv = skv[j];
+            const uint32_t dg = (kv.x >> shift) & 255u;
             const uint32_t dst = gbase[dg] + (uint32_t)j;
-            keys_out[dst] = k;
-            vals_out[dst] = sval[j];
+            keys_out[dst] = kv.x;
+            vals_out[dst] = kv.y;
         }
         __syncthreads();
     }
