@@ -31,8 +31,8 @@ from paper_2010_11305_b200 import workloads as wl  # noqa: E402
 
 METRIC = "embedding rows/sec per training step (fwd+bwd+cache) and % of 8 TB/s HBM"
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum per index of the batch, from the ncu capture summarised in
-# profiles/k_update_cfg4_8tables.md (8 of the 64 tables; traffic grows in proportion to the indices processed)
+# dram__bytes_read.sum + dram__bytes_write.sum per index of the batch, from ncu captures of the kernels on 8 of the 64
+# tables of configuration 4 (same shapes per table; the traffic grows in proportion to the indices processed)
 NCU_DRAM_BYTES_PER_INDEX = {"update": 112.2, "pool": 75.0}
 
 
