@@ -87,7 +87,7 @@ struct Work {
     int32_t* bag_of;       // [L] bag of every index position
     uint32_t* kidx;        // [L] unique-row index of the i-th sorted element
     int32_t* occ_loc;      // [L] by position: cache slot, LOC_MISS or LOC_INVALID
-    int32_t* occ_b;        // [L] by sorted order: sample of the element
+    int32_t* occ_b;        // [L] by sorted order: sample of the element; sign bit: last occurrence of its row
     int32_t *uniq_row, *uniq_t, *seg, *loc, *final_loc, *victim, *hot_base, *uset;   // per unique row
     int32_t* task_k;       // [hot tasks]
     int32_t* hot_k;        // [hot rows]
@@ -335,7 +335,9 @@ k_broadcast(State s, Work w, const uint32_t* __restrict__ spos, StepArgs av) {
         const uint32_t k = w.kidx[i];
         const uint32_t p = spos[i];
         w.occ_loc[p] = w.loc[k];
-        w.occ_b[i] = w.bag_of[p] - w.uniq_t[k] * B;
+        // the sign bit marks the last occurrence of a distinct row (sample ids are below 2^31)
+        const bool last = i + 1 >= L || w.kidx[i + 1] != k;
+        w.occ_b[i] = (w.bag_of[p] - w.uniq_t[k] * B) | (last ? (int32_t)0x80000000 : 0);
     }
 }
 
@@ -674,7 +676,7 @@ __device__ __forceinline__ float4 sum_chunk(const int32_t* __restrict__ occ_b, c
     constexpr int NB = LANES < 8 ? LANES : 8;
     float4 acc;
     if (LANES == 32 && len == 32) {       // a full chunk handled by a whole warp: no bounds to check, 8 rows in flight
-        const uint32_t myb = (uint32_t)occ_b[first + sub];
+        const uint32_t myb = (uint32_t)occ_b[first + sub] & 0x7fffffffU;
         float4 va[4], vb[4];
         auto row = [&](int u) { return __ldg(reinterpret_cast<const float4*>(gcol + (size_t)__shfl_sync(0xffffffffU, myb, u) * stride_bytes)); };
 #pragma unroll
@@ -702,7 +704,7 @@ __device__ __forceinline__ float4 sum_chunk(const int32_t* __restrict__ occ_b, c
     acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int j0 = 0; j0 < len; j0 += LANES) {
         const int n = min(LANES, len - j0);
-        const uint32_t myb = sub < n ? (uint32_t)occ_b[first + j0 + sub] : 0u;
+        const uint32_t myb = sub < n ? (uint32_t)occ_b[first + j0 + sub] & 0x7fffffffU : 0u;
         for (int u0 = 0; u0 < n; u0 += NB) {
             float4 v[NB];
 #pragma unroll
@@ -908,11 +910,20 @@ k_update(State s, Work w, StepArgs av) {
             const int32_t os = Bs.z, oe = Be.z + Be.y;
             const char* src = gcol + (size_t)(uint32_t)recs[rs * 3 + 2].w * 4u;
             const int nbatch = (oe - os + NB - 1) / NB;
-            uint32_t wb = 0;                                   // sample ids of LANES consecutive occurrences, one per lane
+            uint32_t wb = 0, wlast = 0;                        // sample ids of LANES consecutive occurrences, one per lane; their row ends
+            uint32_t pend = 0;                                 // row-end bits of the batches in flight, NB bits per batch
             auto issue = [&](int j) {                          // copies of batch j (none when j is past the end); always one group
                 if (j < nbatch) {
                     const int jw = j % BPW;
-                    if (jw == 0) { const int32_t o = os + j * NB + sub; wb = o < oe ? (uint32_t)w.occ_b[o] : 0u; }
+                    if (jw == 0) {
+                        const int32_t o = os + j * NB + sub;
+                        const uint32_t raw = o < oe ? (uint32_t)w.occ_b[o] : 0u;
+                        wlast = (__ballot_sync(gmask, (raw >> 31) != 0) & gmask) >> gbase;
+                        wb = raw & 0x7fffffffU;
+                    }
+                    constexpr uint32_t BM = (1u << NB) - 1u;
+                    const int f = (j % UPD_DEPTH) * NB;
+                    pend = (pend & ~(BM << f)) | (((wlast >> (jw * NB)) & BM) << f);
                     const int32_t left = oe - (os + j * NB);
                     const uint32_t dst = ring_s + (uint32_t)(((j % UPD_DEPTH) * NB) * LANES * 16);
 #pragma unroll
@@ -925,9 +936,9 @@ k_update(State s, Work w, StepArgs av) {
             };
             // current row: its records, its stored value, how many terms are still to come
             int r = rs;
-            int4 A, Bq; RawRow xr; int rem = 0;
+            int4 A, Bq; RawRow xr;
             auto open_row = [&]() {
-                A = recs[r * 3]; Bq = recs[r * 3 + 1]; rem = Bq.y;
+                A = recs[r * 3]; Bq = recs[r * 3 + 1];
                 if (A.x >= 0) {
                     xr.f = reinterpret_cast<const float4*>(s.slab + (int64_t)A.x * dim)[sub];
                 } else {
@@ -940,22 +951,32 @@ k_update(State s, Work w, StepArgs av) {
 #pragma unroll
             for (int j = 0; j < UPD_DEPTH; ++j) issue(j);
             float4 chunkacc = make_float4(NZ, NZ, NZ, NZ), rowacc = chunkacc;
-            int c = 0;                                         // terms in the current chunk of 32
+            int c = 0;                                         // terms of the current row added so far
             const int nocc = oe - os;
-#pragma unroll 1
-            for (int jo = 0; jo < nocc; ++jo) {
-                if ((jo & (NB - 1)) == 0) {                    // a batch boundary: refill the slots just drained, then wait for this batch
-                    if (jo) issue(jo / NB - 1 + UPD_DEPTH);
-                    cp_async_wait<UPD_DEPTH - 1>();
+            for (int j = 0; j < nbatch; ++j) {
+                if (j) issue(j - 1 + UPD_DEPTH);               // refill the slots just drained,
+                cp_async_wait<UPD_DEPTH - 1>();                // then wait for this batch
+                const uint32_t m = (pend >> ((j % UPD_DEPTH) * NB)) & ((1u << NB) - 1u);      // bit u: occurrence u ends its row
+                const float4* slot = ring + ((j % UPD_DEPTH) * NB) * LANES;
+                const int cnt = min(NB, nocc - j * NB);
+                if (NB == 4 && m == 0 && cnt == 4 && (c & 31) <= 28) {
+                    // four terms of one row and one chunk of 32 (the long rows are mostly made of these): no bookkeeping
+                    chunkacc = add4(add4(add4(add4(chunkacc, slot[0]), slot[LANES]), slot[2 * LANES]), slot[3 * LANES]);
+                    c += 4;
+                    if ((c & 31) == 0) { rowacc = add4(rowacc, chunkacc); chunkacc = make_float4(NZ, NZ, NZ, NZ); }
+                    continue;
                 }
-                {
-                    chunkacc = add4(chunkacc, ring[(jo & (SLOTS - 1)) * LANES]);
-                    ++c; --rem;
-                    if (c == 32 || rem == 0) {                 // a finished chunk joins the sum of chunk sums
+#pragma unroll 1
+                for (int u = 0; u < cnt; ++u) {
+                    chunkacc = add4(chunkacc, slot[u * LANES]);
+                    ++c;
+                    const bool last = (m >> u) & 1u;
+                    if (last || (c & 31) == 0) {               // a finished chunk joins the sum of chunk sums
                         rowacc = add4(rowacc, chunkacc);
-                        chunkacc = make_float4(NZ, NZ, NZ, NZ); c = 0;
+                        chunkacc = make_float4(NZ, NZ, NZ, NZ);
                     }
-                    if (rem == 0) {
+                    if (last) {
+                        c = 0;
                         const int loc = A.x, floc = A.y;
                         float4 x = xr.f;
                         if (loc < 0) x = decode4<BITS>(xr.q, xr.sb);
