@@ -188,7 +188,8 @@ int seg_sort(mpe_handle* h, uint32_t* kA, uint32_t* kB, uint32_t* vA, uint32_t* 
     const int passes = (key_bits + 7) / 8;
     uint32_t *kin = kA, *kout = kB, *vin = nullptr, *vout = vB;
     for (int p = 0; p < passes; ++p) {
-        LAUNCH(h, "sort_hist", k_sort_hist, g, SORT_THREADS, 0, (const uint32_t*)kin, seg_start, (const int32_t*)tile_base, T, 8 * p, h->hist);
+        LAUNCH(h, "sort_hist", k_sort_hist, grid_for(h, max_tiles, SORT_THREADS / 32, 8), SORT_THREADS, 0, (const uint32_t*)kin, seg_start,
+               (const int32_t*)tile_base, T, 8 * p, h->hist);
         scan_u32(h, h->hist, hist_len, 256 * max_tiles);
         LAUNCH(h, "sort_scatter", k_sort_scatter, g, SORT_THREADS, 0, (const uint32_t*)kin, (const uint32_t*)vin, kout, vout,
                seg_start, (const int32_t*)tile_base, T, 8 * p, (const uint32_t*)h->hist);

@@ -82,21 +82,33 @@ __device__ __forceinline__ int find_segment(const int32_t* __restrict__ base, in
 __global__ void __launch_bounds__(SORT_THREADS)
 k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base,
             int T, int shift, uint32_t* __restrict__ hist) {
-    __shared__ uint32_t cnt[256];
+    // one warp per tile: its own 256 counters, eight key loads in flight per lane, no block-wide barrier
+    constexpr int WARPS = SORT_THREADS / 32;
+    __shared__ uint32_t cnt[WARPS][256];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int ntiles = tile_base[T];
-    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    for (int tile = blockIdx.x * WARPS + warp; tile < ntiles; tile += gridDim.x * WARPS) {
         const int t = find_segment(tile_base, T, tile);
         const int local = tile - tile_base[t];
         const int nt = tile_base[t + 1] - tile_base[t];
         const int32_t start = seg_start[t] + local * SORT_TILE;
         const int32_t end = min(start + SORT_TILE, seg_start[t + 1]);
-        cnt[threadIdx.x] = 0;
-        __syncthreads();
-        for (int32_t i = start + threadIdx.x; i < end; i += SORT_THREADS)
-            atomicAdd(&cnt[(keys[i] >> shift) & 255u], 1u);
-        __syncthreads();
-        hist[(size_t)256 * tile_base[t] + (size_t)threadIdx.x * nt + local] = cnt[threadIdx.x];
-        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cnt[warp][i * 32 + lane] = 0;
+        __syncwarp();
+        for (int32_t i0 = start + lane; i0 < end; i0 += 32 * 8) {
+            uint32_t k[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) k[q] = i0 + 32 * q < end ? keys[i0 + 32 * q] : 0u;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (i0 + 32 * q < end) atomicAdd(&cnt[warp][(k[q] >> shift) & 255u], 1u);
+        }
+        __syncwarp();
+        uint32_t* out = hist + (size_t)256 * tile_base[t] + local;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[(size_t)(i * 32 + lane) * nt] = cnt[warp][i * 32 + lane];
+        __syncwarp();
     }
 }
 
