@@ -111,25 +111,34 @@ __global__ void k_set_args_backward(StepArgs* a, const float* grad, float lr, un
     a->grad = grad; a->lr = lr; a->step = step;
 }
 
+// one warp: resets the step's counters and reads where each table's bags begin (the offsets of bags 0, B, 2B, ...), 32
+// tables at a time so that the loads overlap; offsets that do not start at 0, end at L or grow abandon the step
 template <bool IND>
 __global__ void k_prelude(Work w, int T, StepArgs av) {
     StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
-    if (threadIdx.x == 0 && blockIdx.x == 0) {
-        const int32_t* __restrict__ offsets = a.offsets;
-        const int B = a.B;
-        const uint32_t L = a.L;
-        Counters* c = w.ctr;
+    if (blockIdx.x != 0 || threadIdx.x >= 32) return;
+    const int lane = threadIdx.x;
+    const int32_t* __restrict__ offsets = a.offsets;
+    const int B = a.B;
+    const uint32_t L = a.L;
+    Counters* c = w.ctr;
+    if (lane == 0) {
         c->L = L; c->U = 0; c->hot_rows = 0; c->hot_tasks = 0; c->abort = 0; c->dropped = 0; c->hot_occ = 0; c->deferred = 0; c->n_heads = 0; c->upd_next = 0;
-        bool bad = offsets[0] != 0 || offsets[(int64_t)T * B] != (int32_t)L;
-        int32_t prev = 0;
-        w.table_start[0] = 0;
-        for (int t = 1; t < T; ++t) {
-            int32_t v = offsets[(int64_t)t * B];
-            if (v < prev || v > (int32_t)L) { bad = true; v = prev; }
-            w.table_start[t] = v; prev = v;
+    }
+    bool bad = false;
+    for (int t0 = 0; t0 <= T; t0 += 32) {
+        const int t = t0 + lane;
+        if (t <= T) {
+            const int32_t v = offsets[(int64_t)t * B];
+            const int32_t before = t > 0 ? offsets[(int64_t)(t - 1) * B] : 0;
+            if (v < before || v < 0 || v > (int32_t)L || (t == 0 && v != 0) || (t == T && v != (int32_t)L)) bad = true;
+            w.table_start[t] = v;
         }
-        w.table_start[T] = (int32_t)L;
-        if (bad) { c->abort = 1; atomicAdd(&c->err[ERR_OFFSETS], 1ULL); }
+    }
+    bad = __any_sync(0xffffffffU, bad);
+    if (bad) {                                   // nothing downstream may trust the offsets: every table is empty
+        for (int t = lane; t <= T; t += 32) w.table_start[t] = t == T ? (int32_t)L : 0;
+        if (lane == 0) { c->abort = 1; atomicAdd(&c->err[ERR_OFFSETS], 1ULL); }
     }
 }
 
