@@ -50,14 +50,22 @@ __device__ __forceinline__ uint32_t group_mask(int lanes_per_row) {
 
 // The four stored values of one lane (columns 4*sub .. 4*sub+3) are BITS*4 adjacent bits of the row: one byte (INT2),
 // one u16 (INT4), one u32 (INT8) or two u32 (FP16 table, BITS = 16); the lowest column sits in the lowest bits.
+// read-only loads of data that is used once (a low-precision row on its way to FP32): through the non-coherent path and
+// without taking a line of L1, which is better spent on the FP32 rows that many bags share
+__device__ __forceinline__ uint32_t ld_once_u8(const void* p) { uint32_t v; asm("ld.global.nc.L1::no_allocate.u8 %0, [%1];" : "=r"(v) : "l"(p)); return v; }
+__device__ __forceinline__ uint32_t ld_once_u16(const void* p) { unsigned short v; asm("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(v) : "l"(p)); return v; }
+__device__ __forceinline__ uint32_t ld_once_u32(const void* p) { uint32_t v; asm("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p)); return v; }
+__device__ __forceinline__ uint2 ld_once_u32x2(const void* p) { uint2 v; asm("ld.global.nc.L1::no_allocate.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p)); return v; }
+__device__ __forceinline__ float2 ld_once_f32x2(const void* p) { float2 v; asm("ld.global.nc.L1::no_allocate.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p)); return v; }
+
 template <int BITS, bool RO>
 __device__ __forceinline__ uint2 load_codes4(const uint8_t* codes, int64_t grow, int dim, int sub) {
     const uint8_t* row = codes + grow * (dim * BITS / 8);
-    if (BITS == 16) return RO ? __ldg(reinterpret_cast<const uint2*>(row) + sub) : reinterpret_cast<const uint2*>(row)[sub];
+    if (BITS == 16) return RO ? ld_once_u32x2(reinterpret_cast<const uint2*>(row) + sub) : reinterpret_cast<const uint2*>(row)[sub];
     uint32_t q;
-    if (BITS == 8) q = RO ? __ldg(reinterpret_cast<const uint32_t*>(row) + sub) : reinterpret_cast<const uint32_t*>(row)[sub];
-    else if (BITS == 4) q = RO ? __ldg(reinterpret_cast<const uint16_t*>(row) + sub) : reinterpret_cast<const uint16_t*>(row)[sub];
-    else q = RO ? __ldg(row + sub) : row[sub];
+    if (BITS == 8) q = RO ? ld_once_u32(reinterpret_cast<const uint32_t*>(row) + sub) : reinterpret_cast<const uint32_t*>(row)[sub];
+    else if (BITS == 4) q = RO ? ld_once_u16(reinterpret_cast<const uint16_t*>(row) + sub) : reinterpret_cast<const uint16_t*>(row)[sub];
+    else q = RO ? ld_once_u8(row + sub) : row[sub];
     return make_uint2(q, 0u);
 }
 template <int BITS>
@@ -118,7 +126,7 @@ __device__ __forceinline__ float4 decode4(uint2 qq, float2 p) {
 template <int BITS, bool RO>
 __device__ __forceinline__ float4 dequant4(const uint8_t* codes, const float2* sb, int64_t grow, int dim, int sub) {
     float2 p = make_float2(1.0f, 0.0f);
-    if (BITS != 16) p = RO ? __ldg(sb + grow) : sb[grow];
+    if (BITS != 16) p = RO ? ld_once_f32x2(sb + grow) : sb[grow];
     return decode4<BITS>(load_codes4<BITS, RO>(codes, grow, dim, sub), p);
 }
 
