@@ -465,7 +465,7 @@ k_pool(State s, Work w, StepArgs av) {
             const int g = (int)(b / r->B_local);
             dst = r->out[g] + ((b - (int64_t)g * r->B_local) * r->T_global + r->t_base + t) * dim;
         }
-        reinterpret_cast<float4*>(dst)[sub] = acc;
+        __stcs(reinterpret_cast<float4*>(dst) + sub, acc);      // written once, read by somebody else: not worth a place in L2
         b += ng;
         while (b >= B) { b -= B; ++t; }
     }
