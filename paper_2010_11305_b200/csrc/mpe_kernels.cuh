@@ -262,19 +262,16 @@ __global__ void k_ustart(Work w, int T) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// cache tag lookup: one group of `ways` lanes per distinct row (Section 3 "Cache Structure")
+// cache tag lookup: one lane per distinct row, which reads the `ways` tags of the row's set (Section 3 "Cache Structure")
 // ---------------------------------------------------------------------------------------------
 template <bool IND>
 __global__ void __launch_bounds__(256)
 k_probe(State s, Work w, StepArgs av) {
     StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
     const uint32_t epoch = a.epoch;
-    // A warp takes 32 consecutive distinct rows: lane l works out row l's set (32 rows at a time), then the
-    // warp compares the tags of 32/ways rows per round, `ways` lanes per row.
     if (w.ctr->abort) return;
-    const int ways = s.ways, G = 32 / ways;
-    const int lane = threadIdx.x & 31, way = lane & (ways - 1), grp = lane / ways;
-    const uint32_t gmask = group_mask(ways);
+    const int ways = s.ways;
+    const int lane = threadIdx.x & 31;
     const int64_t U = w.ctr->U;
     const uint32_t hot_min = U <= HOT_SMALL_U ? (uint32_t)HOT_MIN_SMALL : (uint32_t)HOT_MIN;
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
@@ -288,32 +285,33 @@ k_probe(State s, Work w, StepArgs av) {
             if (row >= tb.N) myloc = LOC_INVALID;
             else if (tb.n_sets > 0) { set = set_of((uint32_t)row, tb.salt, tb.n_sets); gset = (int32_t)(tb.set_base + set); }
         }
-        // 32 / G rounds, eight at a time (eight tag loads in flight).  In round `it` group g looks at row it*G + g; every
-        // lane sees the whole ballot, and lane l keeps the one of the round that handled its own row (l / G).
-        uint32_t myhit = 0;
-        for (int it0 = 0; it0 < ways; it0 += 8) {
-            int32_t tg[8], rg[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int r = ((it0 + j) * G + grp) & 31;
-                rg[j] = __shfl_sync(0xffffffffU, gset, r);
-                tg[j] = -1;
-                if (it0 + j < ways && rg[j] >= 0) tg[j] = s.tags[(int64_t)rg[j] * ways + way];
-            }
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int it = it0 + j;
-                const int r = (it * G + grp) & 31;
-                const int32_t rrow = __shfl_sync(0xffffffffU, row, r);
-                const bool match = it < ways && rg[j] >= 0 && tg[j] == rrow;
-                const uint32_t hit = __ballot_sync(0xffffffffU, match);
-                if (match) { const int64_t slot = (int64_t)rg[j] * ways + way; s.hit_epoch[slot] = epoch; s.hit_k[slot] = (int32_t)(k0 + r); }
-                if (lane / G == it) myhit = hit;
-            }
-        }
+        // every lane compares its own row with the tags of the row's set (contiguous: `ways` INT32, read 16 bytes at a
+        // time with all loads in flight before any comparison); a set holds a row at most once
         if (gset >= 0) {
-            const uint32_t mine = (myhit >> ((lane % G) * ways)) & (ways == 32 ? 0xffffffffU : ((1u << ways) - 1u));
-            if (mine) myloc = (int)((int64_t)gset * ways + (__ffs(mine) - 1));
+            const int32_t* __restrict__ tg = s.tags + (int64_t)gset * ways;
+            int mw = -1;
+            if (ways >= 4) {
+                for (int w0 = 0; w0 < ways; w0 += 32) {
+                    int4 t4[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        t4[j] = w0 + 4 * j < ways ? *reinterpret_cast<const int4*>(tg + w0 + 4 * j) : make_int4(-1, -1, -1, -1);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (t4[j].x == row) mw = w0 + 4 * j;
+                        if (t4[j].y == row) mw = w0 + 4 * j + 1;
+                        if (t4[j].z == row) mw = w0 + 4 * j + 2;
+                        if (t4[j].w == row) mw = w0 + 4 * j + 3;
+                    }
+                }
+            } else {
+                for (int w0 = 0; w0 < ways; ++w0) if (tg[w0] == row) mw = w0;
+            }
+            if (mw >= 0) {
+                const int64_t slot = (int64_t)gset * ways + mw;
+                myloc = (int)slot;
+                s.hit_epoch[slot] = epoch; s.hit_k[slot] = (int32_t)k;
+            }
         }
         if (k < U) {
             w.loc[k] = myloc; w.final_loc[k] = myloc; w.uset[k] = set;
