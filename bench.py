@@ -51,12 +51,19 @@ class ClockSampler:
                   "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         self.gpu = gpu_index
         self.proc = None
-        self.lines = []
+        self.lines = []            # (arrival time, text)
+        self.t_begin = self.t_end = None
+
+    def begin(self):
+        self.t_begin = time.perf_counter()
+
+    def end(self):
+        self.t_end = time.perf_counter()
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                          "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -64,7 +71,7 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.perf_counter(), line.strip()))
 
     def stop(self):
         if not self.proc:
@@ -73,7 +80,10 @@ class ClockSampler:
         self.thread.join(timeout=2)
         sm, smax, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for l in self.lines:
+        # the samples taken while the timed steps ran (a sample describes the interval before it arrives); all of them
+        # if the region was too short to catch one
+        inside = [l for t, l in self.lines if self.t_begin is not None and self.t_end is not None and self.t_begin <= t <= self.t_end + 0.03]
+        for l in (inside or [l for _, l in self.lines]):
             f = [x.strip() for x in l.split(",")]
             if len(f) < 7:
                 continue
@@ -85,7 +95,7 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "during_timed_steps": bool(inside), "reasons": sorted(reasons)}
 
 
 def describe(cfg):
@@ -197,11 +207,13 @@ def run_ours(args, cfg, rank, world, local_rank):
     time.sleep(0.3)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.begin()
     e0.record(cs)
     for i in range(args.warmup, args.warmup + args.steps):
         step(i)
     e1.record(cs)
     barrier()
+    sampler.end()
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop()
     prof = h.profile_read()
