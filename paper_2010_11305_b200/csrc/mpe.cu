@@ -733,14 +733,12 @@ int mpe_flush(mpe_handle* h) {
     if (!h) return MPE_ERR_ARG;
     DeviceGuard guard(h->device);
     const State& s = h->st;
-    for (int t = 0; t < h->T; ++t) {
-        const int64_t nslot = (int64_t)h->tables[t].n_sets * h->ways;
-        if (nslot == 0) continue;
-        const int g = grid_for(h, nslot, 256 / s.lanes, 8);
-        if (h->bits == 8) LAUNCH(h, "flush", k_flush<8>, g, 256, 0, s, t, (uint64_t)h->last_step);
-        else if (h->bits == 4) LAUNCH(h, "flush", k_flush<4>, g, 256, 0, s, t, (uint64_t)h->last_step);
-        else if (h->bits == 2) LAUNCH(h, "flush", k_flush<2>, g, 256, 0, s, t, (uint64_t)h->last_step);
-        else LAUNCH(h, "flush", k_flush<16>, g, 256, 0, s, t, (uint64_t)h->last_step);
+    if (h->total_slots > 0) {
+        const int g = grid_for(h, h->total_slots, 256 / s.lanes, 8);
+        if (h->bits == 8) LAUNCH(h, "flush", k_flush<8>, g, 256, 0, s, h->total_slots, (uint64_t)h->last_step);
+        else if (h->bits == 4) LAUNCH(h, "flush", k_flush<4>, g, 256, 0, s, h->total_slots, (uint64_t)h->last_step);
+        else if (h->bits == 2) LAUNCH(h, "flush", k_flush<2>, g, 256, 0, s, h->total_slots, (uint64_t)h->last_step);
+        else LAUNCH(h, "flush", k_flush<16>, g, 256, 0, s, h->total_slots, (uint64_t)h->last_step);
     }
     return check_launch(h);
 }

@@ -1088,19 +1088,26 @@ __global__ void k_init_table(State s, int t, float lo, float hi) {
     }
 }
 
+// every resident row of every table is down-converted into the low-precision table (and stays resident): one group of
+// lanes per cache slot of the concatenated cache; the slot's table is found by bisection over the tables' first sets
 template <int BITS>
-__global__ void k_flush(State s, int t, uint64_t step) {
+__global__ void __launch_bounds__(256)
+k_flush(State s, int64_t total_slots, uint64_t step) {
     const int lanes = s.lanes;
     const int sub = threadIdx.x & (lanes - 1);
-    const TableDev tb = s.tables[t];
-    const int64_t nslot = (int64_t)tb.n_sets * s.ways;
     const int64_t gpb = blockDim.x / lanes, ng = gpb * gridDim.x;
-    for (int64_t i = blockIdx.x * gpb + threadIdx.x / lanes; i < nslot; i += ng) {
-        const int64_t slot = tb.set_base * s.ways + i;
+    for (int64_t slot = blockIdx.x * gpb + threadIdx.x / lanes; slot < total_slots; slot += ng) {
         const int32_t tag = s.tags[slot];
         if (tag < 0) continue;
+        const int64_t set = slot / s.ways;
+        int lo = 0, hi = s.T;                      // largest t with tables[t].set_base <= set (tables without a cache share a base)
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s.tables[mid].set_base <= set) lo = mid; else hi = mid;
+        }
+        const int t = lo;
         const float4 x = reinterpret_cast<const float4*>(s.slab + slot * s.dim)[sub];
-        quantize_store<BITS>(x, s.codes, s.sb, tb.row_base + tag, s.dim, sub, lanes,
+        quantize_store<BITS>(x, s.codes, s.sb, s.tables[t].row_base + tag, s.dim, sub, lanes,
                              rowkey(s.seed, DOMAIN_FLUSH, (uint32_t)t, (uint32_t)tag, step), s.rounding != 0);
     }
 }
