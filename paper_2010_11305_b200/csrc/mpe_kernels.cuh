@@ -1096,19 +1096,30 @@ k_flush(State s, int64_t total_slots, uint64_t step) {
     const int lanes = s.lanes;
     const int sub = threadIdx.x & (lanes - 1);
     const int64_t gpb = blockDim.x / lanes, ng = gpb * gridDim.x;
-    for (int64_t slot = blockIdx.x * gpb + threadIdx.x / lanes; slot < total_slots; slot += ng) {
-        const int32_t tag = s.tags[slot];
-        if (tag < 0) continue;
-        const int64_t set = slot / s.ways;
-        int lo = 0, hi = s.T;                      // largest t with tables[t].set_base <= set (tables without a cache share a base)
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (s.tables[mid].set_base <= set) lo = mid; else hi = mid;
+    constexpr int Q = 4;                           // slots per group and round: their loads are in flight together
+    for (int64_t slot0 = blockIdx.x * gpb + threadIdx.x / lanes; slot0 < total_slots; slot0 += Q * ng) {
+        int32_t tag[Q]; float4 x[Q];
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            const int64_t slot = slot0 + q * ng;
+            tag[q] = slot < total_slots ? s.tags[slot] : -1;
         }
-        const int t = lo;
-        const float4 x = reinterpret_cast<const float4*>(s.slab + slot * s.dim)[sub];
-        quantize_store<BITS>(x, s.codes, s.sb, s.tables[t].row_base + tag, s.dim, sub, lanes,
-                             rowkey(s.seed, DOMAIN_FLUSH, (uint32_t)t, (uint32_t)tag, step), s.rounding != 0);
+#pragma unroll
+        for (int q = 0; q < Q; ++q)
+            if (tag[q] >= 0) x[q] = reinterpret_cast<const float4*>(s.slab + (slot0 + q * ng) * s.dim)[sub];
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            if (tag[q] < 0) continue;
+            const int64_t set = (slot0 + q * ng) / s.ways;
+            int lo = 0, hi = s.T;                  // largest t with tables[t].set_base <= set (tables without a cache share a base)
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (s.tables[mid].set_base <= set) lo = mid; else hi = mid;
+            }
+            const int t = lo;
+            quantize_store<BITS>(x[q], s.codes, s.sb, s.tables[t].row_base + tag[q], s.dim, sub, lanes,
+                                 rowkey(s.seed, DOMAIN_FLUSH, (uint32_t)t, (uint32_t)tag[q], step), s.rounding != 0);
+        }
     }
 }
 
