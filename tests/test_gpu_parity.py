@@ -431,3 +431,16 @@ def test_random_configurations(seed):
                cache_fraction=float(rng.choice([0.0, 0.01, 0.1, 0.6])), batch=int(rng.choice([1, 33, 256, 1500])), bag=bag, zipf=zipf,
                lr=0.05, steps=5, seed=seed)
     run_parity(cfg, 5, check_every=2)
+
+
+@pytest.mark.parametrize("policy,ways", [(wl.LFU, 8), (wl.LFU, 1), (wl.LRU, 4)])
+def test_many_steps_keep_the_recorded_set_bounds_valid(policy, ways):
+    """Sixty steps on small tables: residents are replaced again and again, counts and time stamps keep growing, and the
+    per-set lower bounds that let the priority kernel bypass candidates early must never reject a row that Algorithm 2
+    would admit (state, counters and statistics stay bit-equal to the oracle throughout)."""
+    from parity_util import run_parity
+    cfg = _cfg(num_rows=[600, 90, 2500], dim=16, bits=4, policy=policy, ways=ways, cache_fraction=0.1, batch=48,
+               bag=("poisson", 3.0), zipf=[1.1, 0.8, 1.3], steps=60, seed=77)
+    h, o, _ = run_parity(cfg, 60, check_every=10)
+    s = h.stats(0)
+    assert s[4] > 0 and s[6] > 0            # admissions and bypasses both happened
