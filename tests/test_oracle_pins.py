@@ -532,3 +532,36 @@ def test_fp16_table_halves_the_memory():
     o = orc.Oracle([1000], 128, 16, 0.0, 32, orc.LFU)
     m = o.memory_bytes().astype(np.float64)
     assert (m[0] + m[1] + m[2] + m[3]) / m[5] == 0.5
+
+
+@pytest.mark.parametrize("policy", [orc.LRU, orc.LFU])
+def test_lowest_resident_priority_of_a_full_set_never_falls(policy):
+    """Algorithm 2 replaces the resident with the lowest priority value by a row whose value is strictly larger, and
+    counts / time stamps only grow: once a set is full, the minimum over its residents is non-decreasing from step to step.
+    (The CUDA path records that minimum per set and uses it to bypass hopeless candidates early.)"""
+    from paper_2010_11305_b200 import workloads as wl
+    cfg = wl.Config(name="floor", num_rows=[800, 120], dim=8, bits=8, cache_fraction=0.1, ways=4, policy=policy, optimizer=wl.SGD,
+                    lr=0.05, batch=40, bag=("poisson", 3.0), zipf=[1.1, 0.9], steps=40, seed=9)
+    st = wl.Stream(cfg, "cpu")
+    o = orc.Oracle(cfg.num_rows, cfg.dim, cfg.bits, cfg.cache_fraction, cfg.ways, policy, seed=cfg.seed)
+    prev = [None] * cfg.num_tables
+    grew = 0
+    for step in range(1, cfg.steps + 1):
+        idx, off, grad = st.batch(step)
+        o.forward(idx.numpy(), off.numpy(), cfg.batch)
+        o.backward(grad.numpy(), cfg.lr, step)
+        for t in range(cfg.num_tables):
+            tags, _, ts = o.cache(t)
+            tags = tags.reshape(-1, cfg.ways)
+            if policy == orc.LFU:
+                pv = np.array([[o.cnt(t, int(r)) if r >= 0 else -1 for r in row] for row in tags], np.int64)
+            else:
+                pv = np.where(tags >= 0, ts.reshape(-1, cfg.ways).astype(np.int64), -1)
+            low = np.where((tags >= 0).all(1), pv.min(1), -1)          # -1: the set still has an empty way
+            if prev[t] is not None:
+                full_before = prev[t] >= 0
+                assert (low[full_before] >= prev[t][full_before]).all(), (step, t)
+                grew += int((low[full_before] > prev[t][full_before]).sum())
+            prev[t] = low
+    o.close()
+    assert grew > 0                                                     # and it did move
