@@ -169,61 +169,72 @@ class Emulator:
         return int(self.cnt[j]) if self.policy == "lfu" else int(self.ts[s, w])
 
     def backward(self, bags, grad_out, lr, step):
+        """One update of the cached table (Section 3 "update", Section 3 "Cache Replacement Policy", Section 5.1),
+        in four passes over the distinct rows of the batch: merge, priorities, full-precision update, placement."""
         lr = F(lr)
-        occ = {}
-        for b, bag in enumerate(bags):              # sort + merge duplicates (Section 5.1)
+        # merge: one gradient per distinct row, duplicates summed (Section 5.1)
+        where = {}
+        for b, bag in enumerate(bags):
             for i in bag:
                 if 0 <= i < self.N:
-                    occ.setdefault(i, []).append(b)
-        I_U = sorted(occ)
-        resident = {i: (self.n > 0 and i in self.I_C[self.h(i)]) for i in I_U}
-        order = [i for i in I_U if resident[i]] + [i for i in I_U if not resident[i]]
-        for i in order:
-            g = tree_sum([np.asarray(grad_out[b], F) for b in occ[i]])
-            # Update PV[i]
+                    where.setdefault(i, []).append(b)
+        rows = sorted(where)
+        merged = {i: tree_sum([np.asarray(grad_out[b], F) for b in where[i]]) for i in rows}
+        cached = {i: (self.n > 0 and i in self.I_C[self.h(i)]) for i in rows}
+        # priorities: popularity counts every access, recency stamps the cached rows that were used
+        for i in rows:
             if self.policy == "lfu":
-                self.cnt[i] = min(self.cnt[i] + len(occ[i]), M32)
-            elif resident[i]:
+                self.cnt[i] = min(self.cnt[i] + len(where[i]), M32)
+            elif cached[i]:
                 s = self.h(i)
                 self.ts[s, list(self.I_C[s]).index(i)] = step
-            # T[i,:] <- T[i,:] + U[i,:]
-            if self.optimizer == "sgd":
-                mult = lr
-            else:
-                P = []
-                for l in range(self.d // 4):
-                    a = F(g[4 * l] * g[4 * l])
-                    for e in (1, 2, 3):
-                        a = fma32(g[4 * l + e], g[4 * l + e], a)
-                    P.append(a)
-                stride = len(P) // 2
-                while stride >= 1:
-                    for l in range(stride):
-                        P[l] = F(P[l] + P[l + stride])
-                    stride //= 2
-                self.G[i] = F(self.G[i] + F(P[0] * (F(1.0) / F(self.d))))
-                mult = F(lr / F(np.sqrt(self.G[i]) + self.eps))
-            self.T[i] = np.array([fma32(-mult, g[c], self.T[i, c]) for c in range(self.d)], F)
-            key_i = rowkey(self.seed, 2, self.table, i, step)
-            if self.n == 0:
-                self.T[i] = fake_quantize(self.T[i], self.bits, self.rounding, key_i)[0]
+        # update: every touched row moves in full precision, wherever it lives
+        for i in rows:
+            self.T[i] = self._optimizer(i, merged[i], lr)
+        # placement: rows that were cached stay as they are; the others, in ascending row id, either take the place of
+        # their set's lowest-priority resident (which then drops to low precision) or drop to low precision themselves
+        for i in rows:
+            if cached[i]:
                 continue
-            if resident[i]:
-                continue
-            s = self.h(i)
-            pvs = [self._pv_resident(s, w) for w in range(self.alpha)]
-            w_j = int(np.argmin(pvs))               # first minimum = lowest way
-            pv_i = int(self.cnt[i]) if self.policy == "lfu" else step
-            bypass = pv_i <= pvs[w_j]
-            if self.alpha == 1 and self.policy == "lru":
-                bypass = False
-            if bypass:
-                self.T[i] = fake_quantize(self.T[i], self.bits, self.rounding, key_i)[0]
-            else:
-                j = self.I_C[s, w_j]
-                if j >= 0:
-                    self.T[j] = fake_quantize(self.T[j], self.bits, self.rounding,
-                                              rowkey(self.seed, 2, self.table, int(j), step))[0]
-                self.I_C[s, w_j] = i
-                if self.policy == "lru":
-                    self.ts[s, w_j] = step
+            if self.n == 0 or not self._admit(i, step):
+                self.T[i] = self._lower(i, step)
+
+    def _optimizer(self, i, g, lr):
+        if self.optimizer == "sgd":
+            mult = lr
+        else:
+            sq = []
+            for l in range(self.d // 4):
+                a = F(g[4 * l] * g[4 * l])
+                for e in (1, 2, 3):
+                    a = fma32(g[4 * l + e], g[4 * l + e], a)
+                sq.append(a)
+            stride = len(sq) // 2
+            while stride >= 1:
+                for l in range(stride):
+                    sq[l] = F(sq[l] + sq[l + stride])
+                stride //= 2
+            self.G[i] = F(self.G[i] + F(sq[0] * (F(1.0) / F(self.d))))
+            mult = F(lr / F(np.sqrt(self.G[i]) + self.eps))
+        return np.array([fma32(-mult, g[c], self.T[i, c]) for c in range(self.d)], F)
+
+    def _lower(self, i, step):
+        """The row as the low-precision table would hold it after this step (Algorithm 1 with this step's random bits)."""
+        return fake_quantize(self.T[i], self.bits, self.rounding, rowkey(self.seed, 2, self.table, int(i), step))[0]
+
+    def _admit(self, i, step):
+        """Whether row i enters the cache; if so the displaced resident is lowered and i takes its way."""
+        s = self.h(i)
+        standing = [self._pv_resident(s, w) for w in range(self.alpha)]
+        weakest = int(np.argmin(standing))           # first minimum: the lowest way wins a tie, an empty way beats all
+        mine = int(self.cnt[i]) if self.policy == "lfu" else step
+        direct_mapped_recency = self.alpha == 1 and self.policy == "lru"
+        if mine <= standing[weakest] and not direct_mapped_recency:
+            return False
+        out = self.I_C[s, weakest]
+        if out >= 0:
+            self.T[out] = self._lower(out, step)
+        self.I_C[s, weakest] = i
+        if self.policy == "lru":
+            self.ts[s, weakest] = step
+        return True

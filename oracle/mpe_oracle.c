@@ -553,7 +553,7 @@ int orc_backward(orc* o, const float* grad_out, float lr, int64_t step) {
         tb->stats[0] += (uint64_t)n;
         tb->stats[2] += (uint64_t)nu;
         /* --- Algorithm 2, with I_U ordered: all hits first, then misses in ascending row id --- */
-        /* "Update PV[i] according to LRU or LFU" for every i in I_U */
+        /* priority values first: every row of I_U is now one access more popular / more recent (Section 3 "Cache Replacement Policy") */
         for (k = 0; k < nu; ++k) {
             const int64_t row = urow[k];
             int w = -1; int32_t set = 0;
@@ -568,7 +568,7 @@ int orc_backward(orc* o, const float* grad_out, float lr, int64_t step) {
             }
             if (w >= 0) { tb->stats[1] += (uint64_t)umult[k]; tb->stats[3] += 1; }
         }
-        /* "T[i,:] <- T[i,:] + U[i,:]" in full precision, from the value the forward fetched */
+        /* the gradient update itself, in full precision, applied to the value the forward fetched (Section 3 "update") */
         float x[1024];
         for (k = 0; k < nu; ++k) {
             fetch(o, t, urow[k], x);
@@ -592,7 +592,7 @@ int orc_backward(orc* o, const float* grad_out, float lr, int64_t step) {
             const int32_t set = orc_set_index((uint32_t)row, tb->salt, tb->n_sets);
             const int64_t pv_i = o->policy == ORC_LFU ? (int64_t)tb->cnt[rec_get(o, t, row)] : step;
             int j = 0; int64_t pv_j = resident_pv(o, t, set, 0);
-            for (int w = 1; w < A; ++w) {   /* j <- argmin PV over I_C[s]; ties -> lowest way */
+            for (int w = 1; w < A; ++w) {   /* the resident of lowest priority value in the set; ties -> lowest way */
                 int64_t pv = resident_pv(o, t, set, w);
                 if (pv < pv_j) { pv_j = pv; j = w; }
             }
@@ -607,7 +607,7 @@ int orc_backward(orc* o, const float* grad_out, float lr, int64_t step) {
                     store_quantized(o, t, tb->tag[slot], tb->crow + slot * d, ORC_DOMAIN_SR, step);
                     tb->stats[5] += 1;
                 }
-                tb->tag[slot] = (int32_t)row;                 /* replace j by i in I_C[s] */
+                tb->tag[slot] = (int32_t)row;                 /* the newcomer takes over the tag */
                 memcpy(tb->crow + slot * d, xnew + k * d, (size_t)d * sizeof(float));   /* verbatim */
                 if (o->policy == ORC_LRU) tb->ts[slot] = (uint32_t)step;
                 tb->stats[4] += 1;

@@ -12,7 +12,12 @@
  * Algorithm 2 tag/priority sequences, the worked de-duplication example of
  * Section 5.1, the full-cache case against a textbook FP32 embedding-bag
  * trainer, a literal single-array emulator of Algorithms 1+2, brute force
- * without a cache, and the appendix's memory-compression table.
+ * without a cache, the appendix's memory-compression table; and for the parts
+ * the paper does not have -- flush (each resident's entry against the emulator's
+ * own quantizer with the flush stream, cache and fetched values unchanged,
+ * training identical with and without flushes), ids outside a table (equal to
+ * the batch with them deleted), inconsistent offsets (refused, state untouched)
+ * and the table mask (equal to a run whose masked tables receive no indices).
  * Parity unpinned (pure conventions, fixed by this build and mirrored on the
  * GPU): the constants of the counter hash, the cache-set hash, INT4 nibble
  * order, argmin tie-breaks, and the radix (32) of the gradient summation tree.

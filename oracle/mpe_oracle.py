@@ -161,6 +161,17 @@ def tree_sum(terms):
     return out
 
 
+class OracleError(RuntimeError):
+    """A call the oracle refused; `code` is its ORC_ERR_* value."""
+
+    def __init__(self, what, code):
+        super().__init__(f"{what} failed: {code}")
+        self.code = code
+
+
+ERR_ARG, ERR_OFFSETS, ERR_SEQUENCE = -1, -2, -3
+
+
 class Oracle:
     """One embedding collection: T tables sharing dim, precision, cache shape and policy."""
 
@@ -200,7 +211,7 @@ class Oracle:
         out = np.zeros((batch, self.T * self.d), np.float32)
         rc = _forward(self._h, indices if indices.size else np.zeros(1, np.int32), offsets, batch, indices.size, out)
         if rc != 0:
-            raise RuntimeError(f"orc_forward failed: {rc}")
+            raise OracleError("orc_forward", rc)
         self.batch = batch
         return out
 
@@ -208,7 +219,7 @@ class Oracle:
         g = np.ascontiguousarray(grad_out, np.float32)
         rc = _backward(self._h, g, lr, step)
         if rc != 0:
-            raise RuntimeError(f"orc_backward failed: {rc}")
+            raise OracleError("orc_backward", rc)
 
     def flush(self):
         _flush(self._h)

@@ -470,7 +470,7 @@ k_pool(State s, Work w, StepArgs av) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// backward 1: "Update PV[i]" for every i in I_U (Algorithm 2), candidate keys, hot-row tasks, counters
+// backward 1: new priority value of every row of I_U (Section 3 "Cache Replacement Policy"), candidate keys, counters
 // ---------------------------------------------------------------------------------------------
 template <bool IND>
 __global__ void __launch_bounds__(256)
@@ -553,8 +553,8 @@ k_priority(State s, Work w, uint32_t* __restrict__ ckey, StepArgs av) {
 
 // ---------------------------------------------------------------------------------------------
 // backward 2: admission / eviction, integer only.  One group of `ways` lanes walks the miss
-// candidates of one set in ascending row id (Algorithm 2: j <- argmin PV; PV[i] <= PV[j] -> bypass,
-// else replace j by i in I_C[s]).  Lane w holds way w of the set; the candidates are fetched `ways`
+// candidates of one set in ascending row id (Algorithm 2's admission test: a candidate whose priority value does
+// not exceed the lowest one among the residents bypasses, otherwise it takes that resident's place).  Lane w holds way w of the set; the candidates are fetched `ways`
 // at a time (one per lane) and handed round with shuffles.  No row value is read or written here.
 // ---------------------------------------------------------------------------------------------
 constexpr int VICTIM_NONE = -1;       // the way was empty, or the displaced row writes itself back
