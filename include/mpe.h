@@ -150,9 +150,28 @@ int mpe_set_rounding(mpe_handle* h, int32_t mode);
 
 /* One whole step from HOST buffers: copies indices, offsets and grad_out to the device, runs
  * forward and backward, copies the pooled output back and waits for it.  Layouts as above.
- * Uses the stream of the last mpe_forward (default stream if none). */
+ * Uses the stream of the last mpe_forward (default stream if none).  Equal to mpe_step_host_submit
+ * followed by mpe_step_host_wait. */
 int mpe_step_host(mpe_handle* h, const int32_t* h_indices, const int32_t* h_offsets, int32_t batch,
                   int64_t total_indices, const float* h_grad_out, float* h_out, float lr, int64_t step);
+
+/* The same step without waiting, so that consecutive steps overlap on the host link: the call enqueues the
+ * uploads, the kernels and the download of one step on three streams and returns.  The library keeps two sets
+ * of device staging buffers; the upload of step k+1 runs while step k computes, and the download of step k
+ * while step k+1 computes (the steps' kernels themselves run one after the other, in submission order, so the
+ * results are those of mpe_step_host called in a loop).  Any number of steps may be submitted before waiting.
+ *   h_indices, h_offsets, h_grad_out   must stay valid and unchanged until mpe_step_host_wait returns
+ *                                      (pinned memory, or the copies do not overlap with anything);
+ *   h_out                              holds the step's pooled output once mpe_step_host_wait has returned;
+ *                                      give every step in flight its own buffer.
+ * Errors: as mpe_forward / mpe_backward (argument and sequence errors are returned by the submit call;
+ * nothing is enqueued then).  Growing the staging buffers or the workspace (first call, larger batch) waits
+ * for everything in flight and reallocates; the staging buffers are sized for the batch at hand or for the
+ * reservation made with mpe_reserve, whichever is larger, so reserve the largest batch first when batch sizes
+ * vary.  mpe_step_host_wait waits for all submitted steps. */
+int mpe_step_host_submit(mpe_handle* h, const int32_t* h_indices, const int32_t* h_offsets, int32_t batch,
+                         int64_t total_indices, const float* h_grad_out, float* h_out, float lr, int64_t step);
+int mpe_step_host_wait(mpe_handle* h);
 
 /*
  * Evaluation forward that allocates nothing.  (The paper has no counterpart: this is an addition for
@@ -170,8 +189,9 @@ int mpe_step_host(mpe_handle* h, const int32_t* h_indices, const int32_t* h_offs
  * num_tables <= MPE_STATIC_MAX_TABLES; a larger call returns MPE_ERR_TOO_LARGE and does nothing.
  * It calls no cudaMalloc / cudaFree and no allocating library routine.
  *
- * It is an evaluation forward: it never changes table, cache or policy state and cannot be followed by
- * mpe_backward; calling it between the mpe_forward and mpe_backward of a training step returns
+ * It is an evaluation forward: it never changes the tables, the cached rows, the tags or the priority values
+ * (the only handle memory it writes are the per-slot marks "hit in forward call number e", which every forward
+ * rewrites under a fresh call number before anything reads them) and cannot be followed by mpe_backward; calling it between the mpe_forward and mpe_backward of a training step returns
  * MPE_ERR_SEQUENCE.  Out-of-range row ids contribute nothing and inconsistent offsets give all-zero
  * output, as in mpe_forward, but this entry point does not record them for mpe_last_error.
  *
@@ -179,7 +199,8 @@ int mpe_step_host(mpe_handle* h, const int32_t* h_indices, const int32_t* h_offs
  * contents (the call clears the counters it needs at zero): two calls whose GPU work overlaps -- different
  * streams, or different handles -- race on it.  Issue them on one stream, or wait between them.
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress); make that
- * first call outside any stream capture.
+ * first call outside any stream capture.  The look-up is guarded by a lock, so first calls may come from
+ * several host threads (on different handles) at once.
  */
 #define MPE_STATIC_MAX_INDICES 32768
 #define MPE_STATIC_MAX_BAGS 32768
@@ -206,6 +227,9 @@ int mpe_stats(mpe_handle* h, int32_t table, uint64_t* out8);
  * tables: out6 = {low-precision table incl. scale/bias, FP32 cache, tags, LFU counters or LRU
  * timestamps, optimizer state, the FP32 table this replaces}. */
 int mpe_memory_bytes(mpe_handle* h, uint64_t* out6);
+/* Device memory the handle holds beyond the model state: out2 = {bytes of the per-step workspace (sized by
+ * mpe_reserve or by the largest batch seen), bytes of the two staging sets of mpe_step_host / _submit}. */
+int mpe_workspace_bytes(mpe_handle* h, uint64_t* out2);
 /* Geometry of table `table`'s cache. */
 int mpe_cache_geometry(mpe_handle* h, int32_t table, int32_t* n_sets, int32_t* ways);
 /* Figures of the last step: out6 = {valid indices, distinct rows, dropped indices, rows whose gradient
@@ -228,13 +252,15 @@ int mpe_export_aux(mpe_handle* h, int32_t table, const int64_t* h_rows, int64_t 
 /* Steps of up to about four million indices are bound by kernel-launch latency, so by default each half of
  * the step is captured once into a CUDA graph (sized for the reserved workspace) and replayed; the per-call
  * arguments reach the kernels through device memory.  enable = 0 switches to plain launches (larger steps and
- * steps issued while profiling or while the caller captures the stream always use plain launches). */
+ * steps issued while profiling or while the caller captures the stream always use plain launches).  A backward
+ * is replayed only if its forward was.  Not allowed between a forward and its backward (MPE_ERR_SEQUENCE). */
 int mpe_use_graphs(mpe_handle* h, int32_t enable);
 
 /* ---- instrumentation ---------------------------------------------------------------------------- */
 /* Number of kernels this handle has launched so far. */
 int mpe_kernel_launches(mpe_handle* h, uint64_t* count);
-/* With profiling on, every kernel launch is bracketed by CUDA events on the launching stream. */
+/* With profiling on, every kernel launch is bracketed by CUDA events on the launching stream.  Waits for the
+ * handle's stream; not allowed between a forward and its backward (MPE_ERR_SEQUENCE). */
 int mpe_profile(mpe_handle* h, int32_t enable);
 /* Waits for the stream, then reports per kernel name the launches and the summed event time since
  * profiling was switched on (or last read): up to `cap` entries, names are 32-byte C strings.

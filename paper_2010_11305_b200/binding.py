@@ -22,8 +22,8 @@ OK, ERR_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_SEQUENCE, ERR_INDEX, ERR_OFFSETS, ER
 STATIC_MAX_INDICES, STATIC_MAX_BAGS, STATIC_MAX_TABLES = 32768, 32768, 64
 
 EXPORTS = [
-    "mpe_create", "mpe_create_placed", "mpe_reserve", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_set_rounding", "mpe_step_host", "mpe_flush", "mpe_destroy",
-    "mpe_last_error", "mpe_stats", "mpe_memory_bytes", "mpe_cache_geometry", "mpe_step_info", "mpe_export_rows",
+    "mpe_create", "mpe_create_placed", "mpe_reserve", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_set_rounding", "mpe_step_host", "mpe_step_host_submit", "mpe_step_host_wait", "mpe_flush", "mpe_destroy",
+    "mpe_last_error", "mpe_stats", "mpe_memory_bytes", "mpe_workspace_bytes", "mpe_cache_geometry", "mpe_step_info", "mpe_export_rows",
     "mpe_export_cache", "mpe_export_aux", "mpe_use_graphs", "mpe_kernel_launches", "mpe_profile", "mpe_profile_read",
     "mpe_forward_routed", "mpe_gather_grad", "mpe_peer_buffer_alloc", "mpe_peer_buffer_open", "mpe_peer_buffer_close", "mpe_peer_buffer_free",
     "mpe_error_string",
@@ -50,11 +50,14 @@ _lib.mpe_forward.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp]
 _lib.mpe_forward_static.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp]
 _lib.mpe_backward.argtypes = [_vp, _vp, _f32, _i64]
 _lib.mpe_step_host.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp, _f32, _i64]
+_lib.mpe_step_host_submit.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp, _f32, _i64]
+_lib.mpe_step_host_wait.argtypes = [_vp]
 _lib.mpe_flush.argtypes = [_vp]
 _lib.mpe_destroy.argtypes = [_vp]
 _lib.mpe_last_error.argtypes = [_vp, C.POINTER(_i32), C.POINTER(_i64)]
 _lib.mpe_stats.argtypes = [_vp, _i32, _vp]
 _lib.mpe_memory_bytes.argtypes = [_vp, _vp]
+_lib.mpe_workspace_bytes.argtypes = [_vp, _vp]
 _lib.mpe_cache_geometry.argtypes = [_vp, _i32, C.POINTER(_i32), C.POINTER(_i32)]
 _lib.mpe_step_info.argtypes = [_vp, _vp]
 _lib.mpe_export_rows.argtypes = [_vp, _i32, _vp, _i64, _vp, _vp, _vp]
@@ -159,6 +162,15 @@ class Mpe:
         _check(_lib.mpe_step_host(self._h, _ptr(h_indices), _ptr(h_offsets), batch, n, _ptr(h_grad_out), _ptr(h_out),
                                   lr, step), "mpe_step_host")
 
+    def step_host_submit(self, h_indices, h_offsets, batch, h_grad_out, h_out, lr, step):
+        """Enqueue one step from host buffers without waiting; the buffers belong to the library until step_host_wait()."""
+        n = h_indices.size if isinstance(h_indices, np.ndarray) else h_indices.numel()
+        _check(_lib.mpe_step_host_submit(self._h, _ptr(h_indices), _ptr(h_offsets), batch, n, _ptr(h_grad_out), _ptr(h_out),
+                                         lr, step), "mpe_step_host_submit")
+
+    def step_host_wait(self):
+        _check(_lib.mpe_step_host_wait(self._h), "mpe_step_host_wait")
+
     def flush(self):
         _check(_lib.mpe_flush(self._h), "mpe_flush")
 
@@ -177,6 +189,12 @@ class Mpe:
         out = np.zeros(6, np.uint64)
         _check(_lib.mpe_memory_bytes(self._h, out.ctypes.data), "mpe_memory_bytes")
         return out
+
+    def workspace_bytes(self):
+        """(bytes of the per-step workspace, bytes of the host-step staging buffers)."""
+        out = np.zeros(2, np.uint64)
+        _check(_lib.mpe_workspace_bytes(self._h, out.ctypes.data), "mpe_workspace_bytes")
+        return int(out[0]), int(out[1])
 
     def cache_geometry(self, table):
         n, w = _i32(), _i32()

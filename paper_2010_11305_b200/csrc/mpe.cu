@@ -9,6 +9,7 @@
 #include <cstdio>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <string>
 #include <type_traits>
 #include <vector>
@@ -35,20 +36,26 @@ struct mpe_handle {
     TableDev* d_tables = nullptr;
     // workspace
     int64_t cap_L = 0, cap_bags = 0;
-    uint32_t *keyA = nullptr, *keyB = nullptr, *valA = nullptr, *valB = nullptr;
-    uint32_t *ckeyA = nullptr, *ckeyB = nullptr, *cvalA = nullptr, *cvalB = nullptr;
+    uint64_t ws_bytes = 0;                  // bytes of the per-step workspace
+    uint32_t *sortA = nullptr, *sortB = nullptr;   // two buffers of 2 * sort_n words: (key, payload) records, or keys | payloads
+    int64_t sort_n = 0;
     uint32_t *hist = nullptr, *block_sums = nullptr;
     std::vector<void*> ws_allocs;
-    // staging for mpe_step_host
-    int32_t *sh_idx = nullptr, *sh_off = nullptr; float *sh_grad = nullptr, *sh_out = nullptr;
+    // staging for mpe_step_host / mpe_step_host_submit: two slots, so that the copies of one step run next to the kernels of another
+    struct HostSlot {
+        int32_t *idx = nullptr, *off = nullptr; float *grad = nullptr, *out = nullptr;
+        cudaEvent_t ev_idx = nullptr, ev_grad = nullptr, ev_fwd = nullptr, ev_done = nullptr, ev_down = nullptr;
+        bool used = false;
+    } slot[2];
     int64_t sh_cap_L = 0, sh_cap_off = 0, sh_cap_out = 0;
+    uint64_t submitted = 0;
     // step state
     cudaStream_t stream = nullptr;
     cudaStream_t side = nullptr;            // runs the hot rows' partial sums next to the policy kernels
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaStream_t copy_in = nullptr, copy_out = nullptr;   // mpe_step_host: host<->device copies next to the kernels
-    cudaEvent_t ev_idx = nullptr, ev_grad = nullptr, ev_fwd = nullptr, ev_start = nullptr;
     bool have_forward = false;
+    bool fwd_replayed = false;              // the pending forward ran as a graph replay, so the device copy of its arguments is current
     int64_t last_step = 0;
     uint64_t steps = 0;
     uint32_t epoch = 0;
@@ -144,21 +151,31 @@ int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
     auto* tr = &h->ws_allocs;
     const int T = h->T;
     const int64_t n = L + 1;
+    // arrays with one entry per distinct row: there are at most as many distinct rows as indices, and at most as many
+    // as the tables have rows (plus one pseudo row per table that collects its out-of-range ids)
+    const int64_t nu = std::min<int64_t>(L, h->total_rows + T) + 2;
     Work& w = h->wk;
     int rc = MPE_OK;
-#define A(ptr, count) if ((rc = dmalloc(h, &(ptr), (count), tr)) != MPE_OK) return rc
-    A(h->keyA, n); A(h->keyB, n); A(h->valA, n); A(h->valB, n);
-    A(h->ckeyA, n); A(h->ckeyB, n); A(h->cvalA, n); A(h->cvalB, n);
+    h->ws_bytes = 0;
+#define A(ptr, count) do { if ((rc = dmalloc(h, &(ptr), (count), tr)) != MPE_OK) return rc; \
+                           h->ws_bytes += (uint64_t)std::max<int64_t>((count), 1) * sizeof(*(ptr)); } while (0)
+    // the sort's two buffers; the second sort (miss candidates by cache set) runs in backward, when the first sort's
+    // results have been consumed, and uses the same two
+    h->sort_n = (n + 3) & ~int64_t(3);
+    A(h->sortA, 2 * h->sort_n); A(h->sortB, 2 * h->sort_n);
     const int64_t max_tiles = (L + SORT_TILE - 1) / SORT_TILE + T + 1;
     A(h->hist, 256 * max_tiles);
     A(h->block_sums, std::max<int64_t>(256 * max_tiles, n) / SCAN_TILE + 2);
     A(w.ctr, 1); A(w.args, 1);
     A(w.table_start, T + 1); A(w.tile_base, T + 1); A(w.ustart, T + 1); A(w.ctile_base, T + 1);
     A(w.bag_of, n); A(w.kidx, n); A(w.occ_loc, n); A(w.occ_b, n);
-    A(w.uniq_row, n); A(w.uniq_t, n); A(w.seg, n + 1); A(w.loc, n); A(w.final_loc, n); A(w.victim, n);
-    A(w.hot_base, n); A(w.uset, n);
+    A(w.uniq_row, nu); A(w.uniq_t, nu); A(w.seg, nu + 1); A(w.loc, nu); A(w.final_loc, nu);
+    A(w.hot_base, nu); A(w.uset, nu);
+    // written and read by backward only, at most one entry per distinct row: they take the place of per-index arrays
+    // that only forward uses
+    w.victim = w.bag_of; w.defer_k = reinterpret_cast<int32_t*>(w.kidx); w.heads = w.occ_loc;
     const int64_t max_tasks = hot_capacity(L);
-    A(w.task_k, max_tasks); A(w.partial, max_tasks * h->dim); A(w.hot_k, max_tasks); A(w.defer_k, n); A(w.heads, n);
+    A(w.task_k, max_tasks); A(w.partial, max_tasks * h->dim); A(w.hot_k, max_tasks);
 #undef A
     CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), h->stream));
     h->cap_L = L; h->cap_bags = bags;
@@ -166,42 +183,61 @@ int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
 }
 
 // device-wide exclusive prefix sum of data[0 .. *n_ptr) in place
-void scan_u32(mpe_handle* h, uint32_t* data, const uint32_t* n_ptr, int64_t n_upper) {
+void scan_u32(mpe_handle* h, uint32_t* data, const uint32_t* n_ptr, int64_t n_upper, uint32_t* block_sums) {
     if (n_upper <= SCAN1_MAX) {      // small steps are bound by the number of launches
         LAUNCH(h, "scan_single", k_scan_single, 1, SCAN1_THREADS, 0, data, n_ptr);
         return;
     }
     const int g = grid_for(h, n_upper, SCAN_TILE, 8);
-    LAUNCH(h, "scan_reduce", k_scan_reduce, g, SCAN_THREADS, 0, data, n_ptr, h->block_sums);
-    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, n_ptr, (uint32_t)SCAN_TILE, (uint32_t*)nullptr);
-    LAUNCH(h, "scan_apply", k_scan_apply, g, SCAN_THREADS, 0, data, n_ptr, (const uint32_t*)h->block_sums);
+    LAUNCH(h, "scan_reduce", k_scan_reduce, g, SCAN_THREADS, 0, data, n_ptr, block_sums);
+    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, block_sums, n_ptr, (uint32_t)SCAN_TILE, (uint32_t*)nullptr);
+    LAUNCH(h, "scan_apply", k_scan_apply, g, SCAN_THREADS, 0, data, n_ptr, (const uint32_t*)block_sums);
 }
 
-// stable sort of every segment [seg_start[t], seg_start[t+1]) by the low `key_bits` bits of the key;
-// returns which buffer pair holds the result (0 = A, 1 = B)
-int seg_sort(mpe_handle* h, uint32_t* kA, uint32_t* kB, uint32_t* vA, uint32_t* vB, const int32_t* seg_start,
-             int32_t* tile_base, uint32_t* hist_len, int key_bits, int64_t n_upper) {
+// The sort's memory: two buffers of 2 * n words each.  The keys to sort are expected in the first n words of B
+// (sort_input()); between passes the elements are (key, payload) records that alternate between A and B; the last
+// pass leaves the sorted keys in the first n words and the sorted payloads in the second n words of its buffer.
+struct SortBufs { uint32_t *A, *B; int64_t n; uint32_t *hist, *block_sums; };
+uint32_t* sort_input(const SortBufs& b) { return b.B; }
+
+// stable sort of every segment [seg_start[t], seg_start[t+1]) by the low `key_bits` bits of the key, the payload being
+// the element's position before the sort; *skey / *sval receive where the sorted keys / payloads are
+void seg_sort(mpe_handle* h, const SortBufs& b, const int32_t* seg_start, int32_t* tile_base, uint32_t* hist_len, const uint32_t* abort_flag,
+              int key_bits, int64_t n_upper, const uint32_t** skey, const uint32_t** sval) {
     const int T = h->T;
-    LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, seg_start, T, tile_base, hist_len, (const uint32_t*)&h->wk.ctr->abort);
+    LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, seg_start, T, tile_base, hist_len, abort_flag);
     const int64_t max_tiles = (n_upper + SORT_TILE - 1) / SORT_TILE + T;
-    const int g = grid_for(h, max_tiles, 1, 5);
+    const int g = grid_for(h, max_tiles, 1, MPE_SORT_MINB);
+    const int gh = grid_for(h, max_tiles, SORT_THREADS / 32, 8);
     const int passes = (key_bits + 7) / 8;
-    uint32_t *kin = kA, *kout = kB, *vin = nullptr, *vout = vB;
     for (int p = 0; p < passes; ++p) {
-        LAUNCH(h, "sort_hist", k_sort_hist, grid_for(h, max_tiles, SORT_THREADS / 32, 8), SORT_THREADS, 0, (const uint32_t*)kin, seg_start,
-               (const int32_t*)tile_base, T, 8 * p, h->hist);
-        scan_u32(h, h->hist, hist_len, 256 * max_tiles);
-        LAUNCH(h, "sort_scatter", k_sort_scatter, g, SORT_THREADS, 0, (const uint32_t*)kin, (const uint32_t*)vin, kout, vout,
-               seg_start, (const int32_t*)tile_base, T, 8 * p, (const uint32_t*)h->hist);
-        std::swap(kin, kout);
-        vin = vout; vout = (vout == vB) ? vA : vB;
+        const bool first = p == 0, last = p == passes - 1;
+        uint32_t* src = first ? b.B : ((p & 1) ? b.A : b.B);      // pass p writes A when p is even, B when p is odd
+        uint32_t* dst = (p & 1) ? b.B : b.A;
+        if (first) LAUNCH(h, "sort_hist", k_sort_hist<false>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist);
+        else LAUNCH(h, "sort_hist", k_sort_hist<true>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist);
+        scan_u32(h, b.hist, hist_len, 256 * max_tiles, b.block_sums);
+        const uint32_t* kin = src; const uint2* pin = reinterpret_cast<const uint2*>(src);
+        uint2* pout = reinterpret_cast<uint2*>(dst); uint32_t* ok = dst; uint32_t* ov = dst + b.n;
+#define SCATTER(F, L) LAUNCH(h, "sort_scatter", (k_sort_scatter<F, L>), g, SORT_THREADS, 0, kin, pin, pout, ok, ov, seg_start, \
+                             (const int32_t*)tile_base, T, 8 * p, (const uint32_t*)b.hist)
+        if (first && last) SCATTER(true, true);
+        else if (first) SCATTER(true, false);
+        else if (last) SCATTER(false, true);
+        else SCATTER(false, false);
+#undef SCATTER
+        if (last) { *skey = dst; *sval = dst + b.n; }
     }
-    return (passes & 1) ? 1 : 0;
 }
 
 // call f(integral_constant<BITS>, integral_constant<LANES>) for the handle's code width and lanes per row
 template <class F>
 void dispatch(int bits, int lanes, F&& f) {
+#ifdef MPE_ONLY_BITS        // development builds: one code width and one row width only (much shorter compile)
+    (void)bits; (void)lanes;
+    f(std::integral_constant<int, MPE_ONLY_BITS>{}, std::integral_constant<int, MPE_ONLY_LANES>{});
+    return;
+#endif
     auto by_lanes = [&](auto bc) {
         switch (lanes) {
             case 1: f(bc, std::integral_constant<int, 1>{}); break;
@@ -282,10 +318,10 @@ int mpe_create_placed(mpe_handle** out, const mpe_table_spec* tables, int32_t nu
         cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess ||
         cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking) != cudaSuccess ||
         cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->ev_idx, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->ev_grad, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->ev_fwd, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming) != cudaSuccess) { delete h; return MPE_ERR_CUDA; }
+        false) { delete h; return MPE_ERR_CUDA; }
+    for (auto& sl : h->slot)
+        for (cudaEvent_t* e : {&sl.ev_idx, &sl.ev_grad, &sl.ev_fwd, &sl.ev_done, &sl.ev_down})
+            if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) { delete h; return MPE_ERR_CUDA; }
     h->T = num_tables; h->dim = dim; h->bits = bits; h->ways = ways; h->policy = policy; h->optimizer = optimizer;
     h->code_bytes = dim * bits / 8; h->eps = eps; h->lo = init_lo; h->hi = init_hi; h->seed = seed;
     h->tables.resize(num_tables);
@@ -381,12 +417,10 @@ int enqueue_forward(mpe_handle* h, int64_t L_grid, int64_t bags_grid, bool ind) 
     const int T = h->T;
     const StepArgs av = h->args;
     LAUNCH(h, "prelude", (ind ? k_prelude<true> : k_prelude<false>), 1, 32, 0, w, T, av);
-    LAUNCH(h, "make_keys", (ind ? k_make_keys<true> : k_make_keys<false>), grid_for(h, bags_grid, 32, 8), 256, 0, s, w, h->keyA, av);
+    const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->hist, h->block_sums};
+    LAUNCH(h, "make_keys", (ind ? k_make_keys<true> : k_make_keys<false>), grid_for(h, bags_grid, 32, 8), 256, 0, s, w, sort_input(sb), av);
     // sort the row indices of the mini-batch (Section 5.1), table by table
-    const int which = seg_sort(h, h->keyA, h->keyB, h->valA, h->valB, w.table_start, w.tile_base, &w.ctr->hist_len,
-                               bits_for((uint32_t)h->max_rows), L_grid);
-    h->skey = which ? h->keyB : h->keyA;
-    h->spos = which ? h->valB : h->valA;
+    seg_sort(h, sb, w.table_start, w.tile_base, &w.ctr->hist_len, &w.ctr->abort, bits_for((uint32_t)h->max_rows), L_grid, &h->skey, &h->spos);
     // distinct rows
     const int gs = grid_for(h, L_grid, SCAN_TILE, 8);
     LAUNCH(h, "unique_count", k_unique<false>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
@@ -419,13 +453,12 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
         LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, hot_capacity(L), 1, 2), 8 * LANES, 32 * s.dim * sizeof(float), s, w, av);
     });
     CK(h, cudaEventRecord(h->ev_join, h->side));
-    LAUNCH(h, "priority", (ind ? k_priority<true> : k_priority<false>), grid_for(h, L, 1024, 8), 256, 0, s, w, h->ckeyA, av);
+    const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->hist, h->block_sums};
+    LAUNCH(h, "priority", (ind ? k_priority<true> : k_priority<false>), grid_for(h, L, 1024, 8), 256, 0, s, w, sort_input(sb), av);
     if (h->max_sets > 0) {
         // group the rows that missed by cache set, keeping ascending row id inside a set
-        const int which = seg_sort(h, h->ckeyA, h->ckeyB, h->cvalA, h->cvalB, w.ustart, w.ctile_base, &w.ctr->chist_len,
-                                   bits_for((uint32_t)h->max_sets), L);
-        const uint32_t* ck = which ? h->ckeyB : h->ckeyA;
-        const uint32_t* cv = which ? h->cvalB : h->cvalA;
+        const uint32_t *ck = nullptr, *cv = nullptr;
+        seg_sort(h, sb, w.ustart, w.ctile_base, &w.ctr->chist_len, &w.ctr->abort, bits_for((uint32_t)h->max_sets), L, &ck, &cv);
         LAUNCH(h, "policy_heads", k_policy_heads, grid_for(h, L, 256, 8), 256, 0, s, w, ck);
         LAUNCH(h, "policy", (ind ? k_policy<true> : k_policy<false>), grid_for(h, std::min<int64_t>(L, h->total_sets), 256 / s.ways, 8), 256, 0, s, w, ck, cv, av);
     }
@@ -519,13 +552,13 @@ int forward_impl(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offse
             CK(h, cudaGraphExecKernelNodeSetParams(h->x_fwd, h->n_fwd, &kp));
             CK(h, cudaGraphLaunch(h->x_fwd, h->stream));
             h->launches += h->k_fwd;
-            h->have_forward = true;
+            h->have_forward = true; h->fwd_replayed = true;
             return MPE_OK;
         }
     }
     rc = enqueue_forward(h, total_indices, bags, false);
     if (rc != MPE_OK) return rc;
-    h->have_forward = true;
+    h->have_forward = true; h->fwd_replayed = false;
     return MPE_OK;
 }
 
@@ -642,7 +675,9 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
     h->args.grad = d_grad_out; h->args.lr = lr; h->args.step = ustep;
     int rc = MPE_OK;
     bool done = false;
-    if (may_use_graph(h)) {
+    // the replayed kernels read the forward's arguments (indices, offsets, batch, epoch) from the device copy, which only
+    // a replayed forward writes; after a plainly launched forward the backward is launched plainly too
+    if (h->fwd_replayed && may_use_graph(h)) {
         if (!h->x_bwd) {
             rc = capture(h, &h->g_bwd, &h->x_bwd, &h->n_bwd, &h->k_bwd, (const void*)k_set_args_backward, [&]() {
                 LAUNCH(h, "set_args", k_set_args_backward, 1, 1, 0, w.args, d_grad_out, lr, ustep);
@@ -683,50 +718,83 @@ int mpe_set_rounding(mpe_handle* h, int32_t mode) {
 
 int mpe_use_graphs(mpe_handle* h, int32_t enable) {
     if (!h) return MPE_ERR_ARG;
+    if (h->have_forward) return MPE_ERR_SEQUENCE;      // both halves of a step are launched the same way
     h->graphs_enabled = enable != 0;
+    return MPE_OK;
+}
+
+int mpe_step_host_submit(mpe_handle* h, const int32_t* h_indices, const int32_t* h_offsets, int32_t batch,
+                         int64_t total_indices, const float* h_grad_out, float* h_out, float lr, int64_t step) {
+    if (!h || !h_offsets || batch < 0 || total_indices < 0) return MPE_ERR_ARG;
+    if ((total_indices > 0 && !h_indices) || (batch > 0 && (!h_grad_out || !h_out))) return MPE_ERR_ARG;
+    if (h->have_forward) return MPE_ERR_SEQUENCE;
+    if (step < 1 || step > 0xffffffffLL) return MPE_ERR_ARG;
+    if (step <= h->last_step) return MPE_ERR_SEQUENCE;
+    DeviceGuard guard(h->device);
+    const int64_t noff = (int64_t)h->T * batch + 1, nout = (int64_t)batch * h->T * h->dim;
+    // the workspace is sized here, before anything is enqueued (growing it waits for the stream)
+    if (total_indices > h->cap_L || (int64_t)h->T * batch > h->cap_bags || !h->wk.ctr) {
+        int rc = mpe_reserve(h, batch, total_indices);
+        if (rc != MPE_OK) return rc;
+    }
+    if (total_indices > h->sh_cap_L || noff > h->sh_cap_off || nout > h->sh_cap_out) {
+        // larger staging buffers: everything in flight has to finish first
+        CK(h, cudaStreamSynchronize(h->stream)); CK(h, cudaStreamSynchronize(h->copy_in)); CK(h, cudaStreamSynchronize(h->copy_out));
+        // sized like the workspace (mpe_reserve), so that a run of batches of slightly different sizes grows them once
+        h->sh_cap_L = std::max({total_indices, h->sh_cap_L, h->cap_L});
+        h->sh_cap_off = std::max({noff, h->sh_cap_off, h->cap_bags + 1});
+        h->sh_cap_out = std::max({nout, h->sh_cap_out, h->cap_bags * (int64_t)h->dim});
+        for (auto& sl : h->slot) {
+            cudaFree(sl.idx); cudaFree(sl.off); cudaFree(sl.grad); cudaFree(sl.out);
+            sl.idx = nullptr; sl.off = nullptr; sl.grad = nullptr; sl.out = nullptr; sl.used = false;
+            int rc;
+            if ((rc = dmalloc(h, &sl.idx, h->sh_cap_L, nullptr)) != MPE_OK) return rc;
+            if ((rc = dmalloc(h, &sl.off, h->sh_cap_off, nullptr)) != MPE_OK) return rc;
+            if ((rc = dmalloc(h, &sl.grad, h->sh_cap_out, nullptr)) != MPE_OK) return rc;
+            if ((rc = dmalloc(h, &sl.out, h->sh_cap_out, nullptr)) != MPE_OK) return rc;
+        }
+    }
+    // Three streams: uploads, kernels, downloads.  The slot's buffers are free again once the step that used them two
+    // submissions ago has finished its kernels (inputs) and its download (output); the upload of this step therefore runs
+    // while the previous step computes, and the previous step's download while this step's forward runs.
+    mpe_handle::HostSlot& sl = h->slot[h->submitted & 1];
+    cudaStream_t st = h->stream;
+    if (sl.used) CK(h, cudaStreamWaitEvent(h->copy_in, sl.ev_done, 0));
+    if (total_indices) CK(h, cudaMemcpyAsync(sl.idx, h_indices, sizeof(int32_t) * total_indices, cudaMemcpyHostToDevice, h->copy_in));
+    CK(h, cudaMemcpyAsync(sl.off, h_offsets, sizeof(int32_t) * noff, cudaMemcpyHostToDevice, h->copy_in));
+    CK(h, cudaEventRecord(sl.ev_idx, h->copy_in));
+    if (nout) CK(h, cudaMemcpyAsync(sl.grad, h_grad_out, sizeof(float) * nout, cudaMemcpyHostToDevice, h->copy_in));
+    CK(h, cudaEventRecord(sl.ev_grad, h->copy_in));
+    CK(h, cudaStreamWaitEvent(st, sl.ev_idx, 0));
+    if (sl.used) CK(h, cudaStreamWaitEvent(st, sl.ev_down, 0));           // the slot's previous output has left the device
+    int rc = mpe_forward(h, sl.idx, sl.off, batch, total_indices, sl.out, (void*)st);
+    if (rc != MPE_OK) { cudaStreamSynchronize(h->copy_in); return rc; }
+    CK(h, cudaEventRecord(sl.ev_fwd, st));
+    CK(h, cudaStreamWaitEvent(h->copy_out, sl.ev_fwd, 0));
+    if (nout) CK(h, cudaMemcpyAsync(h_out, sl.out, sizeof(float) * nout, cudaMemcpyDeviceToHost, h->copy_out));
+    CK(h, cudaEventRecord(sl.ev_down, h->copy_out));
+    CK(h, cudaStreamWaitEvent(st, sl.ev_grad, 0));
+    rc = mpe_backward(h, sl.grad, lr, step);
+    if (rc != MPE_OK) { cudaStreamSynchronize(h->copy_in); cudaStreamSynchronize(st); h->have_forward = false; return rc; }
+    CK(h, cudaEventRecord(sl.ev_done, st));
+    sl.used = true;
+    ++h->submitted;
+    return MPE_OK;
+}
+
+int mpe_step_host_wait(mpe_handle* h) {
+    if (!h) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    cudaError_t e1 = cudaStreamSynchronize(h->copy_out), e2 = cudaStreamSynchronize(h->stream), e3 = cudaStreamSynchronize(h->copy_in);
+    CK(h, e1); CK(h, e2); CK(h, e3);
     return MPE_OK;
 }
 
 int mpe_step_host(mpe_handle* h, const int32_t* h_indices, const int32_t* h_offsets, int32_t batch,
                   int64_t total_indices, const float* h_grad_out, float* h_out, float lr, int64_t step) {
-    if (!h || !h_offsets || batch < 0 || total_indices < 0) return MPE_ERR_ARG;
-    if ((total_indices > 0 && !h_indices) || (batch > 0 && (!h_grad_out || !h_out))) return MPE_ERR_ARG;
-    DeviceGuard guard(h->device);
-    const int64_t noff = (int64_t)h->T * batch + 1, nout = (int64_t)batch * h->T * h->dim;
-    if (total_indices > h->sh_cap_L || noff > h->sh_cap_off || nout > h->sh_cap_out) {
-        CK(h, cudaStreamSynchronize(h->stream));
-        cudaFree(h->sh_idx); cudaFree(h->sh_off); cudaFree(h->sh_grad); cudaFree(h->sh_out);
-        h->sh_idx = nullptr; h->sh_off = nullptr; h->sh_grad = nullptr; h->sh_out = nullptr;
-        h->sh_cap_L = std::max(total_indices, h->sh_cap_L); h->sh_cap_off = std::max(noff, h->sh_cap_off);
-        h->sh_cap_out = std::max(nout, h->sh_cap_out);
-        int rc;
-        if ((rc = dmalloc(h, &h->sh_idx, h->sh_cap_L, nullptr)) != MPE_OK) return rc;
-        if ((rc = dmalloc(h, &h->sh_off, h->sh_cap_off, nullptr)) != MPE_OK) return rc;
-        if ((rc = dmalloc(h, &h->sh_grad, h->sh_cap_out, nullptr)) != MPE_OK) return rc;
-        if ((rc = dmalloc(h, &h->sh_out, h->sh_cap_out, nullptr)) != MPE_OK) return rc;
-    }
-    // The gradient upload runs next to the forward kernels and the output download next to the backward
-    // kernels (PCIe moves data in both directions at once); only the indices are needed before anything starts.
-    cudaStream_t st = h->stream;
-    CK(h, cudaEventRecord(h->ev_start, st));
-    CK(h, cudaStreamWaitEvent(h->copy_in, h->ev_start, 0));
-    if (total_indices) CK(h, cudaMemcpyAsync(h->sh_idx, h_indices, sizeof(int32_t) * total_indices, cudaMemcpyHostToDevice, h->copy_in));
-    CK(h, cudaMemcpyAsync(h->sh_off, h_offsets, sizeof(int32_t) * noff, cudaMemcpyHostToDevice, h->copy_in));
-    CK(h, cudaEventRecord(h->ev_idx, h->copy_in));
-    if (nout) CK(h, cudaMemcpyAsync(h->sh_grad, h_grad_out, sizeof(float) * nout, cudaMemcpyHostToDevice, h->copy_in));
-    CK(h, cudaEventRecord(h->ev_grad, h->copy_in));
-    CK(h, cudaStreamWaitEvent(st, h->ev_idx, 0));
-    int rc = mpe_forward(h, h->sh_idx, h->sh_off, batch, total_indices, h->sh_out, (void*)st);
-    if (rc != MPE_OK) { cudaStreamSynchronize(h->copy_in); return rc; }
-    CK(h, cudaEventRecord(h->ev_fwd, st));
-    CK(h, cudaStreamWaitEvent(h->copy_out, h->ev_fwd, 0));
-    if (nout) CK(h, cudaMemcpyAsync(h_out, h->sh_out, sizeof(float) * nout, cudaMemcpyDeviceToHost, h->copy_out));
-    CK(h, cudaStreamWaitEvent(st, h->ev_grad, 0));
-    rc = mpe_backward(h, h->sh_grad, lr, step);
-    cudaError_t e1 = cudaStreamSynchronize(h->copy_out), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(h->copy_in);
+    int rc = mpe_step_host_submit(h, h_indices, h_offsets, batch, total_indices, h_grad_out, h_out, lr, step);
     if (rc != MPE_OK) return rc;
-    CK(h, e1); CK(h, e2); CK(h, e3);
-    return MPE_OK;
+    return mpe_step_host_wait(h);
 }
 
 int mpe_flush(mpe_handle* h) {
@@ -753,14 +821,16 @@ int mpe_destroy(mpe_handle* h) {
     if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->copy_in) { cudaStreamSynchronize(h->copy_in); cudaStreamDestroy(h->copy_in); }
     if (h->copy_out) { cudaStreamSynchronize(h->copy_out); cudaStreamDestroy(h->copy_out); }
-    for (cudaEvent_t e : {h->ev_idx, h->ev_grad, h->ev_fwd, h->ev_start}) if (e) cudaEventDestroy(e);
+    for (auto& sl : h->slot) {
+        for (cudaEvent_t e : {sl.ev_idx, sl.ev_grad, sl.ev_fwd, sl.ev_done, sl.ev_down}) if (e) cudaEventDestroy(e);
+        cudaFree(sl.idx); cudaFree(sl.off); cudaFree(sl.grad); cudaFree(sl.out);
+    }
     free_workspace(h);
     State& s = h->st;
     if (h->table_on_host) { cudaFreeHost(s.codes); cudaFreeHost(s.sb); } else { cudaFree(s.codes); cudaFree(s.sb); }
     cudaFree(h->d_route);
     cudaFree(h->d_tables); cudaFree(s.cnt); cudaFree(s.G); cudaFree(s.slab);
     cudaFree(s.tags); cudaFree(s.ts); cudaFree(s.hit_epoch); cudaFree(s.hit_k); cudaFree(s.floor); cudaFree(s.stats);
-    cudaFree(h->sh_idx); cudaFree(h->sh_off); cudaFree(h->sh_grad); cudaFree(h->sh_out);
     for (auto& r : h->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto e : h->event_pool) cudaEventDestroy(e);
     delete h;
@@ -802,6 +872,13 @@ int mpe_memory_bytes(mpe_handle* h, uint64_t* out6) {
     out6[3] = pv;                                                    // INT32 counter per embedding row (LFU) / per cached row (LRU)
     out6[4] = h->optimizer == MPE_ROWWISE_ADAGRAD ? N * 4 : 0;
     out6[5] = N * 4 * d;
+    return MPE_OK;
+}
+
+int mpe_workspace_bytes(mpe_handle* h, uint64_t* out2) {
+    if (!h || !out2) return MPE_ERR_ARG;
+    out2[0] = h->ws_bytes;
+    out2[1] = 2 * ((uint64_t)h->sh_cap_L * 4 + (uint64_t)h->sh_cap_off * 4 + 2 * (uint64_t)h->sh_cap_out * 4);
     return MPE_OK;
 }
 
@@ -909,6 +986,7 @@ int mpe_kernel_launches(mpe_handle* h, uint64_t* count) {
 
 int mpe_profile(mpe_handle* h, int32_t enable) {
     if (!h) return MPE_ERR_ARG;
+    if (h->have_forward) return MPE_ERR_SEQUENCE;      // both halves of a step are launched the same way
     DeviceGuard guard(h->device);
     CK(h, cudaStreamSynchronize(h->stream));
     for (auto& r : h->prof_recs) { h->event_pool.push_back(r.a); h->event_pool.push_back(r.b); }
@@ -952,9 +1030,8 @@ constexpr int64_t STATIC_MAX_INDICES = MPE_STATIC_MAX_INDICES;
 constexpr int64_t STATIC_MAX_BAGS = MPE_STATIC_MAX_BAGS;
 constexpr int STATIC_MAX_TABLES = MPE_STATIC_MAX_TABLES;
 constexpr size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
-constexpr size_t STATIC_PER_INDEX_ARRAYS = 16;     // u32/i32 arrays of STATIC_MAX_INDICES + 2 entries
 constexpr size_t STATIC_SCRATCH_BYTES =
-    STATIC_PER_INDEX_ARRAYS * align256((STATIC_MAX_INDICES + 2) * 4) +                                 // keys, payloads, per-index and per-row maps
+    2 * align256(2 * (STATIC_MAX_INDICES + 4) * 4) + 12 * align256((STATIC_MAX_INDICES + 4) * 4) +                                 // keys, payloads, per-index and per-row maps
     align256(256 * ((STATIC_MAX_INDICES + SORT_TILE - 1) / SORT_TILE + STATIC_MAX_TABLES + 1) * 4) +   // sort histograms
     align256((256 * ((STATIC_MAX_INDICES + SORT_TILE - 1) / SORT_TILE + STATIC_MAX_TABLES + 1) / SCAN_TILE + 2 +
               STATIC_MAX_INDICES / SCAN_TILE + 2) * 4) +                                               // block sums
@@ -967,6 +1044,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_B
 
 constexpr int MAX_DEVICES = 64;
 unsigned char* g_scratch_addr[MAX_DEVICES] = {};     // device address of g_static_scratch, per device, filled on first use
+std::mutex g_scratch_lock;                           // first calls from several host threads fill the table one at a time
 
 struct Carver {
     unsigned char* p; size_t used = 0;
@@ -984,19 +1062,24 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     if (h->have_forward) return MPE_ERR_SEQUENCE;      // a training step is half done: its backward still needs the probe marks
     if (h->device < 0 || h->device >= MAX_DEVICES) return MPE_ERR_ARG;
     DeviceGuard guard(h->device);
-    if (!g_scratch_addr[h->device]) {
-        // once per device, with that device current: ask the runtime where the array lives on this device
-        void* addr = nullptr;
-        CK(h, cudaGetSymbolAddress(&addr, g_static_scratch));
-        g_scratch_addr[h->device] = static_cast<unsigned char*>(addr);
+    unsigned char* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_scratch_lock);
+        if (!g_scratch_addr[h->device]) {
+            // once per device, with that device current: ask the runtime where the array lives on this device
+            void* addr = nullptr;
+            CK(h, cudaGetSymbolAddress(&addr, g_static_scratch));
+            g_scratch_addr[h->device] = static_cast<unsigned char*>(addr);
+        }
+        scratch = g_scratch_addr[h->device];
     }
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     if (stream != h->stream) { CK(h, cudaStreamSynchronize(h->stream)); h->stream = stream; }
 
     // carve the step's arrays out of the scratch (same roles as the handle's own workspace)
-    Carver c{g_scratch_addr[h->device]};
-    const size_t n = (size_t)STATIC_MAX_INDICES + 2;
-    uint32_t *keyA = c.take<uint32_t>(n), *keyB = c.take<uint32_t>(n), *valA = c.take<uint32_t>(n), *valB = c.take<uint32_t>(n);
+    Carver c{scratch};
+    const size_t n = (size_t)STATIC_MAX_INDICES + 4;
+    uint32_t *sortA = c.take<uint32_t>(2 * n), *sortB = c.take<uint32_t>(2 * n);
     Work w{};
     w.bag_of = c.take<int32_t>(n); w.kidx = c.take<uint32_t>(n); w.occ_loc = c.take<int32_t>(n); w.occ_b = c.take<int32_t>(n);
     w.uniq_row = c.take<int32_t>(n); w.uniq_t = c.take<int32_t>(n); w.seg = c.take<int32_t>(n); w.loc = c.take<int32_t>(n);
@@ -1019,30 +1102,12 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), stream));
     StepArgs av{};
     av.indices = d_indices; av.offsets = d_offsets; av.out = d_out; av.B = batch; av.L = L; av.epoch = h->epoch;
+    const SortBufs sb{sortA, sortB, (int64_t)n, hist, block_sums};
     LAUNCH(h, "prelude", k_prelude<false>, 1, 32, 0, w, T, av);
-    LAUNCH(h, "make_keys", k_make_keys<false>, grid_for(h, bags, 32, 8), 256, 0, s, w, keyA, av);
+    LAUNCH(h, "make_keys", k_make_keys<false>, grid_for(h, bags, 32, 8), 256, 0, s, w, sort_input(sb), av);
     // segmented radix sort, as in mpe_forward, on the carved buffers
-    LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, (const int32_t*)w.table_start, T, w.tile_base, &w.ctr->hist_len,
-           (const uint32_t*)&w.ctr->abort);
-    const int64_t tiles_upper = (total_indices + SORT_TILE - 1) / SORT_TILE + T;
-    const int gsort = grid_for(h, tiles_upper, 1, 5);
-    const int gscan = grid_for(h, 256 * tiles_upper, SCAN_TILE, 8);
-    const int passes = (bits_for((uint32_t)h->max_rows) + 7) / 8;
-    uint32_t *kin = keyA, *kout = keyB, *vin = nullptr, *vout = valB;
-    for (int p = 0; p < passes; ++p) {
-        LAUNCH(h, "sort_hist", k_sort_hist, gsort, SORT_THREADS, 0, (const uint32_t*)kin, (const int32_t*)w.table_start,
-               (const int32_t*)w.tile_base, T, 8 * p, hist);
-        LAUNCH(h, "scan_reduce", k_scan_reduce, gscan, SCAN_THREADS, 0, (const uint32_t*)hist, (const uint32_t*)&w.ctr->hist_len, block_sums);
-        LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, block_sums, (const uint32_t*)&w.ctr->hist_len,
-               (uint32_t)SCAN_TILE, (uint32_t*)nullptr);
-        LAUNCH(h, "scan_apply", k_scan_apply, gscan, SCAN_THREADS, 0, hist, (const uint32_t*)&w.ctr->hist_len, (const uint32_t*)block_sums);
-        LAUNCH(h, "sort_scatter", k_sort_scatter, gsort, SORT_THREADS, 0, (const uint32_t*)kin, (const uint32_t*)vin, kout, vout,
-               (const int32_t*)w.table_start, (const int32_t*)w.tile_base, T, 8 * p, (const uint32_t*)hist);
-        std::swap(kin, kout);
-        vin = vout; vout = (vout == valB) ? valA : valB;
-    }
-    const uint32_t* skey = kin;
-    const uint32_t* spos = vin;
+    const uint32_t *skey = nullptr, *spos = nullptr;
+    seg_sort(h, sb, w.table_start, w.tile_base, &w.ctr->hist_len, &w.ctr->abort, bits_for((uint32_t)h->max_rows), total_indices, &skey, &spos);
     const int gs = grid_for(h, total_indices, SCAN_TILE, 8);
     LAUNCH(h, "unique_count", k_unique<false>, gs, SCAN_THREADS, 0, w, T, skey, block_sums);
     LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);

@@ -6,15 +6,23 @@
 // an 8-bit digit with per-(table, digit, tile) counters, so one pass over the
 // whole array sorts all segments at once and never moves a key out of its
 // segment.  No kernel here waits on another block: a pass is histogram ->
-// prefix sum -> scatter, three ordinary launches.
+// prefix sum -> scatter, three ordinary launches.  A tile is 4096 elements:
+// 16 per thread, ranked by warp (match on the digit, warp-private counters),
+// reordered through shared memory so that global writes are runs.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace mpe {
 
+#ifndef MPE_SORT_ITEMS
+#define MPE_SORT_ITEMS 16      // keys per thread of the scatter kernel (even)
+#endif
+#ifndef MPE_SORT_MINB
+#define MPE_SORT_MINB 4        // resident blocks per SM the scatter kernel is compiled for
+#endif
 constexpr int SORT_THREADS = 256;
-constexpr int SORT_ITEMS = 8;
+constexpr int SORT_ITEMS = MPE_SORT_ITEMS;
 constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;   // keys per block
 constexpr int SCAN_THREADS = 256;
 constexpr int SCAN_ITEMS = 16;
@@ -79,11 +87,14 @@ __device__ __forceinline__ int find_segment(const int32_t* __restrict__ base, in
 }
 
 // ---- pass 1 of 3: per-(table, digit, tile) counts ------------------------------
+// PAIRS: the keys are the .x members of (key, payload) records (every pass but the first)
+template <bool PAIRS>
 __global__ void __launch_bounds__(SORT_THREADS)
 k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base,
             int T, int shift, uint32_t* __restrict__ hist) {
     // one warp per tile: its own 256 counters, eight key loads in flight per lane, no block-wide barrier
     constexpr int WARPS = SORT_THREADS / 32;
+    constexpr int STRIDE = PAIRS ? 2 : 1;
     __shared__ uint32_t cnt[WARPS][256];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int ntiles = tile_base[T];
@@ -99,7 +110,7 @@ k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_s
         for (int32_t i0 = start + lane; i0 < end; i0 += 32 * 8) {
             uint32_t k[8];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) k[q] = i0 + 32 * q < end ? keys[i0 + 32 * q] : 0u;
+            for (int q = 0; q < 8; ++q) k[q] = i0 + 32 * q < end ? keys[(size_t)(i0 + 32 * q) * STRIDE] : 0u;
 #pragma unroll
             for (int q = 0; q < 8; ++q)
                 if (i0 + 32 * q < end) atomicAdd(&cnt[warp][(k[q] >> shift) & 255u], 1u);
@@ -113,72 +124,102 @@ k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_s
 }
 
 // ---- pass 3 of 3: stable scatter ------------------------------------------------
-// vals_in == nullptr means "the payload is the element's position" (first pass).
-__global__ void __launch_bounds__(SORT_THREADS, 5)
-k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
-               uint32_t* __restrict__ keys_out, uint32_t* __restrict__ vals_out,
+// Between passes an element travels as one 8-byte (key, payload) record, so a pass reads and writes it with one
+// instruction each and a digit's run of a tile is one contiguous piece of memory.
+// FIRST: the input is the bare key array and the payload is the element's position.
+// LAST: the output is split into the sorted keys and the sorted payloads (out_keys / out_vals), which is what the
+// kernels after the sort read.
+template <bool FIRST, bool LAST>
+__global__ void __launch_bounds__(SORT_THREADS, MPE_SORT_MINB)
+k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint2* __restrict__ pairs_in, uint2* __restrict__ pairs_out,
+               uint32_t* __restrict__ out_keys, uint32_t* __restrict__ out_vals,
                const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base, int T, int shift,
                const uint32_t* __restrict__ hist_scanned) {
     constexpr int WARPS = SORT_THREADS / 32;
-    __shared__ uint32_t wcnt[WARPS][256];      // per-warp digit counters, then per-warp digit bases
-    __shared__ uint32_t gbase[256];            // first global position of each digit of this tile, later minus its tile-local start
+    __shared__ uint32_t wcnt[WARPS][256];      // per-warp digit counters, then tile-local position of the warp's first key of each digit
+    __shared__ uint32_t goff[256];             // first global position of each digit of this tile minus its tile-local start
     __shared__ uint2 skv[SORT_TILE];
     __shared__ uint32_t scan_tmp[SORT_THREADS / 32 + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t lt = (1u << lane) - 1u;
     const int ntiles = tile_base[T];
+    volatile uint32_t* myc = wcnt[warp];
     for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const int t = find_segment(tile_base, T, tile);
         const int local = tile - tile_base[t];
         const int nt = tile_base[t + 1] - tile_base[t];
         const int32_t start = seg_start[t] + local * SORT_TILE;
         const int32_t count = min(SORT_TILE, seg_start[t + 1] - start);
-        for (int i = threadIdx.x; i < WARPS * 256; i += SORT_THREADS) (&wcnt[0][0])[i] = 0;
-        gbase[threadIdx.x] = hist_scanned[(size_t)256 * tile_base[t] + (size_t)threadIdx.x * nt + local];
-        __syncthreads();
-        // warp w owns elements [w*512, w*512+512) of the tile, item i of lane l is w*512 + i*32 + l,
+        // warp w owns elements [w*32*ITEMS, (w+1)*32*ITEMS) of the tile, item i of lane l is w*32*ITEMS + i*32 + l,
         // so "item order, then lane order" is the original order
-        uint32_t key[SORT_ITEMS], rank[SORT_ITEMS];
+        uint32_t key[SORT_ITEMS], val[SORT_ITEMS];
+        const int e0 = warp * (32 * SORT_ITEMS) + lane;
+        if (e0 - lane + 32 * SORT_ITEMS <= count) {                    // the warp's whole share is inside the tile
 #pragma unroll
-        for (int i = 0; i < SORT_ITEMS; ++i) {
-            const int e = warp * (32 * SORT_ITEMS) + i * 32 + lane;
-            key[i] = e < count ? keys_in[start + e] : 0xffffffffU;
+            for (int i = 0; i < SORT_ITEMS; ++i) {
+                const int e = e0 + i * 32;
+                if (FIRST) { key[i] = keys_in[start + e]; val[i] = (uint32_t)(start + e); }
+                else { const uint2 kv = pairs_in[start + e]; key[i] = kv.x; val[i] = kv.y; }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < SORT_ITEMS; ++i) {
+                const int e = e0 + i * 32;
+                key[i] = 0xffffffffU; val[i] = 0u;                     // padding: digit 255 in every pass, behind every real key
+                if (e < count) {
+                    if (FIRST) { key[i] = keys_in[start + e]; val[i] = (uint32_t)(start + e); }
+                    else { const uint2 kv = pairs_in[start + e]; key[i] = kv.x; val[i] = kv.y; }
+                }
+            }
         }
+        const uint32_t gb = hist_scanned[(size_t)256 * tile_base[t] + (size_t)threadIdx.x * nt + local];   // digit threadIdx.x
+#pragma unroll
+        for (int i = 0; i < 8; ++i) wcnt[warp][i * 32 + lane] = 0;
+        __syncwarp();
+        // stable rank among the warp's keys of the same digit: the counters are the warp's own, so the first lane of each
+        // group of equal digits updates them with plain loads and stores
+        uint32_t rank[SORT_ITEMS / 2];
 #pragma unroll
         for (int i = 0; i < SORT_ITEMS; ++i) {
             const uint32_t dg = (key[i] >> shift) & 255u;
             const uint32_t peers = __match_any_sync(0xffffffffU, dg);
             const int leader = __ffs(peers) - 1;
             uint32_t before = 0;
-            if (lane == leader) before = atomicAdd(&wcnt[warp][dg], (uint32_t)__popc(peers));   // one lane per digit value
+            if (lane == leader) { before = myc[dg]; myc[dg] = before + (uint32_t)__popc(peers); }
             before = __shfl_sync(0xffffffffU, before, leader);
-            rank[i] = before + __popc(peers & ((1u << lane) - 1u));
+            const uint32_t r = before + (uint32_t)__popc(peers & lt);
+            if (i & 1) rank[i >> 1] |= r << 16; else rank[i >> 1] = r;
+            __syncwarp();
         }
         __syncthreads();
         // digit d (= threadIdx.x): exclusive sum over warps, then over digits
-        uint32_t cw[WARPS], tot = 0;
+        uint32_t tot = 0;
 #pragma unroll
-        for (int w = 0; w < WARPS; ++w) { cw[w] = tot; tot += wcnt[w][threadIdx.x]; }
+        for (int w = 0; w < WARPS; ++w) tot += wcnt[w][threadIdx.x];
         uint32_t all;
         const uint32_t ds = block_exclusive_scan<SORT_THREADS>(tot, &all, scan_tmp);
+        uint32_t run = ds;
 #pragma unroll
-        for (int w = 0; w < WARPS; ++w) wcnt[w][threadIdx.x] = ds + cw[w];     // tile-local position of warp w's first key with this digit
-        gbase[threadIdx.x] -= ds;                                              // global position = gbase + tile-local position
+        for (int w = 0; w < WARPS; ++w) {                                      // tile-local position of warp w's first key with this digit
+            const uint32_t c = wcnt[w][threadIdx.x];
+            wcnt[w][threadIdx.x] = run;
+            run += c;
+        }
+        goff[threadIdx.x] = gb - ds;                                           // global position = goff + tile-local position
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < SORT_ITEMS; ++i) {
-            const int e = warp * (32 * SORT_ITEMS) + i * 32 + lane;
             const uint32_t dg = (key[i] >> shift) & 255u;
-            const uint32_t pos = wcnt[warp][dg] + rank[i];
-            skv[pos] = make_uint2(key[i], e < count ? (vals_in ? vals_in[start + e] : (uint32_t)(start + e)) : 0u);
+            const uint32_t r = (i & 1) ? rank[i >> 1] >> 16 : rank[i >> 1] & 0xffffu;
+            skv[wcnt[warp][dg] + r] = make_uint2(key[i], val[i]);
         }
         __syncthreads();
-        // padding keys (0xffffffff, digit 255) follow every real key of the tile, so positions [0,count) are real
+        // padding keys follow every real key of the tile, so positions [0,count) are real
         for (int j = threadIdx.x; j < count; j += SORT_THREADS) {
             const uint2 kv = skv[j];
-            const uint32_t dg = (kv.x >> shift) & 255u;
-            const uint32_t dst = gbase[dg] + (uint32_t)j;
-            keys_out[dst] = kv.x;
-            vals_out[dst] = kv.y;
+            const uint32_t dst = goff[(kv.x >> shift) & 255u] + (uint32_t)j;
+            if (LAST) { out_keys[dst] = kv.x; out_vals[dst] = kv.y; }
+            else pairs_out[dst] = kv;
         }
         __syncthreads();
     }

@@ -32,10 +32,11 @@ def test_config1_all_steps():
     assert info[0][0] == 512 and 0 < info[0][1] <= 512
 
 
-def test_config2_lfu_many_tables():
+def test_config2_all_tables_all_hundred_steps():
     from parity_util import run_parity
     cfg = wl.config(2)
-    run_parity(cfg, 12, check_every=4)
+    assert cfg.steps == 100 and cfg.num_tables == 26
+    run_parity(cfg, cfg.steps, check_every=25)
 
 
 def test_config2_with_the_table_sizes_the_paper_prints():
@@ -266,6 +267,29 @@ def test_host_buffer_step_matches_device_step():
         o.backward(grad.numpy(), cfg.lr, step)
         assert np.array_equal(out, ref)
     compare_state(h, o, cfg, [0, 1], rng)
+    # overlapped: several steps submitted before anything is waited for, batches of different sizes (the staging
+    # buffers regrow in between), pinned inputs; results are those of the same steps run one after the other
+    pending = []
+    step = 3
+    for batch in (64, 64, 200, 32, 64, 64, 64):
+        step += 1
+        cfg.batch = batch
+        idx, off, grad = wl.Stream(cfg, "cpu").batch(step)
+        hb = [x.pin_memory() for x in (idx, off, grad)]
+        out = torch.zeros(batch, cfg.num_tables * cfg.dim).pin_memory()
+        h.step_host_submit(hb[0], hb[1], batch, hb[2], out, cfg.lr, step)
+        pending.append((hb, out, batch, step))
+    h.step_host_wait()
+    for (idx, off, grad), out, batch, stp in pending:
+        ref = o.forward(idx.numpy(), off.numpy(), batch)
+        o.backward(grad.numpy(), cfg.lr, stp)
+        assert np.array_equal(out.numpy(), ref), f"overlapped step {stp}"
+    compare_state(h, o, cfg, [0, 1], rng)
+    from paper_2010_11305_b200 import binding as mpe
+    with pytest.raises(mpe.MpeError) as e:                 # the step number still has to grow
+        h.step_host_submit(hb[0], hb[1], batch, hb[2], out, cfg.lr, step)
+    assert e.value.code == mpe.ERR_SEQUENCE
+    assert h.last_error() == (0, 0)
 
 
 def test_memory_accounting_matches_the_appendix_table():
@@ -286,7 +310,9 @@ def test_memory_accounting_matches_the_appendix_table():
 # Full-size configurations, in the launch configuration the benchmark times.  The oracle follows a
 # sample of the tables (tables are independent); everything observable of those tables is compared.
 # ---------------------------------------------------------------------------------------------
-def _full_size(cfg, tables, steps):
+def _full_size(cfg, tables, steps, check_at=()):
+    """A configuration at its full size in the launch configuration the benchmark times; the oracle follows the
+    sampled tables only.  State is compared at the steps in check_at, at the last step, and again after a flush."""
     from parity_util import make_pair, compare_state
     h, o = make_pair(cfg, tables)
     st = wl.Stream(cfg, "cuda")
@@ -301,6 +327,8 @@ def _full_size(cfg, tables, steps):
         h.backward(grad, cfg.lr, step)
         o.backward(grad.cpu().numpy(), cfg.lr, step)
         assert h.last_error() == (0, 0)
+        if step in check_at:
+            compare_state(h, o, cfg, tables, rng)
     compare_state(h, o, cfg, tables, rng)
     h.flush()
     o.flush()
@@ -308,23 +336,64 @@ def _full_size(cfg, tables, steps):
     return h
 
 
-def test_full_size_config4_sampled_tables():
+def test_full_size_config4_all_twenty_steps():
+    """64 tables x 5M rows, all 20 steps of the configuration; the oracle follows the tables with the largest and the
+    smallest Zipf exponent (the most and the fewest rows on the multi-block gradient path) and one in between."""
     cfg = wl.config(4)
-    h = _full_size(cfg, [0, 37, 63], 3)
+    assert cfg.steps == 20
+    z = np.array(cfg.zipf)
+    tables = sorted({int(z.argmax()), int(z.argmin()), 37})
+    h = _full_size(cfg, tables, cfg.steps, check_at=(3, 10))
     info = h.step_info()
     assert info[0] > 25_000_000 and info[3] > 500      # ~31M indices, thousands of hot rows
+    s = h.stats(tables[0])
+    assert s[4] > 0 and s[5] > 0 and s[6] > 0          # past the fill phase: admissions, evictions and bypasses all happen
     h.close()
 
 
-def test_full_size_config3_sampled_tables():
+def test_full_size_config3_all_fifty_steps():
     cfg = wl.config(3)
-    _full_size(cfg, [0, 5], 4).close()
+    assert cfg.steps == 50
+    _full_size(cfg, [0, 5], cfg.steps, check_at=(4, 25)).close()
 
 
-def test_full_size_config5_points():
-    pts = list(wl.sweep5())
-    for i in (5, 30, 58):
-        _full_size(pts[i], [1], 3).close()
+@pytest.mark.parametrize("point", [1, 6, 11, 19, 30, 40, 53, 58, 63])
+def test_full_size_config5_points_fifty_plus_fifty_steps(point):
+    """Points of the policy/skew sweep at full size, over the 50 warm-up + 50 measured steps the sweep runs: both code
+    widths, both policies, all four cache sizes, uniform indices and every Zipf exponent occur among them."""
+    cfg = list(wl.sweep5())[point]
+    assert cfg.steps == 100
+    _full_size(cfg, [point % 4], cfg.steps, check_at=(50,)).close()
+
+
+def test_launch_mode_cannot_change_between_a_forward_and_its_backward():
+    """Replayed kernels read the step's arguments from device memory, plainly launched ones get them by value: the two
+    halves of a step must be launched the same way, whatever the caller toggles in between."""
+    from parity_util import make_pair, compare_state
+    from paper_2010_11305_b200 import binding as mpe
+    cfg = _cfg(num_rows=[3000, 400], dim=16, bits=4, batch=48, bag=("poisson", 4.0), zipf=[1.1, 0.9], policy=wl.LFU, ways=4,
+               cache_fraction=0.1, seed=12)
+    h, o = make_pair(cfg)
+    rng = np.random.default_rng(0)
+    st = wl.Stream(cfg, "cpu")
+    step = 0
+    for graphs_fwd, toggle in ((True, "graphs"), (False, "graphs"), (True, "profile"), (False, "profile"), (True, None)):
+        step += 1
+        h.use_graphs(graphs_fwd)
+        idx, off, grad = st.batch(step)
+        out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, device="cuda")
+        h.forward(idx.cuda(), off.cuda(), cfg.batch, out)
+        with pytest.raises(mpe.MpeError) as e:
+            if toggle == "profile":
+                h.profile(True)
+            else:
+                h.use_graphs(not graphs_fwd)
+        assert e.value.code == mpe.ERR_SEQUENCE
+        h.backward(grad.cuda(), cfg.lr, step)
+        assert np.array_equal(out.cpu().numpy(), o.forward(idx.numpy(), off.numpy(), cfg.batch))
+        o.backward(grad.numpy(), cfg.lr, step)
+        compare_state(h, o, cfg, [0, 1], rng)
+    assert h.last_error() == (0, 0)
 
 
 def test_graph_replay_and_plain_launches_agree_with_the_oracle():
