@@ -11,7 +11,7 @@ tags and priority values.  It is written independently of the C file: own
 hash, own quantizer, own fused multiply-add (exact rational arithmetic).
 
 The conventions the paper leaves open (hash constants, order of I_U, LFU
-increment, timestamp unit, order of the gradient additions) are the same as in the C oracle;
+increment, timestamp unit, summation tree) are the same as in the C oracle;
 they are what "parity unpinned" refers to there.
 """
 from fractions import Fraction
@@ -121,19 +121,15 @@ def fake_quantize(r, bits, mode, key):
     return out, codes, s, b
 
 
-def merge_sum(terms, samples, block=256):
-    """Duplicate gradients of one row: the terms of each block of `block` consecutive samples are added left to
-    right, then the block sums are added left to right (blocks without a term take no part)."""
-    by_block = {}
-    for t, b in zip(terms, samples):
-        by_block.setdefault(b // block, []).append(t)
-    total = None
-    for blk in sorted(by_block):
-        part = by_block[blk][0].copy()
-        for t in by_block[blk][1:]:
-            part = (part + t).astype(F)
-        total = part if total is None else (total + part).astype(F)
-    return total
+def tree_sum(terms):
+    """Radix-32 tree: up to 32 terms are added left to right; longer lists are cut
+    into consecutive chunks of 32 whose sums are reduced by the same rule."""
+    if len(terms) <= 32:
+        acc = terms[0].copy()
+        for t in terms[1:]:
+            acc = (acc + t).astype(F)
+        return acc
+    return tree_sum([tree_sum(terms[i:i + 32]) for i in range(0, len(terms), 32)])
 
 
 class Emulator:
@@ -183,7 +179,7 @@ class Emulator:
                 if 0 <= i < self.N:
                     where.setdefault(i, []).append(b)
         rows = sorted(where)
-        merged = {i: merge_sum([np.asarray(grad_out[b], F) for b in where[i]], where[i]) for i in rows}
+        merged = {i: tree_sum([np.asarray(grad_out[b], F) for b in where[i]]) for i in rows}
         cached = {i: (self.n > 0 and i in self.I_C[self.h(i)]) for i in rows}
         # priorities: popularity counts every access, recency stamps the cached rows that were used
         for i in rows:

@@ -17,8 +17,7 @@
  *   Conventions (the paper is silent): the counter hash, the set hash, the
  *   order of I_U in Algorithm 2 (hits first, then misses in ascending row id),
  *   timestamps = step number, LFU increment = multiplicity in the batch, the
- *   order in which duplicate gradients are added (by blocks of 256 samples),
- *   row-wise Adagrad's formula, and the
+ *   radix-32 gradient summation tree, row-wise Adagrad's formula, and the
  *   multiplication by 1/scale instead of a division per element.
  */
 #include "mpe_oracle.h"
@@ -200,26 +199,26 @@ void orc_init_row(uint64_t seed, uint32_t table, uint32_t row, int32_t d, float 
 }
 
 /* ------------------------------------------------------------------------ */
-/* Duplicate-gradient merge (Section 5.1): the order of the additions        */
+/* Duplicate-gradient merge (Section 5.1): radix-32 summation tree            */
 /* ------------------------------------------------------------------------ */
-/* The paper says that the gradients of equal rows are merged, not in which order.  The order fixed here: the terms
- * of a row arrive in ascending index position, i.e. by ascending sample; samples are taken in blocks of
- * ORC_SAMPLE_BLOCK consecutive samples (sample >> 8); the terms of one block are added left to right, and the block
- * sums are added left to right in ascending block order (blocks without a term do not take part).  sample[j] is the
- * sample the j-th term belongs to (non-decreasing). */
-void orc_merge_sum(const float* const* terms, const int32_t* sample, int64_t m, int32_t d, float* out) {
-    float* block = (float*)malloc((size_t)d * sizeof(float));
-    int64_t j = 0;
-    int first_block = 1;
-    while (j < m) {
-        const int32_t blk = sample[j] / ORC_SAMPLE_BLOCK;
-        for (int c = 0; c < d; ++c) block[c] = terms[j][c];
-        for (++j; j < m && sample[j] / ORC_SAMPLE_BLOCK == blk; ++j)
-            for (int c = 0; c < d; ++c) block[c] = block[c] + terms[j][c];
-        if (first_block) { for (int c = 0; c < d; ++c) out[c] = block[c]; first_block = 0; }
-        else for (int c = 0; c < d; ++c) out[c] = out[c] + block[c];
+void orc_tree_sum(const float* const* terms, int64_t m, int32_t d, float* out) {
+    if (m <= 32) {
+        for (int c = 0; c < d; ++c) out[c] = terms[0][c];
+        for (int64_t j = 1; j < m; ++j)
+            for (int c = 0; c < d; ++c) out[c] = out[c] + terms[j][c];
+        return;
     }
-    free(block);
+    int64_t nchunk = (m + 31) / 32;
+    float* sums = (float*)malloc((size_t)nchunk * (size_t)d * sizeof(float));
+    const float** ptr = (const float**)malloc((size_t)nchunk * sizeof(float*));
+    for (int64_t k = 0; k < nchunk; ++k) {
+        int64_t len = m - 32 * k < 32 ? m - 32 * k : 32;
+        orc_tree_sum(terms + 32 * k, len, d, sums + k * d);
+        ptr[k] = sums + k * d;
+    }
+    orc_tree_sum(ptr, nchunk, d, out);
+    free(ptr);
+    free(sums);
 }
 
 /* ------------------------------------------------------------------------ */
@@ -544,13 +543,10 @@ int orc_backward(orc* o, const float* grad_out, float lr, int64_t step) {
             while (j < n && occ[j].row == occ[i].row) ++j;
             const int64_t m = j - i;
             const float** terms = (const float**)malloc((size_t)m * sizeof(float*));
-            int32_t* smp = (int32_t*)malloc((size_t)m * sizeof(int32_t));
-            for (int64_t a = 0; a < m; ++a) {  /* ascending position: the sort is stable by construction */
-                smp[a] = bag_of[occ[i + a].p - p0];
-                terms[a] = grad_out + ((int64_t)smp[a] * o->T + t) * d;
-            }
-            orc_merge_sum(terms, smp, m, d, ug + k * d);
-            free(terms); free(smp);
+            for (int64_t a = 0; a < m; ++a)   /* ascending position: the sort is stable by construction */
+                terms[a] = grad_out + ((int64_t)bag_of[occ[i + a].p - p0] * o->T + t) * d;
+            orc_tree_sum(terms, m, d, ug + k * d);
+            free(terms);
             urow[k] = occ[i].row; umult[k] = (int32_t)m;
             ++k; i = j;
         }

@@ -20,8 +20,7 @@
  * and the table mask (equal to a run whose masked tables receive no indices).
  * Parity unpinned (pure conventions, fixed by this build and mirrored on the
  * GPU): the constants of the counter hash, the cache-set hash, INT4 nibble
- * order, argmin tie-breaks, and the order in which duplicate gradients are added
- * (by blocks of 256 samples).
+ * order, argmin tie-breaks, and the radix (32) of the gradient summation tree.
  */
 #ifndef MPE_ORACLE_H
 #define MPE_ORACLE_H
@@ -60,10 +59,8 @@ float    orc_half_to_float(uint16_t h);
 uint16_t orc_float_to_half(float f, int32_t direction);
 void orc_to_half_row(const float* x, int32_t d, int32_t mode, uint32_t rowkey, uint16_t* codes16);
 void orc_init_row(uint64_t seed, uint32_t table, uint32_t row, int32_t d, float lo, float hi, float* x);
-/* Sum of m rows of d floats (terms[j] points to row j, sample[j] is the sample it comes from, non-decreasing): the
- * terms of each block of ORC_SAMPLE_BLOCK consecutive samples left to right, then the block sums left to right. */
-enum { ORC_SAMPLE_BLOCK = 256 };
-void orc_merge_sum(const float* const* terms, const int32_t* sample, int64_t m, int32_t d, float* out);
+/* Radix-32 summation tree over m rows of d floats (terms[j] points to row j). */
+void orc_tree_sum(const float* const* terms, int64_t m, int32_t d, float* out);
 
 /* ---- the stateful step --------------------------------------------------- */
 orc* orc_create(const int64_t* num_rows, int32_t num_tables, int32_t dim, int32_t bits,

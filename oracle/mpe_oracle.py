@@ -49,7 +49,7 @@ _h2f = _sig("orc_half_to_float", C.c_float, C.c_uint16)
 _f2h = _sig("orc_float_to_half", C.c_uint16, C.c_float, C.c_int32)
 _to_half_row = _sig("orc_to_half_row", None, _f32p, C.c_int32, C.c_int32, C.c_uint32, np.ctypeslib.ndpointer(np.uint16, flags="C_CONTIGUOUS"))
 _init_row = _sig("orc_init_row", None, C.c_uint64, C.c_uint32, C.c_uint32, C.c_int32, C.c_float, C.c_float, _f32p)
-_merge_sum = _sig("orc_merge_sum", None, C.POINTER(C.c_void_p), _i32p, C.c_int64, C.c_int32, _f32p)
+_tree_sum = _sig("orc_tree_sum", None, C.POINTER(C.c_void_p), C.c_int64, C.c_int32, _f32p)
 
 _create = _sig("orc_create", C.c_void_p, _i64p, C.c_int32, C.c_int32, C.c_int32, C.c_double, C.c_int32,
                C.c_int32, C.c_int32, C.c_float, C.c_float, C.c_float, C.c_uint64)
@@ -151,17 +151,13 @@ def init_row(seed, table, row, d, lo, hi):
     return x
 
 
-SAMPLE_BLOCK = 256
-
-
-def merge_sum(terms, sample):
-    """Sum of the rows of terms[m, d] in the order fixed for duplicate gradients: sample[j] is the sample term j comes from."""
+def tree_sum(terms):
+    """Radix-32 summation tree over the rows of terms[m, d]."""
     terms = np.ascontiguousarray(terms, np.float32)
-    sample = np.ascontiguousarray(sample, np.int32)
     m, d = terms.shape
     ptrs = (C.c_void_p * m)(*[terms.ctypes.data + i * d * 4 for i in range(m)])
     out = np.zeros(d, np.float32)
-    _merge_sum(ptrs, sample, m, d, out)
+    _tree_sum(ptrs, m, d, out)
     return out
 
 

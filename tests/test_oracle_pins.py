@@ -192,32 +192,25 @@ def test_dedup_example_from_section_5_1():
     del before
 
 
-def test_merge_order_of_duplicate_gradients():
-    """Terms are taken in blocks of 256 consecutive samples: left to right inside a block, then the block sums left
-    to right.  Cancellation cases tell this order from every other one."""
+def test_tree_sum_shape():
     rng = np.random.default_rng(1)
-    for m, B in ((1, 1), (2, 300), (31, 256), (33, 40), (64, 16384), (1000, 500), (1025, 16384), (5000, 700), (33000, 40000)):
+    for m in (1, 2, 31, 32, 33, 64, 65, 1000, 1024, 1025, 1057, 33000):
         terms = rng.normal(0, 1, (m, 4)).astype(F)
-        samples = np.sort(rng.integers(0, B, m)).astype(np.int32)
-        got = orc.merge_sum(terms, samples)
-        # the exact sum in float64 bounds the error; and the order equals the independent Python spelling
+        got = orc.tree_sum(terms)
+        # exact sum in float64 bounds the error; and the tree equals the independent Python spelling
         assert np.allclose(got, terms.astype(np.float64).sum(0), rtol=0, atol=1e-3 * np.sqrt(m))
-        if m <= 5000:
-            assert np.array_equal(got, emu.merge_sum([t for t in terms], [int(b) for b in samples]))
-    one = lambda vals, smp: orc.merge_sum(np.array(vals, F)[:, None], np.array(smp, np.int32))[0]
-    # inside one block the order is plain left to right
-    assert one([1e8, 1.0, -1e8, 1.0], [0, 3, 3, 255]) == F(F(F(F(1e8) + F(1.0)) + F(-1e8)) + F(1.0)) == F(1.0)
-    # the same terms in two blocks: (1e8 + 1) + (-1e8 + 1) = 1e8 + (-1e8) = 0
-    assert one([1e8, 1.0, -1e8, 1.0], [0, 255, 256, 300]) == F(0.0)
-    # 2^24 swallows ones that meet it one by one, but not a block that has summed to 40 first
-    assert one([2 ** 24] + [1.0] * 40, [0] * 41) == F(2 ** 24)
-    assert one([2 ** 24] + [1.0] * 40, [0] + [256] * 40) == F(2 ** 24 + 40)
-    assert one([2 ** 24] + [1.0] * 40, [0] + list(range(256, 256 + 40 * 256, 256))) == F(2 ** 24)     # forty blocks of a single one
-    # block boundaries sit at multiples of 256 samples, wherever the terms fall
-    assert one([2 ** 24, 1.0, 1.0], [255, 256, 511]) == F(2 ** 24 + 2)
-    assert one([2 ** 24, 1.0, 1.0], [254, 255, 256]) == F(2 ** 24)
-    # a block sum starts from its first term, the total from the first block sum: the sign of a zero survives
-    assert np.signbit(one([-0.0], [7])) and np.signbit(one([-0.0, -0.0], [7, 300]))
+        if m <= 1100:
+            assert np.array_equal(got, emu.tree_sum([t for t in terms]))
+    # up to 32 terms the order is plain left to right
+    t = np.array([[1e8], [1.0], [-1e8], [1.0]], F)
+    assert orc.tree_sum(t)[0] == F(F(F(F(1e8) + F(1.0)) + F(-1e8)) + F(1.0))
+    # 33 terms: first 32 are summed, then the 33rd is added to that sum
+    t = np.ones((33, 1), F)
+    t[0] = 2 ** 24
+    assert orc.tree_sum(t)[0] == F(2 ** 24) + F(1.0)      # 31 ones are lost one by one, the last one too
+    t = np.ones((64, 1), F)
+    t[0] = 2 ** 24
+    assert orc.tree_sum(t)[0] == F(2 ** 24 + 32)          # the second chunk sums to 32 before it meets 2^24
 
 
 # ------------------------------------------- Algorithm 2 by hand (P3) ----
