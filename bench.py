@@ -243,10 +243,18 @@ def run_ours(args, cfg, rank, world, local_rank):
 
     counter = [0]       # the step number: strictly increasing over the handle's life
 
+    # The next batch is sorted and de-duplicated on a second stream while the current step runs (mpe_prepare): that
+    # part of a step needs the indices only.  Every timed step prepares its successor, so the work of K batches is
+    # inside the region that times K steps.
+    side = torch.cuda.Stream(dev)
+    ahead = not args.no_prepare
+
     def step(i):
         idx, off, grad = batches[i]
         counter[0] += 1
         h.forward(idx, off, cfg.batch, out, sp)
+        if ahead and i + 1 < len(batches):
+            h.prepare(batches[i + 1][0], batches[i + 1][1], cfg.batch, side.cuda_stream)
         h.backward(grad, cfg.lr, counter[0])
 
     # Small steps are replayed from CUDA graphs, which per-kernel event records would break up: for them the timed
@@ -353,6 +361,7 @@ def run_ours(args, cfg, rank, world, local_rank):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": describe(cfg), "l2": "inputs larger than L2; a new batch every step",
                    "launch": "CUDA graph replay (per-kernel times from a second, plainly launched pass)" if graph_sized else "plain launches",
+                   "next_batch": "sorted ahead on a second stream (mpe_prepare) while the current step runs" if ahead and not graph_sized else "not prepared ahead",
                    "sharding": "each rank trains its own tables (no data-path collective)" if world > 1 else "one GPU"},
         "clocks": clocks,
         "e2e": {"value": e2e_rows / e2e_s if e2e_s > 0 else None, "unit": "rows/s", "h2d_bytes_per_step": h2d,
@@ -556,6 +565,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prepare", action="store_true", help="do not sort the next batch ahead of time (mpe_prepare)")
     ap.add_argument("--sweep5", action="store_true", help="run every point of the policy/skew sweep (configuration 5): one JSON line per point")
     ap.add_argument("--tiering", action="store_true", help="forward/backward effective bandwidth vs hit rate, table in HBM and in host memory")
     ap.add_argument("--sweep-assoc", action="store_true", help="associativity sweep (1..32 ways, LRU and LFU) on configuration 5's shape")

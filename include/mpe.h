@@ -98,6 +98,23 @@ int mpe_reserve(mpe_handle* h, int32_t max_batch, int64_t max_total_indices);
 int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch,
                 int64_t total_indices, float* d_out, void* cuda_stream);
 
+/*
+ * Optional: start on the NEXT batch while the current step still runs.  The first part of a forward pass -- sorting the
+ * indices and merging duplicates (Section 5.1) -- needs the indices only, not the tables, the cache or the policy state,
+ * and its kernels leave most of the GPU idle.  mpe_prepare enqueues that part for the given batch on `cuda_stream`
+ * (any stream on which the indices and offsets are ready; typically not the stream of the training step) into a second
+ * workspace of the handle.  A later mpe_forward / mpe_forward_routed with the same d_indices, d_offsets, batch and
+ * total_indices takes the result over (it waits for it on its own stream) and only looks up the tags and pools;
+ * results are bit-identical with and without the call.  Layouts as in mpe_forward; the two buffers must stay
+ * unchanged until that forward.  One batch can be prepared at a time; a forward with other arguments discards it.
+ * The call does nothing (and returns MPE_OK) when the batch does not fit the workspace reserved with mpe_reserve, or
+ * when steps of this size are replayed from a CUDA graph.  The first call allocates the second workspace
+ * (cudaMalloc; as large as the first, see mpe_workspace_bytes).
+ * Typical loop:  forward(k); prepare(k+1, other_stream); backward(k); forward(k+1); ...
+ */
+int mpe_prepare(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch, int64_t total_indices,
+                void* cuda_stream);
+
 /* ---- Tables partitioned over several GPUs (Section 1: embeddings are placed model-parallel, with no replication) ----
  * Each rank owns some of the tables and sees the whole batch's indices for them; sample b of a batch of `batch` samples
  * belongs to rank b / (batch / n_ranks).  After the forward pass every rank needs the pooled vectors of ITS samples for ALL
@@ -228,7 +245,7 @@ int mpe_stats(mpe_handle* h, int32_t table, uint64_t* out8);
  * timestamps, optimizer state, the FP32 table this replaces}. */
 int mpe_memory_bytes(mpe_handle* h, uint64_t* out6);
 /* Device memory the handle holds beyond the model state: out2 = {bytes of the per-step workspace (sized by
- * mpe_reserve or by the largest batch seen), bytes of the two staging sets of mpe_step_host / _submit}. */
+ * mpe_reserve or by the largest batch seen; twice that once mpe_prepare has been used), bytes of the two staging sets of mpe_step_host / _submit}. */
 int mpe_workspace_bytes(mpe_handle* h, uint64_t* out2);
 /* Geometry of table `table`'s cache. */
 int mpe_cache_geometry(mpe_handle* h, int32_t table, int32_t* n_sets, int32_t* ways);

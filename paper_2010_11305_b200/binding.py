@@ -22,7 +22,7 @@ OK, ERR_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_SEQUENCE, ERR_INDEX, ERR_OFFSETS, ER
 STATIC_MAX_INDICES, STATIC_MAX_BAGS, STATIC_MAX_TABLES = 32768, 32768, 64
 
 EXPORTS = [
-    "mpe_create", "mpe_create_placed", "mpe_reserve", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_set_rounding", "mpe_step_host", "mpe_step_host_submit", "mpe_step_host_wait", "mpe_flush", "mpe_destroy",
+    "mpe_create", "mpe_create_placed", "mpe_reserve", "mpe_prepare", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_set_rounding", "mpe_step_host", "mpe_step_host_submit", "mpe_step_host_wait", "mpe_flush", "mpe_destroy",
     "mpe_last_error", "mpe_stats", "mpe_memory_bytes", "mpe_workspace_bytes", "mpe_cache_geometry", "mpe_step_info", "mpe_export_rows",
     "mpe_export_cache", "mpe_export_aux", "mpe_use_graphs", "mpe_kernel_launches", "mpe_profile", "mpe_profile_read",
     "mpe_forward_routed", "mpe_gather_grad", "mpe_peer_buffer_alloc", "mpe_peer_buffer_open", "mpe_peer_buffer_close", "mpe_peer_buffer_free",
@@ -47,6 +47,7 @@ _lib.mpe_create.argtypes = [C.POINTER(_vp), C.POINTER(TableSpec), _i32, _i32, _f
 _lib.mpe_create_placed.argtypes = [C.POINTER(_vp), C.POINTER(TableSpec), _i32, _i32, _f64, _i32, _i32, _i32, _f32, _f32, _f32, _u64, _i32, _i32]
 _lib.mpe_reserve.argtypes = [_vp, _i32, _i64]
 _lib.mpe_forward.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp]
+_lib.mpe_prepare.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp]
 _lib.mpe_forward_static.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp]
 _lib.mpe_backward.argtypes = [_vp, _vp, _f32, _i64]
 _lib.mpe_step_host.argtypes = [_vp, _vp, _vp, _i32, _i64, _vp, _vp, _f32, _i64]
@@ -132,6 +133,10 @@ class Mpe:
     # ---- the step -------------------------------------------------------------------------
     def reserve(self, max_batch, max_total_indices):
         _check(_lib.mpe_reserve(self._h, max_batch, max_total_indices), "mpe_reserve")
+
+    def prepare(self, d_indices, d_offsets, batch, stream=None):
+        """Sort and de-duplicate the next batch on `stream` while the current step runs; the forward of that batch takes it over."""
+        _check(_lib.mpe_prepare(self._h, _ptr(d_indices), _ptr(d_offsets), batch, d_indices.numel(), stream), "mpe_prepare")
 
     def forward(self, d_indices, d_offsets, batch, d_out, stream=None):
         _check(_lib.mpe_forward(self._h, _ptr(d_indices), _ptr(d_offsets), batch, d_indices.numel(), _ptr(d_out),

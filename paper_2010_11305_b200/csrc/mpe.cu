@@ -41,6 +41,22 @@ struct mpe_handle {
     int64_t sort_n = 0;
     uint32_t *hist = nullptr, *block_sums = nullptr;
     std::vector<void*> ws_allocs;
+    cudaEvent_t ev_free = nullptr;          // recorded behind the last kernel that uses this workspace
+    // A second workspace, allocated on the first mpe_prepare: the next batch is sorted and de-duplicated there while the
+    // kernels of the current step still run.  `alt` holds exactly the members above that belong to a workspace.
+    struct WsSet {
+        Work wk{};
+        uint32_t *sortA = nullptr, *sortB = nullptr, *hist = nullptr, *block_sums = nullptr;
+        int64_t sort_n = 0;
+        const uint32_t *skey = nullptr, *spos = nullptr;
+        std::vector<void*> allocs;
+        cudaEvent_t ev_free = nullptr;
+        uint64_t bytes = 0;
+    } alt;
+    bool prepared = false;                  // `alt` holds a sorted batch that the next forward may take over
+    StepArgs prep_args{};                   // ... of these inputs
+    cudaEvent_t ev_prep = nullptr;
+    cudaStream_t prep = nullptr;            // mpe_step_host_submit prepares on this stream
     // staging for mpe_step_host / mpe_step_host_submit: two slots, so that the copies of one step run next to the kernels of another
     struct HostSlot {
         int32_t *idx = nullptr, *off = nullptr; float *grad = nullptr, *out = nullptr;
@@ -138,16 +154,47 @@ void drop_graphs(mpe_handle* h) {
     h->x_fwd = h->x_bwd = nullptr; h->g_fwd = h->g_bwd = nullptr; h->n_fwd = h->n_bwd = nullptr;
 }
 
-void free_workspace(mpe_handle* h) {
-    drop_graphs(h);                       // they hold the workspace's addresses
+// the current workspace and the other one change places
+void swap_sets(mpe_handle* h) {
+    std::swap(h->wk, h->alt.wk);
+    std::swap(h->sortA, h->alt.sortA); std::swap(h->sortB, h->alt.sortB);
+    std::swap(h->hist, h->alt.hist); std::swap(h->block_sums, h->alt.block_sums);
+    std::swap(h->sort_n, h->alt.sort_n);
+    std::swap(h->skey, h->alt.skey); std::swap(h->spos, h->alt.spos);
+    std::swap(h->ws_allocs, h->alt.allocs);
+    std::swap(h->ev_free, h->alt.ev_free);
+    std::swap(h->ws_bytes, h->alt.bytes);
+}
+
+void free_set(mpe_handle* h) {
     for (void* p : h->ws_allocs) cudaFree(p);
     h->ws_allocs.clear();
+    h->wk = Work{};
+    h->ws_bytes = 0;
+}
+
+void free_workspace(mpe_handle* h) {
+    drop_graphs(h);                       // they hold the workspace's addresses
+    free_set(h);
+    swap_sets(h); free_set(h); swap_sets(h);
+    h->prepared = false;
     h->cap_L = 0; h->cap_bags = 0;
 }
 
+int alloc_set(mpe_handle* h, int64_t L, int64_t bags);
+
 int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
-    // everything a step needs between its first and last kernel, sized for L indices
     free_workspace(h);
+    int rc = alloc_set(h, L, bags);
+    if (rc != MPE_OK) return rc;
+    h->cap_L = L; h->cap_bags = bags;
+    return MPE_OK;
+}
+
+int alloc_set(mpe_handle* h, int64_t L, int64_t bags) {
+    // everything a step needs between its first and last kernel, sized for L indices
+    (void)bags;
+    free_set(h);
     auto* tr = &h->ws_allocs;
     const int T = h->T;
     const int64_t n = L + 1;
@@ -177,8 +224,7 @@ int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
     const int64_t max_tasks = hot_capacity(L);
     A(w.task_k, max_tasks); A(w.partial, max_tasks * h->dim); A(w.hot_k, max_tasks);
 #undef A
-    CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), h->stream));
-    h->cap_L = L; h->cap_bags = bags;
+    CK(h, cudaMemset(w.ctr, 0, sizeof(Counters)));
     return MPE_OK;
 }
 
@@ -318,6 +364,9 @@ int mpe_create_placed(mpe_handle** out, const mpe_table_spec* tables, int32_t nu
         cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess ||
         cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking) != cudaSuccess ||
         cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&h->prep, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_free, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_prep, cudaEventDisableTiming) != cudaSuccess ||
         false) { delete h; return MPE_ERR_CUDA; }
     for (auto& sl : h->slot)
         for (cudaEvent_t* e : {&sl.ev_idx, &sl.ev_grad, &sl.ev_fwd, &sl.ev_done, &sl.ev_down})
@@ -402,6 +451,7 @@ int mpe_reserve(mpe_handle* h, int32_t max_batch, int64_t max_total_indices) {
     if (max_total_indices <= h->cap_L && bags <= h->cap_bags && h->wk.ctr) return MPE_OK;
     if (h->have_forward) return MPE_ERR_SEQUENCE;     // a pending backward still needs the old workspace
     CK(h, cudaStreamSynchronize(h->stream));
+    if (h->ev_prep) CK(h, cudaEventSynchronize(h->ev_prep));       // so does a batch that is being prepared
     return alloc_workspace(h, std::max(max_total_indices, h->cap_L), std::max(bags, h->cap_bags));
 }
 
@@ -411,11 +461,11 @@ namespace {
 
 // Launch sizes follow L_grid / bags_grid (upper bounds: every kernel walks its range with a grid stride and reads the
 // true sizes from device memory), so one captured graph serves every batch that fits the workspace.
-int enqueue_forward(mpe_handle* h, int64_t L_grid, int64_t bags_grid, bool ind) {
+// First half of forward, which needs the indices only (no table, cache or policy state): keys, sort, distinct rows.
+void enqueue_index_chain(mpe_handle* h, int64_t L_grid, int64_t bags_grid, bool ind, const StepArgs& av) {
     const State& s = h->st;
     Work& w = h->wk;
     const int T = h->T;
-    const StepArgs av = h->args;
     LAUNCH(h, "prelude", (ind ? k_prelude<true> : k_prelude<false>), 1, 32, 0, w, T, av);
     const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->hist, h->block_sums};
     LAUNCH(h, "make_keys", (ind ? k_make_keys<true> : k_make_keys<false>), grid_for(h, bags_grid, 32, 8), 256, 0, s, w, sort_input(sb), av);
@@ -427,7 +477,12 @@ int enqueue_forward(mpe_handle* h, int64_t L_grid, int64_t bags_grid, bool ind) 
     LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);
     LAUNCH(h, "unique_write", k_unique<true>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
     LAUNCH(h, "ustart", k_ustart, 1, 256, 0, w, T);
-    // tag lookup, then fetch + pool
+}
+
+// Second half: tag lookup, then fetch + pool.
+void enqueue_lookup(mpe_handle* h, int64_t L_grid, int64_t bags_grid, bool ind, const StepArgs& av) {
+    const State& s = h->st;
+    Work& w = h->wk;
     LAUNCH(h, "probe", (ind ? k_probe<true> : k_probe<false>), grid_for(h, L_grid, 256, 8), 256, 0, s, w, av);
     LAUNCH(h, "broadcast", (ind ? k_broadcast<true> : k_broadcast<false>), grid_for(h, L_grid, 256, 8), 256, 0, s, w, h->spos, av);
     const int gp = grid_for(h, bags_grid, 256 / s.lanes, 8);
@@ -436,6 +491,12 @@ int enqueue_forward(mpe_handle* h, int64_t L_grid, int64_t bags_grid, bool ind) 
         auto kern = ind ? k_pool<BITS, LANES, true> : k_pool<BITS, LANES, false>;
         LAUNCH(h, "pool", kern, gp, 256, 0, s, w, av);
     });
+}
+
+int enqueue_forward(mpe_handle* h, int64_t L_grid, int64_t bags_grid, bool ind) {
+    const StepArgs av = h->args;
+    enqueue_index_chain(h, L_grid, bags_grid, ind, av);
+    enqueue_lookup(h, L_grid, bags_grid, ind, av);
     return check_launch(h);
 }
 
@@ -556,9 +617,57 @@ int forward_impl(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offse
             return MPE_OK;
         }
     }
-    rc = enqueue_forward(h, total_indices, bags, false);
+    if (h->prepared && h->prep_args.indices == d_indices && h->prep_args.offsets == d_offsets && h->prep_args.B == batch &&
+        h->prep_args.L == L) {
+        // the batch was sorted and de-duplicated ahead of time in the other workspace: it becomes the current one
+        h->prepared = false;
+        swap_sets(h);
+        CK(h, cudaStreamWaitEvent(h->stream, h->ev_prep, 0));
+        enqueue_lookup(h, total_indices, bags, false, h->args);
+        rc = check_launch(h);
+    } else {
+        h->prepared = false;                 // whatever was prepared was for another batch
+        rc = enqueue_forward(h, total_indices, bags, false);
+    }
     if (rc != MPE_OK) return rc;
+    if (h->ev_free) CK(h, cudaEventRecord(h->ev_free, h->stream));
     h->have_forward = true; h->fwd_replayed = false;
+    return MPE_OK;
+}
+
+// see mpe_prepare in mpe.h
+int prepare_impl(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch, int64_t total_indices,
+                 cudaStream_t stream) {
+    const int64_t bags = (int64_t)h->T * batch;
+    h->prepared = false;
+    // only what fits the reserved workspace, and only steps that are launched plainly (replayed steps are bound by launch
+    // latency, not by their kernels): otherwise the forward simply does all of its work itself
+    if (total_indices > h->cap_L || bags > h->cap_bags || !h->wk.ctr || may_use_graph(h)) return MPE_OK;
+    if (!h->alt.wk.ctr) {                    // first use: the second workspace
+        swap_sets(h);
+        int rc = alloc_set(h, h->cap_L, h->cap_bags);
+        if (rc == MPE_OK && !h->ev_free && cudaEventCreateWithFlags(&h->ev_free, cudaEventDisableTiming) != cudaSuccess) rc = MPE_ERR_CUDA;
+        if (rc != MPE_OK) free_set(h);
+        swap_sets(h);
+        if (rc != MPE_OK) return rc;
+    }
+    StepArgs av{};
+    av.indices = d_indices; av.offsets = d_offsets; av.B = batch; av.L = (uint32_t)total_indices;
+    cudaStream_t user = h->stream;
+    swap_sets(h);
+    h->stream = stream;
+    cudaError_t e = h->ev_free ? cudaStreamWaitEvent(stream, h->ev_free, 0) : cudaSuccess;   // the step that used this workspace last has finished
+    if (e == cudaSuccess) {
+        enqueue_index_chain(h, total_indices, bags, false, av);
+        e = cudaEventRecord(h->ev_prep, stream);
+    }
+    int rc = check_launch(h);
+    h->stream = user;
+    swap_sets(h);
+    if (e != cudaSuccess) { h->last_cuda_error = (int)e; return MPE_ERR_CUDA; }
+    if (rc != MPE_OK) return rc;
+    h->prepared = true;
+    h->prep_args = av;
     return MPE_OK;
 }
 
@@ -592,6 +701,14 @@ int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offset
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     if (stream != h->stream) { CK(h, cudaStreamSynchronize(h->stream)); h->stream = stream; }
     return forward_impl(h, d_indices, d_offsets, batch, total_indices, d_out, nullptr);
+}
+
+int mpe_prepare(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch, int64_t total_indices,
+                void* cuda_stream) {
+    if (!h || !d_offsets || batch < 0 || total_indices < 0 || total_indices > 0x7ffffff0LL) return MPE_ERR_ARG;
+    if (total_indices > 0 && !d_indices) return MPE_ERR_ARG;
+    DeviceGuard guard(h->device);
+    return prepare_impl(h, d_indices, d_offsets, batch, total_indices, (cudaStream_t)cuda_stream);
 }
 
 int mpe_forward_routed(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch, int64_t total_indices,
@@ -700,6 +817,7 @@ int mpe_backward(mpe_handle* h, const float* d_grad_out, float lr, int64_t step)
         rc = enqueue_backward(h, h->L, false);
         if (rc != MPE_OK) return rc;
     }
+    if (h->ev_free) CK(h, cudaEventRecord(h->ev_free, h->stream));
     h->have_forward = false;
     h->last_step = step;
     ++h->steps;
@@ -765,9 +883,14 @@ int mpe_step_host_submit(mpe_handle* h, const int32_t* h_indices, const int32_t*
     CK(h, cudaEventRecord(sl.ev_idx, h->copy_in));
     if (nout) CK(h, cudaMemcpyAsync(sl.grad, h_grad_out, sizeof(float) * nout, cudaMemcpyHostToDevice, h->copy_in));
     CK(h, cudaEventRecord(sl.ev_grad, h->copy_in));
+    // the part of forward that needs the indices only starts as soon as they have arrived, beside whatever the previous
+    // step still has to do
+    CK(h, cudaStreamWaitEvent(h->prep, sl.ev_idx, 0));
+    int rc = prepare_impl(h, sl.idx, sl.off, batch, total_indices, h->prep);
+    if (rc != MPE_OK) { cudaStreamSynchronize(h->copy_in); return rc; }
     CK(h, cudaStreamWaitEvent(st, sl.ev_idx, 0));
     if (sl.used) CK(h, cudaStreamWaitEvent(st, sl.ev_down, 0));           // the slot's previous output has left the device
-    int rc = mpe_forward(h, sl.idx, sl.off, batch, total_indices, sl.out, (void*)st);
+    rc = mpe_forward(h, sl.idx, sl.off, batch, total_indices, sl.out, (void*)st);
     if (rc != MPE_OK) { cudaStreamSynchronize(h->copy_in); return rc; }
     CK(h, cudaEventRecord(sl.ev_fwd, st));
     CK(h, cudaStreamWaitEvent(h->copy_out, sl.ev_fwd, 0));
@@ -819,6 +942,8 @@ int mpe_destroy(mpe_handle* h) {
     if (h->cap) cudaStreamDestroy(h->cap);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->prep) { cudaStreamSynchronize(h->prep); cudaStreamDestroy(h->prep); }
+    for (cudaEvent_t e : {h->ev_free, h->alt.ev_free, h->ev_prep}) if (e) cudaEventDestroy(e);
     if (h->copy_in) { cudaStreamSynchronize(h->copy_in); cudaStreamDestroy(h->copy_in); }
     if (h->copy_out) { cudaStreamSynchronize(h->copy_out); cudaStreamDestroy(h->copy_out); }
     for (auto& sl : h->slot) {
@@ -845,9 +970,15 @@ int mpe_last_error(mpe_handle* h, int32_t* code, int64_t* detail) {
     CK(h, cudaStreamSynchronize(h->stream));
     Counters c;
     CK(h, cudaMemcpy(&c, h->wk.ctr, sizeof(c), cudaMemcpyDeviceToHost));
+    CK(h, cudaMemset(&h->wk.ctr->err[0], 0, sizeof(c.err)));
+    if (h->alt.wk.ctr && !h->prepared) {     // steps alternate between the two workspaces: conditions seen in either count
+        Counters c2;                         // (a batch that is prepared but not yet taken over reports with its own step)
+        CK(h, cudaMemcpy(&c2, h->alt.wk.ctr, sizeof(c2), cudaMemcpyDeviceToHost));
+        CK(h, cudaMemset(&h->alt.wk.ctr->err[0], 0, sizeof(c2.err)));
+        c.err[ERR_OFFSETS] += c2.err[ERR_OFFSETS]; c.err[ERR_INDEX] += c2.err[ERR_INDEX];
+    }
     if (c.err[ERR_OFFSETS]) { *code = MPE_ERR_OFFSETS; *detail = (int64_t)c.err[ERR_OFFSETS]; }
     else if (c.err[ERR_INDEX]) { *code = MPE_ERR_INDEX; *detail = (int64_t)c.err[ERR_INDEX]; }
-    CK(h, cudaMemset(&h->wk.ctr->err[0], 0, sizeof(c.err)));
     return MPE_OK;
 }
 
@@ -877,7 +1008,7 @@ int mpe_memory_bytes(mpe_handle* h, uint64_t* out6) {
 
 int mpe_workspace_bytes(mpe_handle* h, uint64_t* out2) {
     if (!h || !out2) return MPE_ERR_ARG;
-    out2[0] = h->ws_bytes;
+    out2[0] = h->ws_bytes + h->alt.bytes;
     out2[1] = 2 * ((uint64_t)h->sh_cap_L * 4 + (uint64_t)h->sh_cap_off * 4 + 2 * (uint64_t)h->sh_cap_out * 4);
     return MPE_OK;
 }

@@ -366,6 +366,49 @@ def test_full_size_config5_points_fifty_plus_fifty_steps(point):
     _full_size(cfg, [point % 4], cfg.steps, check_at=(50,)).close()
 
 
+def test_batches_prepared_ahead_give_the_same_results():
+    """mpe_prepare sorts the next batch on another stream while the current step runs; the forward of that batch takes
+    the result over.  Prepared, unprepared, discarded (other batch than the one prepared) and ignored (does not fit the
+    reservation) batches in one run, all equal to the oracle; ids outside a table in a prepared batch are reported."""
+    from parity_util import make_pair, compare_state
+    from paper_2010_11305_b200 import binding as mpe
+    cfg = _cfg(num_rows=[30000, 900, 40], dim=64, bits=4, batch=512, bag=("poisson", 9.0), zipf=[1.1, 0.9, None], policy=wl.LFU, ways=8,
+               cache_fraction=0.05, seed=21)
+    h, o = make_pair(cfg)
+    h.use_graphs(False)                                  # replayed steps ignore the call: this test is about the plain path
+    st = wl.Stream(cfg, "cpu")
+    rng = np.random.default_rng(0)
+    side = torch.cuda.Stream()
+    steps = 9
+    batches = [st.batch(s) for s in range(1, steps + 2)]
+    batches[4][0][::50] = 30000                          # step 5's batch has ids outside its tables
+    dev = [(i.cuda(), f.cuda(), g.cuda()) for i, f, g in batches]
+    h.reserve(cfg.batch, max(b[0].numel() for b in batches[:7]))
+    torch.cuda.synchronize()
+    mode = ["prepare", "prepare", "none", "prepare", "wrong", "prepare", "prepare", "too_large", "prepare"]
+    for k in range(steps):
+        idx, off, grad = dev[k]
+        out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, device="cuda")
+        h.forward(idx, off, cfg.batch, out)
+        nxt = mode[k]                                    # what happens for step k + 1 while step k runs
+        if nxt in ("prepare", "too_large"):
+            h.prepare(dev[k + 1][0], dev[k + 1][1], cfg.batch, side.cuda_stream)
+        elif nxt == "wrong":
+            h.prepare(dev[k][0], dev[k][1], cfg.batch, side.cuda_stream)
+        h.backward(grad, cfg.lr, k + 1)
+        ref = o.forward(batches[k][0].numpy(), batches[k][1].numpy(), cfg.batch)
+        o.backward(batches[k][2].numpy(), cfg.lr, k + 1)
+        assert np.array_equal(out.cpu().numpy(), ref), f"step {k + 1}"
+        if k == 4:
+            code, detail = h.last_error()
+            assert code == mpe.ERR_INDEX and detail == int((batches[4][0] == 30000).sum())
+        if k % 3 == 2 or k == steps - 1:
+            compare_state(h, o, cfg, [0, 1, 2], rng)
+    assert h.last_error() == (0, 0)
+    one, _ = h.workspace_bytes()
+    assert one > 0
+
+
 def test_launch_mode_cannot_change_between_a_forward_and_its_backward():
     """Replayed kernels read the step's arguments from device memory, plainly launched ones get them by value: the two
     halves of a step must be launched the same way, whatever the caller toggles in between."""
