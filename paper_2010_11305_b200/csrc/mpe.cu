@@ -212,12 +212,13 @@ int alloc_set(mpe_handle* h, int64_t L, int64_t bags) {
     A(h->sortA, 2 * h->sort_n); A(h->sortB, 2 * h->sort_n);
     const int64_t max_tiles = (L + SORT_TILE - 1) / SORT_TILE + T + 1;
     A(h->hist, 256 * max_tiles);
-    A(h->block_sums, std::max<int64_t>(256 * max_tiles, n) / SCAN_TILE + 2);
+    A(h->block_sums, std::max<int64_t>(256 * max_tiles, n) / std::min<int64_t>(SCAN_TILE, PRI_CHUNK) + 2);
     A(w.ctr, 1); A(w.args, 1);
     A(w.table_start, T + 1); A(w.tile_base, T + 1); A(w.ustart, T + 1); A(w.ctile_base, T + 1);
     A(w.bag_of, n); A(w.kidx, n); A(w.occ_loc, n); A(w.occ_b, n);
     A(w.uniq_row, nu); A(w.uniq_t, nu); A(w.seg, nu + 1); A(w.loc, nu); A(w.final_loc, nu);
-    A(w.hot_base, nu); A(w.uset, nu);
+    A(w.hot_base, nu); A(w.uset, nu); A(w.cand_key, nu); A(w.cand_cnt, T); A(w.cstart, T + 1);
+    CK(h, cudaMemset(w.cand_cnt, 0, sizeof(int32_t) * T));
     // written and read by backward only, at most one entry per distinct row: they take the place of per-index arrays
     // that only forward uses
     w.victim = w.bag_of; w.defer_k = reinterpret_cast<int32_t*>(w.kidx); w.heads = w.occ_loc;
@@ -249,7 +250,7 @@ uint32_t* sort_input(const SortBufs& b) { return b.B; }
 // stable sort of every segment [seg_start[t], seg_start[t+1]) by the low `key_bits` bits of the key, the payload being
 // the element's position before the sort; *skey / *sval receive where the sorted keys / payloads are
 void seg_sort(mpe_handle* h, const SortBufs& b, const int32_t* seg_start, int32_t* tile_base, uint32_t* hist_len, const uint32_t* abort_flag,
-              int key_bits, int64_t n_upper, const uint32_t** skey, const uint32_t** sval) {
+              int key_bits, int64_t n_upper, const uint32_t** skey, const uint32_t** sval, bool input_pairs = false) {
     const int T = h->T;
     LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, seg_start, T, tile_base, hist_len, abort_flag);
     const int64_t max_tiles = (n_upper + SORT_TILE - 1) / SORT_TILE + T;
@@ -257,8 +258,8 @@ void seg_sort(mpe_handle* h, const SortBufs& b, const int32_t* seg_start, int32_
     const int gh = grid_for(h, max_tiles, SORT_THREADS / 32, 8);
     const int passes = (key_bits + 7) / 8;
     for (int p = 0; p < passes; ++p) {
-        const bool first = p == 0, last = p == passes - 1;
-        uint32_t* src = first ? b.B : ((p & 1) ? b.A : b.B);      // pass p writes A when p is even, B when p is odd
+        const bool first = p == 0 && !input_pairs, last = p == passes - 1;    // input_pairs: B holds (key, payload) records already
+        uint32_t* src = (p & 1) ? b.A : b.B;                      // pass p reads B and writes A when p is even, the other way round when odd
         uint32_t* dst = (p & 1) ? b.B : b.A;
         if (first) LAUNCH(h, "sort_hist", k_sort_hist<false>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist);
         else LAUNCH(h, "sort_hist", k_sort_hist<true>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist);
@@ -515,11 +516,15 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
     });
     CK(h, cudaEventRecord(h->ev_join, h->side));
     const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->hist, h->block_sums};
-    LAUNCH(h, "priority", (ind ? k_priority<true> : k_priority<false>), grid_for(h, L, 1024, 8), 256, 0, s, w, sort_input(sb), av);
+    LAUNCH(h, "priority", (ind ? k_priority<true> : k_priority<false>), grid_for(h, L, PRI_CHUNK, 8), 256, 0, s, w, h->block_sums, av);
     if (h->max_sets > 0) {
-        // group the rows that missed by cache set, keeping ascending row id inside a set
+        // the rows that may be admitted (few, once the caches are warm) are gathered in row order ...
+        LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, (const uint32_t*)&w.ctr->U, (uint32_t)PRI_CHUNK, &w.ctr->n_cand);
+        LAUNCH(h, "cand_write", k_cand_write, grid_for(h, L, PRI_CHUNK, 8), 256, 0, s, w, (const uint32_t*)h->block_sums, reinterpret_cast<uint2*>(sb.B));
+        LAUNCH(h, "cand_starts", k_cand_starts, 1, 32, 0, w, h->T);
+        // ... and grouped by cache set, keeping ascending row id inside a set
         const uint32_t *ck = nullptr, *cv = nullptr;
-        seg_sort(h, sb, w.ustart, w.ctile_base, &w.ctr->chist_len, &w.ctr->abort, bits_for((uint32_t)h->max_sets), L, &ck, &cv);
+        seg_sort(h, sb, w.cstart, w.ctile_base, &w.ctr->chist_len, &w.ctr->abort, bits_for((uint32_t)h->max_sets), L, &ck, &cv, true);
         LAUNCH(h, "policy_heads", k_policy_heads, grid_for(h, L, 256, 8), 256, 0, s, w, ck);
         LAUNCH(h, "policy", (ind ? k_policy<true> : k_policy<false>), grid_for(h, std::min<int64_t>(L, h->total_sets), 256 / s.ways, 8), 256, 0, s, w, ck, cv, av);
     }

@@ -39,6 +39,7 @@ struct Counters {
     uint32_t deferred;     // newcomers that wait for the write-back of an updated row
     uint32_t n_heads;      // cache sets that have miss candidates in this step
     uint32_t upd_next;     // next block of 32 distinct rows to hand to a warp of k_update
+    uint32_t n_cand;       // candidates for admission in this step
     unsigned long long dropped;      // out-of-range indices in this batch
     unsigned long long hot_occ;      // indices that belong to hot rows
     unsigned long long err[2];       // sticky: ERR_INDEX, ERR_OFFSETS
@@ -91,6 +92,9 @@ struct Work {
     int32_t *uniq_row, *uniq_t, *seg, *loc, *final_loc, *victim, *hot_base, *uset;   // per unique row
     int32_t* task_k;       // [hot tasks]
     int32_t* hot_k;        // [hot rows]
+    uint32_t* cand_key;    // [distinct rows] the row's set if it is a candidate for admission, else the table's number of sets
+    int32_t* cand_cnt;     // [T] candidates of each table (counted by k_priority, cleared by k_cand_starts)
+    int32_t* cstart;       // [T+1] where each table's candidates begin in the compacted candidate list
     int32_t* defer_k;      // [deferred newcomers]
     int32_t* heads;        // [sets with candidates] position of the set's first candidate in the set-sorted list
     float* partial;        // [hot tasks][dim]
@@ -472,21 +476,28 @@ k_pool(State s, Work w, StepArgs av) {
 // ---------------------------------------------------------------------------------------------
 // backward 1: new priority value of every row of I_U (Section 3 "Cache Replacement Policy"), candidate keys, counters
 // ---------------------------------------------------------------------------------------------
+constexpr int PRI_Q = 4;                 // independent rows per thread: the counter updates are random accesses
+constexpr int PRI_CHUNK = PRI_Q * 256;   // rows per block and round
+
 template <bool IND>
 __global__ void __launch_bounds__(256)
-k_priority(State s, Work w, uint32_t* __restrict__ ckey, StepArgs av) {
+k_priority(State s, Work w, uint32_t* __restrict__ block_sums, StepArgs av) {
     StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
+    __shared__ uint32_t chunk_cand;
     if (w.ctr->abort) return;
     const uint32_t step = (uint32_t)a.step;
-    constexpr int Q = 4;                                     // independent rows per thread: the counter updates are random accesses
+    constexpr int Q = PRI_Q;
     const int64_t U = w.ctr->U;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    const int64_t U32 = (U + 31) & ~31LL;
-    for (int64_t k0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k0 < U32; k0 += Q * stride) {
+    uint32_t* __restrict__ ckey = w.cand_key;
+    if (threadIdx.x == 0) chunk_cand = 0;
+    __syncthreads();
+    // a block takes PRI_CHUNK consecutive rows at a time, thread i the rows i, i + 256, i + 512, i + 768 of them
+    for (int64_t c0 = (int64_t)blockIdx.x * PRI_CHUNK; c0 < U; c0 += (int64_t)gridDim.x * PRI_CHUNK) {
         int t[Q], loc[Q]; int32_t row[Q]; uint32_t mult[Q], old[Q]; int64_t rb[Q], sbase[Q]; int32_t nsets[Q];
+        uint32_t ncand = 0;
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
-            const int64_t k = k0 + q * stride;
+            const int64_t k = c0 + q * 256 + threadIdx.x;
             t[q] = -1;
             if (k < U) { t[q] = w.uniq_t[k]; row[q] = w.uniq_row[k]; loc[q] = w.loc[k]; mult[q] = (uint32_t)(w.seg[k + 1] - w.seg[k]); }
         }
@@ -501,10 +512,10 @@ k_priority(State s, Work w, uint32_t* __restrict__ ckey, StepArgs av) {
         }
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
-            const int64_t k = k0 + q * stride;
-            unsigned long long m = 0, hitm = 0, uh = 0, un = 0, byp = 0;
+            const int64_t k = c0 + q * 256 + threadIdx.x;
+            unsigned long long m = 0, hitm = 0, uh = 0, un = 0, byp = 0, cand = 0;
             if (t[q] >= 0) {
-                uint32_t key = (uint32_t)nsets[q];           // sorts behind every real set: not a candidate
+                uint32_t key = (uint32_t)nsets[q];           // not a candidate
                 if (loc[q] != LOC_INVALID) {
                     m = mult[q]; un = 1;
                     uint32_t pv = step;                      // the priority value the row has from now on
@@ -518,37 +529,91 @@ k_priority(State s, Work w, uint32_t* __restrict__ ckey, StepArgs av) {
                     else if (nsets[q] > 0) {
                         // The lowest priority value in a set never falls (counts and time stamps only grow, a replacement
                         // puts a larger value in the place of the lowest, no way is ever emptied), so a row that does not
-                        // beat a bound recorded earlier is bypassed whatever happens in this step (Algorithm 2: PV[i] <= PV[j]).
+                        // beat a bound recorded earlier is bypassed whatever happens in this step (Algorithm 2's test).
                         const int32_t set = w.uset[k];
                         const bool always = s.ways == 1 && s.policy == 0;
                         if (!always && pv <= s.floor[sbase[q] + set]) byp = 1;
-                        else key = (uint32_t)set;
+                        else { key = (uint32_t)set; cand = 1; }
                     }
                 }
                 ckey[k] = key;
             }
+            ncand += (uint32_t)cand;
             // counters: one atomic per warp when the warp sits inside one table
-            if (k0 + q * stride - (threadIdx.x & 31) >= U32) continue;       // warp-uniform: nothing left for this q
+            if (c0 + q * 256 + (threadIdx.x & ~31) >= U) continue;           // warp-uniform: nothing left for this q
             const int t0 = __shfl_sync(0xffffffffU, t[q], 0);
             const bool same = __all_sync(0xffffffffU, t[q] == t0 || t[q] < 0);
             if (same && t0 >= 0) {
                 for (int o = 16; o > 0; o >>= 1) {
                     m += __shfl_xor_sync(0xffffffffU, m, o); hitm += __shfl_xor_sync(0xffffffffU, hitm, o);
                     uh += __shfl_xor_sync(0xffffffffU, uh, o); un += __shfl_xor_sync(0xffffffffU, un, o);
-                    byp += __shfl_xor_sync(0xffffffffU, byp, o);
+                    byp += __shfl_xor_sync(0xffffffffU, byp, o); cand += __shfl_xor_sync(0xffffffffU, cand, o);
                 }
                 if ((threadIdx.x & 31) == 0) {
                     unsigned long long* st = s.stats + (int64_t)t0 * 8;
                     atomicAdd(st + 0, m); atomicAdd(st + 1, hitm); atomicAdd(st + 2, un); atomicAdd(st + 3, uh);
                     if (byp) atomicAdd(st + 6, byp);
+                    if (cand) atomicAdd(&w.cand_cnt[t0], (int32_t)cand);
                 }
             } else if (t[q] >= 0) {
                 unsigned long long* st = s.stats + (int64_t)t[q] * 8;
                 atomicAdd(st + 0, m); atomicAdd(st + 1, hitm); atomicAdd(st + 2, un); atomicAdd(st + 3, uh);
                 if (byp) atomicAdd(st + 6, byp);
+                if (cand) atomicAdd(&w.cand_cnt[t[q]], 1);
             }
         }
+        // candidates of this chunk of rows (for the compaction that follows)
+        ncand = __reduce_add_sync(0xffffffffU, ncand);
+        if ((threadIdx.x & 31) == 0 && ncand) atomicAdd(&chunk_cand, ncand);
+        __syncthreads();
+        if (threadIdx.x == 0) { block_sums[c0 / PRI_CHUNK] = chunk_cand; chunk_cand = 0; }
+        __syncthreads();
     }
+}
+
+// The candidates for admission, in the order of the distinct rows (table, then row id), as (set, distinct-row index)
+// records: block_sums holds the exclusive prefix of the per-chunk counts.
+__global__ void __launch_bounds__(256)
+k_cand_write(State s, Work w, const uint32_t* __restrict__ block_sums, uint2* __restrict__ pairs) {
+    __shared__ uint32_t tmp[256 / 32 + 1];
+    if (w.ctr->abort) return;
+    const int64_t U = w.ctr->U;
+    const uint32_t* __restrict__ ckey = w.cand_key;
+    for (int64_t c0 = (int64_t)blockIdx.x * PRI_CHUNK; c0 < U; c0 += (int64_t)gridDim.x * PRI_CHUNK) {
+        const int64_t k0 = c0 + 4 * threadIdx.x;             // four consecutive rows per thread
+        uint32_t key[4]; bool is[4]; uint32_t n = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            is[i] = false; key[i] = 0;
+            if (k0 + i < U) {
+                key[i] = ckey[k0 + i];
+                is[i] = key[i] < (uint32_t)s.tables[w.uniq_t[k0 + i]].n_sets;
+            }
+            n += is[i];
+        }
+        uint32_t total;
+        uint32_t pos = block_exclusive_scan<256>(n, &total, tmp) + block_sums[c0 / PRI_CHUNK];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (is[i]) pairs[pos++] = make_uint2(key[i], (uint32_t)(k0 + i));
+    }
+}
+
+// where each table's candidates begin (one warp; the per-table counts are cleared for the next step)
+__global__ void k_cand_starts(Work w, int T) {
+    if (blockIdx.x != 0 || threadIdx.x >= 32) return;
+    const int lane = threadIdx.x;
+    int32_t run = 0;
+    for (int t0 = 0; t0 < T; t0 += 32) {
+        const int t = t0 + lane;
+        const int32_t c = t < T ? w.cand_cnt[t] : 0;
+        int32_t inc = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int32_t v = __shfl_up_sync(0xffffffffU, inc, o); if (lane >= o) inc += v; }
+        if (t < T) { w.cstart[t] = run + inc - c; w.cand_cnt[t] = 0; }
+        run += __shfl_sync(0xffffffffU, inc, 31);
+    }
+    if (lane == 0) w.cstart[T] = w.ctr->abort ? 0 : run;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -563,15 +628,15 @@ constexpr int VICTIM_DEFER = -2;      // the displaced row was hit in this step:
 // the first candidate of every set that has any (the set-sorted list is grouped by table, then set)
 __global__ void k_policy_heads(State s, Work w, const uint32_t* __restrict__ ckey) {
     if (w.ctr->abort) return;
-    const int64_t U = w.ctr->U;
+    const int64_t U = w.cstart[s.T];                           // candidates, sorted by (table, set), row ids ascending inside a set
     const int64_t U32 = (U + 31) & ~31LL;
     const int lane = threadIdx.x & 31;
     for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < U32; j += (int64_t)gridDim.x * blockDim.x) {
         bool head = false;
         if (j < U) {
             const uint32_t key = ckey[j];
-            const int t = find_segment(w.ustart, s.T, (int32_t)j);
-            head = key < (uint32_t)s.tables[t].n_sets && (j == w.ustart[t] || ckey[j - 1] != key);
+            const int t = find_segment(w.cstart, s.T, (int32_t)j);
+            head = j == w.cstart[t] || ckey[j - 1] != key;
         }
         const uint32_t m = __ballot_sync(0xffffffffU, head);
         uint32_t base = 0;
@@ -595,7 +660,7 @@ k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __r
     for (int64_t hi = blockIdx.x * gpb + threadIdx.x / ways; hi < nheads; hi += ng) {
         const int64_t j = w.heads[hi];
         const uint32_t key = ckey[j];
-        const int t = find_segment(w.ustart, s.T, (int32_t)j);
+        const int t = find_segment(w.cstart, s.T, (int32_t)j);
         const TableDev tb = s.tables[t];
         const int64_t slot = (tb.set_base + key) * ways + way;
         int32_t tag = s.tags[slot];
@@ -603,7 +668,7 @@ k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __r
         if (tag >= 0) pri = s.policy == 1 ? s.cnt[tb.row_base + tag] : s.ts[slot];
         int32_t cand = -1, vict = VICTIM_NONE;
         uint32_t n_admit = 0, n_evict = 0, n_bypass = 0;
-        const int64_t jend = w.ustart[t + 1];
+        const int64_t jend = w.cstart[t + 1];
         for (int64_t jj0 = j;; jj0 += ways) {
             const int64_t jj = jj0 + way;
             const bool valid = jj < jend && ckey[jj] == key;
