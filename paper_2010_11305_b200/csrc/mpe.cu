@@ -416,7 +416,7 @@ int mpe_create_placed(mpe_handle** out, const mpe_table_spec* tables, int32_t nu
     if (optimizer == MPE_ROWWISE_ADAGRAD && (rc = dmalloc(h, &s.G, h->total_rows, nullptr)) != MPE_OK) return fail(rc);
     if ((rc = dmalloc(h, &s.slab, h->total_slots * dim, nullptr)) != MPE_OK) return fail(rc);
     if ((rc = dmalloc(h, &s.tags, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
-    if (policy == MPE_LRU && (rc = dmalloc(h, &s.ts, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
+    if ((rc = dmalloc(h, &s.ts, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
     if ((rc = dmalloc(h, &s.hit_epoch, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
     if ((rc = dmalloc(h, &s.hit_k, h->total_slots, nullptr)) != MPE_OK) return fail(rc);
     if ((rc = dmalloc(h, &s.floor, std::max<int64_t>(1, h->total_sets), nullptr)) != MPE_OK) return fail(rc);
@@ -1087,8 +1087,8 @@ int mpe_export_cache(mpe_handle* h, int32_t table, int32_t* h_tags, float* h_row
     if (h_tags) CK(h, cudaMemcpy(h_tags, h->st.tags + first, sizeof(int32_t) * nslot, cudaMemcpyDeviceToHost));
     if (h_rows) CK(h, cudaMemcpy(h_rows, h->st.slab + first * h->dim, sizeof(float) * nslot * h->dim, cudaMemcpyDeviceToHost));
     if (h_ts) {
-        if (h->st.ts) CK(h, cudaMemcpy(h_ts, h->st.ts + first, sizeof(uint32_t) * nslot, cudaMemcpyDeviceToHost));
-        else memset(h_ts, 0, sizeof(uint32_t) * nslot);
+        if (h->policy == MPE_LRU) CK(h, cudaMemcpy(h_ts, h->st.ts + first, sizeof(uint32_t) * nslot, cudaMemcpyDeviceToHost));
+        else memset(h_ts, 0, sizeof(uint32_t) * nslot);      // under LFU the per-slot values are copies of the rows' counts
     }
     return MPE_OK;
 }

@@ -57,7 +57,7 @@ struct State {
     float* G;              // Adagrad: [sum N]
     float* slab;           // [slots][dim]
     int32_t* tags;         // [slots], -1 empty
-    uint32_t* ts;          // LRU: [slots]
+    uint32_t* ts;          // [slots] priority value of the resident row: LRU time stamp, or a copy of its LFU count
     uint32_t* hit_epoch;   // [slots] forward call in which the slot was last hit
     int32_t* hit_k;        // [slots] unique-row index of that hit
     uint32_t* floor;       // [sets] a lower bound of the lowest priority value among the set's residents (0: none known)
@@ -522,9 +522,10 @@ k_priority(State s, Work w, uint32_t* __restrict__ block_sums, StepArgs av) {
                     if (s.policy == 1) {                     // LFU: access count of the row, saturating
                         pv = old[q] + mult[q] < old[q] ? 0xffffffffU : old[q] + mult[q];
                         s.cnt[rb[q] + row[q]] = pv;
-                    } else if (loc[q] >= 0) {
-                        s.ts[loc[q]] = step;                 // LRU: time stamp of the cached row
                     }
+                    // the cached row's priority value, kept per slot: the LRU time stamp, or a copy of the LFU count (so
+                    // that the policy kernel reads one line per set instead of one counter per resident row)
+                    if (loc[q] >= 0) s.ts[loc[q]] = pv;
                     if (loc[q] >= 0) { hitm = mult[q]; uh = 1; }
                     else if (nsets[q] > 0) {
                         // The lowest priority value in a set never falls (counts and time stamps only grow, a replacement
@@ -665,7 +666,7 @@ k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __r
         const int64_t slot = (tb.set_base + key) * ways + way;
         int32_t tag = s.tags[slot];
         uint32_t pri = 0;
-        if (tag >= 0) pri = s.policy == 1 ? s.cnt[tb.row_base + tag] : s.ts[slot];
+        if (tag >= 0) pri = s.ts[slot];
         int32_t cand = -1, vict = VICTIM_NONE;
         uint32_t n_admit = 0, n_evict = 0, n_bypass = 0;
         const int64_t jend = w.cstart[t + 1];
@@ -723,7 +724,7 @@ k_policy(State s, Work w, const uint32_t* __restrict__ ckey, const uint32_t* __r
         }
         if (cand >= 0) {
             s.tags[slot] = tag;
-            if (s.policy == 0) s.ts[slot] = step;
+            s.ts[slot] = pri;                            // the newcomer's priority value (LRU: this step)
             w.final_loc[cand] = (int32_t)slot;
             w.victim[cand] = vict;
             if (vict == VICTIM_DEFER) w.defer_k[atomicAdd(&w.ctr->deferred, 1u)] = cand;
