@@ -229,18 +229,6 @@ int alloc_set(mpe_handle* h, int64_t L, int64_t bags) {
     return MPE_OK;
 }
 
-// device-wide exclusive prefix sum of data[0 .. *n_ptr) in place
-void scan_u32(mpe_handle* h, uint32_t* data, const uint32_t* n_ptr, int64_t n_upper, uint32_t* block_sums) {
-    if (n_upper <= SCAN1_MAX) {      // small steps are bound by the number of launches
-        LAUNCH(h, "scan_single", k_scan_single, 1, SCAN1_THREADS, 0, data, n_ptr);
-        return;
-    }
-    const int g = grid_for(h, n_upper, SCAN_TILE, 8);
-    LAUNCH(h, "scan_reduce", k_scan_reduce, g, SCAN_THREADS, 0, data, n_ptr, block_sums);
-    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, block_sums, n_ptr, (uint32_t)SCAN_TILE, (uint32_t*)nullptr);
-    LAUNCH(h, "scan_apply", k_scan_apply, g, SCAN_THREADS, 0, data, n_ptr, (const uint32_t*)block_sums);
-}
-
 // The sort's memory: two buffers of 2 * n words each.  The keys to sort are expected in the first n words of B
 // (sort_input()); between passes the elements are (key, payload) records that alternate between A and B; the last
 // pass leaves the sorted keys in the first n words and the sorted payloads in the second n words of its buffer.
@@ -249,10 +237,10 @@ uint32_t* sort_input(const SortBufs& b) { return b.B; }
 
 // stable sort of every segment [seg_start[t], seg_start[t+1]) by the low `key_bits` bits of the key, the payload being
 // the element's position before the sort; *skey / *sval receive where the sorted keys / payloads are
-void seg_sort(mpe_handle* h, const SortBufs& b, const int32_t* seg_start, int32_t* tile_base, uint32_t* hist_len, const uint32_t* abort_flag,
+// tile_base: the segments' tile bookkeeping (warp_tile_bases), filled by the kernel that produced seg_start
+void seg_sort(mpe_handle* h, const SortBufs& b, const int32_t* seg_start, const int32_t* tile_base,
               int key_bits, int64_t n_upper, const uint32_t** skey, const uint32_t** sval, bool input_pairs = false) {
     const int T = h->T;
-    LAUNCH(h, "sort_tile_setup", k_tile_setup, 1, 32, 0, seg_start, T, tile_base, hist_len, abort_flag);
     const int64_t max_tiles = (n_upper + SORT_TILE - 1) / SORT_TILE + T;
     const int g = grid_for(h, max_tiles, 1, MPE_SORT_MINB);
     const int gh = grid_for(h, max_tiles, SORT_THREADS / 32, 8);
@@ -263,7 +251,7 @@ void seg_sort(mpe_handle* h, const SortBufs& b, const int32_t* seg_start, int32_
         uint32_t* dst = (p & 1) ? b.B : b.A;
         if (first) LAUNCH(h, "sort_hist", k_sort_hist<false>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist);
         else LAUNCH(h, "sort_hist", k_sort_hist<true>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist);
-        scan_u32(h, b.hist, hist_len, 256 * max_tiles, b.block_sums);
+        LAUNCH(h, "sort_offsets", k_sort_offsets, std::min(T, h->num_sms * 2), OFFS_THREADS, 0, b.hist, seg_start, (const int32_t*)tile_base, T);
         const uint32_t* kin = src; const uint2* pin = reinterpret_cast<const uint2*>(src);
         uint2* pout = reinterpret_cast<uint2*>(dst); uint32_t* ok = dst; uint32_t* ov = dst + b.n;
 #define SCATTER(F, L) LAUNCH(h, "sort_scatter", (k_sort_scatter<F, L>), g, SORT_THREADS, 0, kin, pin, pout, ok, ov, seg_start, \
@@ -471,7 +459,7 @@ void enqueue_index_chain(mpe_handle* h, int64_t L_grid, int64_t bags_grid, bool 
     const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->hist, h->block_sums};
     LAUNCH(h, "make_keys", (ind ? k_make_keys<true> : k_make_keys<false>), grid_for(h, bags_grid, 32, 8), 256, 0, s, w, sort_input(sb), av);
     // sort the row indices of the mini-batch (Section 5.1), table by table
-    seg_sort(h, sb, w.table_start, w.tile_base, &w.ctr->hist_len, &w.ctr->abort, bits_for((uint32_t)h->max_rows), L_grid, &h->skey, &h->spos);
+    seg_sort(h, sb, w.table_start, w.tile_base, bits_for((uint32_t)h->max_rows), L_grid, &h->skey, &h->spos);
     // distinct rows
     const int gs = grid_for(h, L_grid, SCAN_TILE, 8);
     LAUNCH(h, "unique_count", k_unique<false>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
@@ -524,7 +512,7 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
         LAUNCH(h, "cand_starts", k_cand_starts, 1, 32, 0, w, h->T);
         // ... and grouped by cache set, keeping ascending row id inside a set
         const uint32_t *ck = nullptr, *cv = nullptr;
-        seg_sort(h, sb, w.cstart, w.ctile_base, &w.ctr->chist_len, &w.ctr->abort, bits_for((uint32_t)h->max_sets), L, &ck, &cv, true);
+        seg_sort(h, sb, w.cstart, w.ctile_base, bits_for((uint32_t)h->max_sets), L, &ck, &cv, true);
         LAUNCH(h, "policy_heads", k_policy_heads, grid_for(h, L, 256, 8), 256, 0, s, w, ck);
         LAUNCH(h, "policy", (ind ? k_policy<true> : k_policy<false>), grid_for(h, std::min<int64_t>(L, h->total_sets), 256 / s.ways, 8), 256, 0, s, w, ck, cv, av);
     }
@@ -1243,7 +1231,7 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     LAUNCH(h, "make_keys", k_make_keys<false>, grid_for(h, bags, 32, 8), 256, 0, s, w, sort_input(sb), av);
     // segmented radix sort, as in mpe_forward, on the carved buffers
     const uint32_t *skey = nullptr, *spos = nullptr;
-    seg_sort(h, sb, w.table_start, w.tile_base, &w.ctr->hist_len, &w.ctr->abort, bits_for((uint32_t)h->max_rows), total_indices, &skey, &spos);
+    seg_sort(h, sb, w.table_start, w.tile_base, bits_for((uint32_t)h->max_rows), total_indices, &skey, &spos);
     const int gs = grid_for(h, total_indices, SCAN_TILE, 8);
     LAUNCH(h, "unique_count", k_unique<false>, gs, SCAN_THREADS, 0, w, T, skey, block_sums);
     LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);

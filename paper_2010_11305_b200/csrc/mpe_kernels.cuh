@@ -31,8 +31,7 @@ struct TableDev {
 struct Counters {
     uint32_t L;            // indices in this batch
     uint32_t U;            // distinct (table,row) pairs incl. one pseudo row per table that had bad indices
-    uint32_t hist_len;     // 256 * number of sort tiles (main sort)
-    uint32_t chist_len;    // same for the candidate sort
+    uint32_t unused0, unused1;
     uint32_t hot_rows;
     uint32_t hot_tasks;
     uint32_t abort;        // offsets were inconsistent: every later kernel of the step returns at once
@@ -144,6 +143,8 @@ __global__ void k_prelude(Work w, int T, StepArgs av) {
         for (int t = lane; t <= T; t += 32) w.table_start[t] = t == T ? (int32_t)L : 0;
         if (lane == 0) { c->abort = 1; atomicAdd(&c->err[ERR_OFFSETS], 1ULL); }
     }
+    __syncwarp();
+    warp_tile_bases(w.table_start, T, w.tile_base, bad);     // the sort's tiles, table by table
 }
 
 // keys for the sort: the row id, or N_t for an id outside [0, N_t); eight lanes per bag, four bags per warp
@@ -615,6 +616,8 @@ __global__ void k_cand_starts(Work w, int T) {
         run += __shfl_sync(0xffffffffU, inc, 31);
     }
     if (lane == 0) w.cstart[T] = w.ctr->abort ? 0 : run;
+    __syncwarp();
+    warp_tile_bases(w.cstart, T, w.ctile_base, w.ctr->abort != 0);     // the tiles of the sort by set
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -6,7 +6,7 @@
 // an 8-bit digit with per-(table, digit, tile) counters, so one pass over the
 // whole array sorts all segments at once and never moves a key out of its
 // segment.  No kernel here waits on another block: a pass is histogram ->
-// prefix sum -> scatter, three ordinary launches.  A tile is 4096 elements:
+// offsets (one block per table) -> scatter, three ordinary launches.  A tile is 4096 elements:
 // 16 per thread, ranked by warp (match on the digit, warp-private counters),
 // reordered through shared memory so that global writes are runs.
 #pragma once
@@ -59,21 +59,22 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* t
 }
 
 // ---- segment -> tile bookkeeping ----------------------------------------------
-// tile_base[t] = number of SORT_TILE-sized tiles of segments 0..t-1; tile_base[T] = total.
-// A non-zero *skip (the step was abandoned) yields zero tiles, which turns the whole sort into a no-op.
-__global__ void k_tile_setup(const int32_t* __restrict__ seg_start, int T, int32_t* __restrict__ tile_base,
-                             uint32_t* __restrict__ hist_len, const uint32_t* __restrict__ skip) {
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        const bool off = *skip != 0;
-        int32_t acc = 0;
-        for (int t = 0; t < T; ++t) {
-            tile_base[t] = acc;
-            int32_t len = off ? 0 : seg_start[t + 1] - seg_start[t];
-            acc += (len + SORT_TILE - 1) / SORT_TILE;
-        }
-        tile_base[T] = acc;
-        *hist_len = (uint32_t)acc * 256u;
+// tile_base[t] = number of SORT_TILE-sized tiles of segments 0..t-1; tile_base[T] = total.  Called by one warp whose
+// lanes all take part; `off` (the step was abandoned) yields zero tiles, which turns the whole sort into a no-op.
+__device__ __forceinline__ void warp_tile_bases(const int32_t* seg_start, int T, int32_t* tile_base, bool off) {
+    const int lane = threadIdx.x & 31;
+    int32_t run = 0;
+    for (int t0 = 0; t0 < T; t0 += 32) {
+        const int t = t0 + lane;
+        const int32_t len = (t < T && !off) ? seg_start[t + 1] - seg_start[t] : 0;
+        const int32_t c = (len + SORT_TILE - 1) / SORT_TILE;
+        int32_t inc = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int32_t v = __shfl_up_sync(0xffffffffU, inc, o); if (lane >= o) inc += v; }
+        if (t < T) tile_base[t] = run + inc - c;
+        run += __shfl_sync(0xffffffffU, inc, 31);
     }
+    if (lane == 0) tile_base[T] = run;
 }
 
 __device__ __forceinline__ int find_segment(const int32_t* __restrict__ base, int T, int32_t v) {
@@ -120,6 +121,76 @@ k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_s
 #pragma unroll
         for (int i = 0; i < 8; ++i) out[(size_t)(i * 32 + lane) * nt] = cnt[warp][i * 32 + lane];
         __syncwarp();
+    }
+}
+
+// ---- pass 2 of 3: counts -> first global position of every (table, digit, tile) ----------------
+// One block per table.  The counts of table t sit as 256 rows (one per digit value) of nt tiles; the first key of
+// (digit d, tile j) goes to  seg_start[t] + (all keys of the table with a smaller digit) + (keys with digit d in the
+// tiles before j).  A warp takes rows d = warp, warp + 32, ...: an exclusive prefix sum along the row, the row totals
+// to shared memory, then the prefix sum over the 256 totals, then the rows again to add their base.
+constexpr int OFFS_THREADS = 1024;
+constexpr int OFFS_SMALL_NT = 32;        // up to this many tiles in a table: one thread per digit value
+__global__ void __launch_bounds__(OFFS_THREADS)
+k_sort_offsets(uint32_t* __restrict__ hist, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base, int T) {
+    __shared__ uint32_t total[256];
+    __shared__ uint32_t scan_tmp[OFFS_THREADS / 32 + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int t = blockIdx.x; t < T; t += gridDim.x) {
+        const int nt = tile_base[t + 1] - tile_base[t];
+        if (nt == 0) continue;                                   // block-uniform
+        uint32_t* __restrict__ rows = hist + (size_t)256 * tile_base[t];
+        if (nt <= OFFS_SMALL_NT) {
+            // few tiles: one thread per digit value walks its row (eight loads in flight at a time)
+            uint32_t* __restrict__ row = rows + (size_t)threadIdx.x * nt;
+            uint32_t sum = 0;
+            if (threadIdx.x < 256) {
+                for (int j0 = 0; j0 < nt; j0 += 8) {
+                    uint32_t v[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) v[q] = j0 + q < nt ? row[j0 + q] : 0u;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) { if (j0 + q < nt) row[j0 + q] = sum; sum += v[q]; }
+                }
+            }
+            uint32_t all;
+            const uint32_t base = block_exclusive_scan<OFFS_THREADS>(threadIdx.x < 256 ? sum : 0u, &all, scan_tmp) + (uint32_t)seg_start[t];
+            if (threadIdx.x < 256) {
+                for (int j0 = 0; j0 < nt; j0 += 8) {
+                    uint32_t v[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) v[q] = j0 + q < nt ? row[j0 + q] : 0u;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) if (j0 + q < nt) row[j0 + q] = v[q] + base;
+                }
+            }
+            continue;
+        }
+        for (int d = warp; d < 256; d += OFFS_THREADS / 32) {
+            uint32_t* __restrict__ row = rows + (size_t)d * nt;
+            uint32_t carry = 0;
+            for (int j0 = 0; j0 < nt; j0 += 32) {
+                const uint32_t v = j0 + lane < nt ? row[j0 + lane] : 0u;
+                uint32_t inc = v;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { const uint32_t n = __shfl_up_sync(0xffffffffU, inc, o); if (lane >= o) inc += n; }
+                if (j0 + lane < nt) row[j0 + lane] = carry + inc - v;
+                carry += __shfl_sync(0xffffffffU, inc, 31);
+            }
+            if (lane == 0) total[d] = carry;
+        }
+        __syncthreads();
+        uint32_t all;
+        const uint32_t mine = threadIdx.x < 256 ? total[threadIdx.x] : 0u;
+        const uint32_t ex = block_exclusive_scan<OFFS_THREADS>(mine, &all, scan_tmp);
+        if (threadIdx.x < 256) total[threadIdx.x] = ex + (uint32_t)seg_start[t];
+        __syncthreads();
+        for (int d = warp; d < 256; d += OFFS_THREADS / 32) {
+            uint32_t* __restrict__ row = rows + (size_t)d * nt;
+            const uint32_t base = total[d];
+            for (int j = lane; j < nt; j += 32) row[j] += base;
+        }
+        __syncthreads();
     }
 }
 
@@ -225,23 +296,7 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint2* __restrict__ p
     }
 }
 
-// ---- device-wide exclusive prefix sum over uint32 (length read from device memory) ------------
-__global__ void __launch_bounds__(SCAN_THREADS)
-k_scan_reduce(const uint32_t* __restrict__ in, const uint32_t* __restrict__ n_ptr, uint32_t* __restrict__ block_sums) {
-    __shared__ uint32_t tmp[SCAN_THREADS / 32 + 1];
-    const uint32_t n = *n_ptr;
-    const uint32_t nblk = (n + SCAN_TILE - 1) / SCAN_TILE;
-    for (uint32_t b = blockIdx.x; b < nblk; b += gridDim.x) {
-        uint32_t s = 0;
-        const uint32_t base = b * SCAN_TILE + threadIdx.x * SCAN_ITEMS;
-#pragma unroll
-        for (int i = 0; i < SCAN_ITEMS; ++i) if (base + i < n) s += in[base + i];
-        uint32_t total;
-        block_exclusive_scan<SCAN_THREADS>(s, &total, tmp);
-        if (threadIdx.x == 0) block_sums[b] = total;
-    }
-}
-
+// ---- prefix sum over per-block counts (the compactions of the step: distinct rows, admission candidates) ----
 // one small block (it has to fit next to whatever else is resident): exclusive scan of block_sums[0..nblk) in place;
 // the grand total goes to *total_out
 constexpr int BSUM_THREADS = 256;
@@ -264,46 +319,6 @@ k_scan_block_sums(uint32_t* __restrict__ block_sums, const uint32_t* __restrict_
         carry += total;
     }
     if (threadIdx.x == 0 && total_out) *total_out = carry;
-}
-
-__global__ void __launch_bounds__(SCAN_THREADS)
-k_scan_apply(uint32_t* __restrict__ data, const uint32_t* __restrict__ n_ptr, const uint32_t* __restrict__ block_sums) {
-    __shared__ uint32_t tmp[SCAN_THREADS / 32 + 1];
-    const uint32_t n = *n_ptr;
-    const uint32_t nblk = (n + SCAN_TILE - 1) / SCAN_TILE;
-    for (uint32_t b = blockIdx.x; b < nblk; b += gridDim.x) {
-        uint32_t v[SCAN_ITEMS];
-        uint32_t s = 0;
-        const uint32_t base = b * SCAN_TILE + threadIdx.x * SCAN_ITEMS;
-#pragma unroll
-        for (int i = 0; i < SCAN_ITEMS; ++i) { v[i] = base + i < n ? data[base + i] : 0; s += v[i]; }
-        uint32_t total;
-        uint32_t ex = block_exclusive_scan<SCAN_THREADS>(s, &total, tmp) + block_sums[b];
-#pragma unroll
-        for (int i = 0; i < SCAN_ITEMS; ++i) { if (base + i < n) data[base + i] = ex; ex += v[i]; }
-    }
-}
-
-// short arrays: the whole exclusive scan in one block and one launch (in place)
-constexpr int SCAN1_THREADS = 512;
-constexpr int SCAN1_ITEMS = 8;
-constexpr int64_t SCAN1_MAX = 32768;
-__global__ void __launch_bounds__(SCAN1_THREADS)
-k_scan_single(uint32_t* __restrict__ data, const uint32_t* __restrict__ n_ptr) {
-    __shared__ uint32_t tmp[SCAN1_THREADS / 32 + 1];
-    const uint32_t n = *n_ptr;
-    uint32_t carry = 0;
-    for (uint32_t base = 0; base < n; base += SCAN1_THREADS * SCAN1_ITEMS) {
-        const uint32_t i = base + threadIdx.x * SCAN1_ITEMS;
-        uint32_t v[SCAN1_ITEMS], sum = 0;
-#pragma unroll
-        for (int q = 0; q < SCAN1_ITEMS; ++q) { v[q] = i + q < n ? data[i + q] : 0; sum += v[q]; }
-        uint32_t total;
-        uint32_t ex = carry + block_exclusive_scan<SCAN1_THREADS>(sum, &total, tmp);
-#pragma unroll
-        for (int q = 0; q < SCAN1_ITEMS; ++q) { if (i + q < n) data[i + q] = ex; ex += v[q]; }
-        carry += total;
-    }
 }
 
 }  // namespace mpe
