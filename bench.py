@@ -389,6 +389,77 @@ def run_ours(args, cfg, rank, world, local_rank):
     return result
 
 
+def make_routed(cfg, rank, world, device, sharded_cls=None, backend=None, stream_device=None):
+    """The table-wise partition of a model `world` times the configuration's size: every rank owns the configuration's
+    tables (its own seed, hence its own rows and index streams), sees the whole batch's bags for them, and the pooled
+    vectors / gradients change hands through the ranks' exchange buffers (mpe_forward_routed, mpe_gather_grad).
+    Returns (ShardedMpe, Stream of this rank's tables)."""
+    from paper_2010_11305_b200 import sharded
+    cls = sharded_cls or sharded.ShardedMpe
+    rows_global = list(cfg.num_rows) * world
+    kw = {} if backend is None else {"backend": backend}
+    sm = cls(rows_global, cfg.dim, cfg.bits, cfg.cache_fraction, cfg.ways, cfg.policy, cfg.optimizer, cfg.eps, cfg.init_lo,
+             cfg.init_hi, cfg.seed, cfg.batch, device, **kw)
+    assert sm.local_rows == list(cfg.num_rows), "equal tables must split evenly over the ranks"
+    return sm, wl.Stream(shard_config(cfg, rank), stream_device if stream_device is not None else torch.device("cuda", device))
+
+
+def routed_step(sm, batch, lr, step):
+    """One training step of the partitioned model: forward with the pooled vectors stored into their owners' buffers,
+    a rendezvous, the owners' gradients pulled back, backward.  (The gradient buffer keeps what was put there before
+    the timed region: the dense model that would write it is outside this library.)"""
+    idx, off, _ = batch
+    sm.forward(idx, off)
+    sm.backward(lr, step)
+
+
+def run_routed(args, cfg, rank, world, local_rank):
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    sm, stream_gen = make_routed(cfg, rank, world, local_rank)
+    total = args.warmup + args.steps
+    batches = [stream_gen.batch(s) for s in range(1, total + 1)]
+    sm.h.reserve(cfg.batch, max(b[0].numel() for b in batches))
+    sm.grad.normal_(0.0, 1e-2)
+    torch.distributed.barrier()
+    torch.cuda.synchronize(dev)
+    for i in range(args.warmup):
+        routed_step(sm, batches[i], cfg.lr, i + 1)
+    torch.distributed.barrier()
+    torch.cuda.synchronize(dev)
+    launches0 = sm.h.kernel_launches()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    cs = torch.cuda.current_stream(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.begin()
+    e0.record(cs)
+    rows = 0
+    for i in range(args.warmup, total):
+        routed_step(sm, batches[i], cfg.lr, i + 1)
+        rows += batches[i][0].numel()
+    e1.record(cs)
+    torch.distributed.barrier()
+    torch.cuda.synchronize(dev)
+    sampler.end()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    launches = sm.h.kernel_launches() - launches0
+    (ms,), (rows_all,) = aggregate([ms], [float(rows)], world, dev)
+    sm.close()
+    if rank != 0:
+        return None
+    K = args.steps
+    return {"metric": METRIC, "value": rows_all / (ms * 1e-3), "unit": "rows/s", "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": describe(cfg) + f" on each of {world} ranks ({cfg.num_tables * world} tables in all)",
+                       "l2": "inputs larger than L2; a new batch every step",
+                       "sharding": "tables partitioned over the ranks; pooled vectors stored into the sample owners' buffers by the pooling "
+                                   "kernel, gradients pulled from them (peer loads/stores, two host rendezvous per step)"},
+            "clocks": clocks, "gpu_launches": int(launches), "e2e": None, "roofline": None}
+
+
 def run_tiering(args, local_rank):
     """Effective bandwidth of forward and backward against the cache hit rate, with the low-precision table in HBM
     and in pinned host memory (the experiment of the paper's Section 5.2, on synthetic streams).  One JSON line per point."""
@@ -565,6 +636,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--routed", action="store_true", help="with --gpus N > 1: partition the tables over the ranks and time the step with the "
+                    "exchange of pooled vectors and gradients inside it (default: every rank trains its own tables, no exchange)")
     ap.add_argument("--no-prepare", action="store_true", help="do not sort the next batch ahead of time (mpe_prepare)")
     ap.add_argument("--sweep5", action="store_true", help="run every point of the policy/skew sweep (configuration 5): one JSON line per point")
     ap.add_argument("--tiering", action="store_true", help="forward/backward effective bandwidth vs hit rate, table in HBM and in host memory")
@@ -641,9 +714,9 @@ def main():
         return
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    result = run_ours(args, cfg, rank, world, local_rank)
+    result = run_routed(args, cfg, rank, world, local_rank) if (args.routed and world > 1) else run_ours(args, cfg, rank, world, local_rank)
     if rank == 0:
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and result is not None:
             sdev = torch.device("cuda", local_rank)
             r = run_oracle(make_cfg(), 3, 1, sdev, budget_rows=10_000_000)
             result["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample", "cpu", "nproc")}

@@ -93,6 +93,7 @@ struct mpe_handle {
     std::vector<ProfRec> prof_recs;
     std::vector<cudaEvent_t> event_pool;
     int last_cuda_error = 0;
+    std::map<const void*, int> resident;    // blocks per SM, per kernel
 };
 
 namespace {
@@ -133,6 +134,19 @@ int grid_for(const mpe_handle* h, int64_t work_items, int64_t items_per_block, i
     int64_t need = (work_items + items_per_block - 1) / items_per_block;
     int64_t cap = (int64_t)h->num_sms * blocks_per_sm;
     return (int)std::max<int64_t>(1, std::min(need, cap));
+}
+
+// how many blocks of a kernel fit on one SM at a time (asked once per kernel): grids of the kernels that loop over their
+// work are sized as whole waves of resident blocks, so that no kernel ends with a wave that fills a fraction of the GPU
+template <class K>
+int resident_blocks(mpe_handle* h, K kernel, int threads, size_t smem) {
+    const void* key = reinterpret_cast<const void*>(kernel);
+    auto it = h->resident.find(key);
+    if (it != h->resident.end()) return it->second;
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, smem) != cudaSuccess || n < 1) { cudaGetLastError(); n = 1; }
+    h->resident[key] = n;
+    return n;
 }
 
 int bits_for(uint32_t v) { int b = 1; while (b < 32 && (v >> b) != 0) ++b; return b; }
@@ -514,7 +528,8 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
         const uint32_t *ck = nullptr, *cv = nullptr;
         seg_sort(h, sb, w.cstart, w.ctile_base, bits_for((uint32_t)h->max_sets), L, &ck, &cv, true);
         LAUNCH(h, "policy_heads", k_policy_heads, grid_for(h, L, 256, 8), 256, 0, s, w, ck);
-        LAUNCH(h, "policy", (ind ? k_policy<true> : k_policy<false>), grid_for(h, std::min<int64_t>(L, h->total_sets), 256 / s.ways, 8), 256, 0, s, w, ck, cv, av);
+        auto pol = ind ? k_policy<true> : k_policy<false>;
+        LAUNCH(h, "policy", pol, grid_for(h, std::min<int64_t>(L, h->total_sets), 256 / s.ways, resident_blocks(h, pol, 256, 0)), 256, 0, s, w, ck, cv, av);
     }
     const int gu = grid_for(h, (L + 7) / 8, UPD_WARPS, 8);
     const int gh = grid_for(h, hot_capacity(L), 256 / s.lanes, 4);
