@@ -35,8 +35,28 @@ NOMINAL_HBM_GBS = 8000.0
 # proportion to the indices processed): dram__bytes_read.sum + dram__bytes_write.sum per index of the batch, and the
 # limiter the counters point at.  The summaries under profiles/ give the commands and the counters.
 KERNEL_EVIDENCE = {
-    "update": {"dram_bytes_per_index": 112.2, "bound": "issue", "profile": "profiles/k_update_cfg4_8tables.md"},
-    "pool": {"dram_bytes_per_index": 75.0, "bound": "latency", "profile": "profiles/k_pool_cfg4_8tables.md"},
+    "update": {"dram_bytes_per_index": 112.7, "bound": "issue",
+               "evidence": "80 % of the issue slots used, 317 warp instructions per distinct row; DRAM 29 %, L2 26 % of peak",
+               "profile": "profiles/k_update_cfg4_8tables.md"},
+    "pool": {"dram_bytes_per_index": 72.8, "bound": "latency",
+             "evidence": "7.3 long-scoreboard stall cycles per issue at 46 % of the warp slots (64 registers); L1 50 %, DRAM 22 % of peak; 61 % of the sectors hit in L1",
+             "profile": "profiles/k_pool_cfg4_8tables.md"},
+    "hot_partial": {"dram_bytes_per_index": 20.9, "bound": "l2-latency",
+                    "evidence": "gradient rows come from L2 (83 % hits, 36 % of its throughput), 11.2 long-scoreboard stall cycles per issue at 24 % of the warp slots (kept small on purpose: it runs beside other kernels)",
+                    "profile": "profiles/k_hot_partial_cfg4_8tables.md"},
+    # on the 8-table case a pass of the sort is L2 resident, so its DRAM traffic does not scale to the full size: none given
+    "sort_scatter": {"dram_bytes_per_index": None, "bound": "shared-memory latency",
+                     "evidence": "10.5 short-scoreboard stall cycles per issue (ranking through shared-memory counters), 28 % of the issue slots; 83 % of each store's sectors useful",
+                     "profile": "profiles/k_sort_scatter_cfg4_8tables.md"},
+    "broadcast": {"dram_bytes_per_index": 14.1, "bound": "l2",
+                  "evidence": "64 % of the L2 throughput (4-byte scatters and gathers inside a table's window), 80 long-scoreboard and 13.6 lg_throttle stall cycles per issue",
+                  "profile": "profiles/k_broadcast_cfg4_8tables.md"},
+    "priority": {"dram_bytes_per_index": 16.2, "bound": "dram-latency",
+                 "evidence": "one random read-modify-write of a counter per distinct row: 30 long-scoreboard stall cycles per issue, 13 % of the issue slots",
+                 "profile": "profiles/small_kernels_cfg4_8tables.md"},
+    "policy": {"dram_bytes_per_index": 6.3, "bound": "latency",
+               "evidence": "8.8 long-scoreboard stall cycles per issue, 47 % of the issue slots",
+               "profile": "profiles/small_kernels_cfg4_8tables.md"},
 }
 
 
@@ -212,7 +232,7 @@ def kernel_roofline(name, tms, n, K, L, model, peak, peak_kind, evidence_ok, ste
     pa, comp, basis = model.get(name, (0.0, 0.0, "not modelled"))
     pa, comp = pa / lps, comp / lps
     ev = KERNEL_EVIDENCE.get(name) if evidence_ok else None
-    traffic = ev["dram_bytes_per_index"] * L / lps if ev else None
+    traffic = ev["dram_bytes_per_index"] * L / lps if ev and ev["dram_bytes_per_index"] is not None else None
     sec = per_launch_ms * 1e-3
     achieved = pa / sec / 1e9 if sec > 0 else 0.0
     return {"kernel": name, "bound": ev["bound"] if ev else "unprofiled", "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
@@ -221,7 +241,7 @@ def kernel_roofline(name, tms, n, K, L, model, peak, peak_kind, evidence_ok, ste
             "dram_frac": traffic / sec / 1e9 / peak if traffic else None,
             "bytes_per_launch": pa, "compulsory_bytes_per_launch": comp, "compulsory_frac": comp / sec / 1e9 / peak if sec > 0 else None,
             "ms_per_launch": per_launch_ms, "launches_per_step": n / K, "share_of_step": tms / K / step_ms,
-            "profile": ev["profile"] if ev else None}
+            "evidence": ev["evidence"] if ev else None, "profile": ev["profile"] if ev else None}
 
 
 def run_ours(args, cfg, rank, world, local_rank):
@@ -248,17 +268,20 @@ def run_ours(args, cfg, rank, world, local_rank):
     # inside the region that times K steps.
     side = torch.cuda.Stream(dev)
     ahead = not args.no_prepare
+    use_prepare = [ahead]
 
     def step(i):
         idx, off, grad = batches[i]
         counter[0] += 1
         h.forward(idx, off, cfg.batch, out, sp)
-        if ahead and i + 1 < len(batches):
+        if use_prepare[0] and i + 1 < len(batches):
             h.prepare(batches[i + 1][0], batches[i + 1][1], cfg.batch, side.cuda_stream)
         h.backward(grad, cfg.lr, counter[0])
 
-    # Small steps are replayed from CUDA graphs, which per-kernel event records would break up: for them the timed
-    # region runs without the records and the per-kernel times come from a second pass over the same batches.
+    # Small steps are replayed from CUDA graphs (which per-kernel event records would break up) and large steps run
+    # beside the next batch's preparation (which makes a kernel's bracketing events include its neighbours): the timed
+    # region runs without the records, and the per-kernel times come from a second pass over the same batches, launched
+    # plainly and without the preparation.
     graph_sized = maxL <= (4 << 20)
 
     def barrier():
@@ -271,7 +294,6 @@ def run_ours(args, cfg, rank, world, local_rank):
     barrier()
     stats0 = np.sum([h.stats(t) for t in range(cfg.num_tables)], axis=0).astype(np.int64)
     launches0 = h.kernel_launches()
-    h.profile(not graph_sized)
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
@@ -288,8 +310,6 @@ def run_ours(args, cfg, rank, world, local_rank):
     ms = marks[0].elapsed_time(marks[K])
     per_step_ms = [marks[j].elapsed_time(marks[j + 1]) for j in range(K)]
     clocks = sampler.stop()
-    prof = h.profile_read()
-    h.profile(False)
     launches = h.kernel_launches() - launches0
     stats1 = np.sum([h.stats(t) for t in range(cfg.num_tables)], axis=0).astype(np.int64)
     code, detail = h.last_error()
@@ -330,12 +350,13 @@ def run_ours(args, cfg, rank, world, local_rank):
             h.step_host(idx, off, cfg.batch, grad, h_outs[0], cfg.lr, counter[0])
         torch.cuda.synchronize(dev)
         e2e_serial_s = time.perf_counter() - t0
-    if graph_sized:
-        h.profile(True)
-        for i in range(args.warmup, args.warmup + args.steps):
-            step(i)
-        prof = h.profile_read()
-        h.profile(False)
+    h.profile(True)
+    use_prepare[0] = False
+    for i in range(args.warmup, args.warmup + args.steps):
+        step(i)
+    prof = h.profile_read()
+    h.profile(False)
+    use_prepare[0] = ahead
 
     # aggregate over ranks: total rows / max time
     (ms, e2e_s, e2e_serial_s), (rows_timed, e2e_rows) = aggregate([ms, e2e_s, e2e_serial_s], [float(ds[0]), float(e2e_rows)], world, dev)
@@ -360,7 +381,7 @@ def run_ours(args, cfg, rank, world, local_rank):
         "warmup": args.warmup, "ms_per_step": ms_step, "ms_per_step_median": ms_median, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": describe(cfg), "l2": "inputs larger than L2; a new batch every step",
-                   "launch": "CUDA graph replay (per-kernel times from a second, plainly launched pass)" if graph_sized else "plain launches",
+                   "launch": ("CUDA graph replay" if graph_sized else "plain launches") + "; per-kernel times from a second, plainly launched pass without the preparation",
                    "next_batch": "sorted ahead on a second stream (mpe_prepare) while the current step runs" if ahead and not graph_sized else "not prepared ahead",
                    "sharding": "each rank trains its own tables (no data-path collective)" if world > 1 else "one GPU"},
         "clocks": clocks,

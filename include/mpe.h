@@ -108,7 +108,9 @@ int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offset
  * results are bit-identical with and without the call.  Layouts as in mpe_forward; the two buffers must stay
  * unchanged until that forward.  One batch can be prepared at a time; a forward with other arguments discards it.
  * The call does nothing (and returns MPE_OK) when the batch does not fit the workspace reserved with mpe_reserve, or
- * when steps of this size are replayed from a CUDA graph.  The first call allocates the second workspace
+ * when steps of this size are replayed from a CUDA graph.  Do not prepare a batch whose forward will be issued while
+ * the caller captures its stream into a graph (the hand-over is an event recorded outside that capture).
+ * The first call allocates the second workspace
  * (cudaMalloc; as large as the first, see mpe_workspace_bytes).
  * Typical loop:  forward(k); prepare(k+1, other_stream); backward(k); forward(k+1); ...
  */

@@ -195,6 +195,9 @@ void free_workspace(mpe_handle* h) {
     h->cap_L = 0; h->cap_bags = 0;
 }
 
+// Steps this small are bound by launch latency (they are replayed from CUDA graphs); above it the launches hide behind the kernels.
+constexpr int64_t GRAPH_MAX_INDICES = 4 << 20;
+
 int alloc_set(mpe_handle* h, int64_t L, int64_t bags);
 
 int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
@@ -224,7 +227,9 @@ int alloc_set(mpe_handle* h, int64_t L, int64_t bags) {
     // results have been consumed, and uses the same two
     h->sort_n = (n + 3) & ~int64_t(3);
     A(h->sortA, 2 * h->sort_n); A(h->sortB, 2 * h->sort_n);
-    const int64_t max_tiles = (L + SORT_TILE - 1) / SORT_TILE + T + 1;
+    // small batches (the ones that are replayed from a graph) get small tiles, so that every SM has one
+    w.sort_tile = sort_tile(L <= GRAPH_MAX_INDICES);
+    const int64_t max_tiles = (L + w.sort_tile - 1) / w.sort_tile + T + 1;
     A(h->hist, 256 * max_tiles);
     A(h->block_sums, std::max<int64_t>(256 * max_tiles, n) / std::min<int64_t>(SCAN_TILE, PRI_CHUNK) + 2);
     A(w.ctr, 1); A(w.args, 1);
@@ -246,7 +251,7 @@ int alloc_set(mpe_handle* h, int64_t L, int64_t bags) {
 // The sort's memory: two buffers of 2 * n words each.  The keys to sort are expected in the first n words of B
 // (sort_input()); between passes the elements are (key, payload) records that alternate between A and B; the last
 // pass leaves the sorted keys in the first n words and the sorted payloads in the second n words of its buffer.
-struct SortBufs { uint32_t *A, *B; int64_t n; uint32_t *hist, *block_sums; };
+struct SortBufs { uint32_t *A, *B; int64_t n; uint32_t *hist, *block_sums; int tile; };
 uint32_t* sort_input(const SortBufs& b) { return b.B; }
 
 // stable sort of every segment [seg_start[t], seg_start[t+1]) by the low `key_bits` bits of the key, the payload being
@@ -255,7 +260,7 @@ uint32_t* sort_input(const SortBufs& b) { return b.B; }
 void seg_sort(mpe_handle* h, const SortBufs& b, const int32_t* seg_start, const int32_t* tile_base,
               int key_bits, int64_t n_upper, const uint32_t** skey, const uint32_t** sval, bool input_pairs = false) {
     const int T = h->T;
-    const int64_t max_tiles = (n_upper + SORT_TILE - 1) / SORT_TILE + T;
+    const int64_t max_tiles = (n_upper + b.tile - 1) / b.tile + T;
     const int g = grid_for(h, max_tiles, 1, MPE_SORT_MINB);
     const int gh = grid_for(h, max_tiles, SORT_THREADS / 32, 8);
     const int passes = (key_bits + 7) / 8;
@@ -263,13 +268,15 @@ void seg_sort(mpe_handle* h, const SortBufs& b, const int32_t* seg_start, const 
         const bool first = p == 0 && !input_pairs, last = p == passes - 1;    // input_pairs: B holds (key, payload) records already
         uint32_t* src = (p & 1) ? b.A : b.B;                      // pass p reads B and writes A when p is even, the other way round when odd
         uint32_t* dst = (p & 1) ? b.B : b.A;
-        if (first) LAUNCH(h, "sort_hist", k_sort_hist<false>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist);
-        else LAUNCH(h, "sort_hist", k_sort_hist<true>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist);
+        if (first) LAUNCH(h, "sort_hist", k_sort_hist<false>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist, b.tile);
+        else LAUNCH(h, "sort_hist", k_sort_hist<true>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist, b.tile);
         LAUNCH(h, "sort_offsets", k_sort_offsets, std::min(T, h->num_sms * 2), OFFS_THREADS, 0, b.hist, seg_start, (const int32_t*)tile_base, T);
         const uint32_t* kin = src; const uint2* pin = reinterpret_cast<const uint2*>(src);
         uint2* pout = reinterpret_cast<uint2*>(dst); uint32_t* ok = dst; uint32_t* ov = dst + b.n;
-#define SCATTER(F, L) LAUNCH(h, "sort_scatter", (k_sort_scatter<F, L>), g, SORT_THREADS, 0, kin, pin, pout, ok, ov, seg_start, \
-                             (const int32_t*)tile_base, T, 8 * p, (const uint32_t*)b.hist)
+#define SCATTER(F, L) do { if (b.tile == sort_tile(true)) LAUNCH(h, "sort_scatter", (k_sort_scatter<F, L, SORT_ITEMS_SMALL>), g, SORT_THREADS, 0, kin, pin, pout, ok, ov, seg_start, \
+                                                               (const int32_t*)tile_base, T, 8 * p, (const uint32_t*)b.hist); \
+                           else LAUNCH(h, "sort_scatter", (k_sort_scatter<F, L, SORT_ITEMS_LARGE>), g, SORT_THREADS, 0, kin, pin, pout, ok, ov, seg_start, \
+                                       (const int32_t*)tile_base, T, 8 * p, (const uint32_t*)b.hist); } while (0)
         if (first && last) SCATTER(true, true);
         else if (first) SCATTER(true, false);
         else if (last) SCATTER(false, true);
@@ -470,7 +477,7 @@ void enqueue_index_chain(mpe_handle* h, int64_t L_grid, int64_t bags_grid, bool 
     Work& w = h->wk;
     const int T = h->T;
     LAUNCH(h, "prelude", (ind ? k_prelude<true> : k_prelude<false>), 1, 32, 0, w, T, av);
-    const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->hist, h->block_sums};
+    const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->hist, h->block_sums, h->wk.sort_tile};
     LAUNCH(h, "make_keys", (ind ? k_make_keys<true> : k_make_keys<false>), grid_for(h, bags_grid, 32, 8), 256, 0, s, w, sort_input(sb), av);
     // sort the row indices of the mini-batch (Section 5.1), table by table
     seg_sort(h, sb, w.table_start, w.tile_base, bits_for((uint32_t)h->max_rows), L_grid, &h->skey, &h->spos);
@@ -517,7 +524,7 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
         LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, hot_capacity(L), 1, 2), 8 * LANES, 32 * s.dim * sizeof(float), s, w, av);
     });
     CK(h, cudaEventRecord(h->ev_join, h->side));
-    const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->hist, h->block_sums};
+    const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->hist, h->block_sums, h->wk.sort_tile};
     LAUNCH(h, "priority", (ind ? k_priority<true> : k_priority<false>), grid_for(h, L, PRI_CHUNK, 8), 256, 0, s, w, h->block_sums, av);
     if (h->max_sets > 0) {
         // the rows that may be admitted (few, once the caches are warm) are gathered in row order ...
@@ -546,8 +553,6 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
     return check_launch(h);
 }
 
-// Steps this small are bound by launch latency; above it the launches hide behind the kernels.
-constexpr int64_t GRAPH_MAX_INDICES = 4 << 20;
 
 bool may_use_graph(mpe_handle* h) {
     if (!h->graphs_enabled || h->profiling || h->cap_L > GRAPH_MAX_INDICES) return false;
@@ -1171,8 +1176,8 @@ constexpr int STATIC_MAX_TABLES = MPE_STATIC_MAX_TABLES;
 constexpr size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 constexpr size_t STATIC_SCRATCH_BYTES =
     2 * align256(2 * (STATIC_MAX_INDICES + 4) * 4) + 12 * align256((STATIC_MAX_INDICES + 4) * 4) +                                 // keys, payloads, per-index and per-row maps
-    align256(256 * ((STATIC_MAX_INDICES + SORT_TILE - 1) / SORT_TILE + STATIC_MAX_TABLES + 1) * 4) +   // sort histograms
-    align256((256 * ((STATIC_MAX_INDICES + SORT_TILE - 1) / SORT_TILE + STATIC_MAX_TABLES + 1) / SCAN_TILE + 2 +
+    align256(256 * ((STATIC_MAX_INDICES + sort_tile(true) - 1) / sort_tile(true) + STATIC_MAX_TABLES + 1) * 4) +   // sort histograms
+    align256((256 * ((STATIC_MAX_INDICES + sort_tile(true) - 1) / sort_tile(true) + STATIC_MAX_TABLES + 1) / SCAN_TILE + 2 +
               STATIC_MAX_INDICES / SCAN_TILE + 2) * 4) +                                               // block sums
     4 * align256((STATIC_MAX_TABLES + 1) * 4) +                                                        // per-table starts
     2 * align256(hot_capacity(STATIC_MAX_INDICES) * 4) +                                             // hot-row lists
@@ -1223,7 +1228,7 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     w.bag_of = c.take<int32_t>(n); w.kidx = c.take<uint32_t>(n); w.occ_loc = c.take<int32_t>(n); w.occ_b = c.take<int32_t>(n);
     w.uniq_row = c.take<int32_t>(n); w.uniq_t = c.take<int32_t>(n); w.seg = c.take<int32_t>(n); w.loc = c.take<int32_t>(n);
     w.final_loc = c.take<int32_t>(n); w.uset = c.take<int32_t>(n); w.hot_base = c.take<int32_t>(n); w.victim = c.take<int32_t>(n);
-    const size_t max_tiles = (STATIC_MAX_INDICES + SORT_TILE - 1) / SORT_TILE + STATIC_MAX_TABLES + 1;
+    const size_t max_tiles = (STATIC_MAX_INDICES + sort_tile(true) - 1) / sort_tile(true) + STATIC_MAX_TABLES + 1;
     uint32_t* hist = c.take<uint32_t>(256 * max_tiles);
     uint32_t* block_sums = c.take<uint32_t>(256 * max_tiles / SCAN_TILE + 2 + STATIC_MAX_INDICES / SCAN_TILE + 2);
     w.table_start = c.take<int32_t>(STATIC_MAX_TABLES + 1); w.tile_base = c.take<int32_t>(STATIC_MAX_TABLES + 1);
@@ -1241,7 +1246,8 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), stream));
     StepArgs av{};
     av.indices = d_indices; av.offsets = d_offsets; av.out = d_out; av.B = batch; av.L = L; av.epoch = h->epoch;
-    const SortBufs sb{sortA, sortB, (int64_t)n, hist, block_sums};
+    w.sort_tile = sort_tile(true);
+    const SortBufs sb{sortA, sortB, (int64_t)n, hist, block_sums, w.sort_tile};
     LAUNCH(h, "prelude", k_prelude<false>, 1, 32, 0, w, T, av);
     LAUNCH(h, "make_keys", k_make_keys<false>, grid_for(h, bags, 32, 8), 256, 0, s, w, sort_input(sb), av);
     // segmented radix sort, as in mpe_forward, on the carved buffers

@@ -97,6 +97,7 @@ struct Work {
     int32_t* defer_k;      // [deferred newcomers]
     int32_t* heads;        // [sets with candidates] position of the set's first candidate in the set-sorted list
     float* partial;        // [hot tasks][dim]
+    int32_t sort_tile;     // keys per tile of the sorts of this workspace
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -144,7 +145,7 @@ __global__ void k_prelude(Work w, int T, StepArgs av) {
         if (lane == 0) { c->abort = 1; atomicAdd(&c->err[ERR_OFFSETS], 1ULL); }
     }
     __syncwarp();
-    warp_tile_bases(w.table_start, T, w.tile_base, bad);     // the sort's tiles, table by table
+    warp_tile_bases(w.table_start, T, w.tile_base, bad, w.sort_tile);     // the sort's tiles, table by table
 }
 
 // keys for the sort: the row id, or N_t for an id outside [0, N_t); eight lanes per bag, four bags per warp
@@ -617,7 +618,7 @@ __global__ void k_cand_starts(Work w, int T) {
     }
     if (lane == 0) w.cstart[T] = w.ctr->abort ? 0 : run;
     __syncwarp();
-    warp_tile_bases(w.cstart, T, w.ctile_base, w.ctr->abort != 0);     // the tiles of the sort by set
+    warp_tile_bases(w.cstart, T, w.ctile_base, w.ctr->abort != 0, w.sort_tile);     // the tiles of the sort by set
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -15,15 +15,16 @@
 
 namespace mpe {
 
-#ifndef MPE_SORT_ITEMS
-#define MPE_SORT_ITEMS 16      // keys per thread of the scatter kernel (even)
-#endif
 #ifndef MPE_SORT_MINB
 #define MPE_SORT_MINB 4        // resident blocks per SM the scatter kernel is compiled for
 #endif
 constexpr int SORT_THREADS = 256;
-constexpr int SORT_ITEMS = MPE_SORT_ITEMS;
-constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;   // keys per block
+// Keys per thread of the scatter kernel, hence keys per tile: 16 (4096-key tiles) for large batches, where the fixed cost
+// of a tile is spread over more keys and a digit's run is longer; 8 (2048-key tiles) for batches so small that larger
+// tiles would leave SMs without a tile.  The tile size of a sort travels as an argument.
+constexpr int SORT_ITEMS_LARGE = 16, SORT_ITEMS_SMALL = 8;
+constexpr int SORT_TILE_MAX = SORT_THREADS * SORT_ITEMS_LARGE;
+__host__ __device__ constexpr int sort_tile(bool small) { return SORT_THREADS * (small ? SORT_ITEMS_SMALL : SORT_ITEMS_LARGE); }
 constexpr int SCAN_THREADS = 256;
 constexpr int SCAN_ITEMS = 16;
 constexpr int SCAN_TILE = SCAN_THREADS * SCAN_ITEMS;
@@ -59,15 +60,15 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* t
 }
 
 // ---- segment -> tile bookkeeping ----------------------------------------------
-// tile_base[t] = number of SORT_TILE-sized tiles of segments 0..t-1; tile_base[T] = total.  Called by one warp whose
+// tile_base[t] = number of tiles (of `tile` keys) of segments 0..t-1; tile_base[T] = total.  Called by one warp whose
 // lanes all take part; `off` (the step was abandoned) yields zero tiles, which turns the whole sort into a no-op.
-__device__ __forceinline__ void warp_tile_bases(const int32_t* seg_start, int T, int32_t* tile_base, bool off) {
+__device__ __forceinline__ void warp_tile_bases(const int32_t* seg_start, int T, int32_t* tile_base, bool off, int tile) {
     const int lane = threadIdx.x & 31;
     int32_t run = 0;
     for (int t0 = 0; t0 < T; t0 += 32) {
         const int t = t0 + lane;
         const int32_t len = (t < T && !off) ? seg_start[t + 1] - seg_start[t] : 0;
-        const int32_t c = (len + SORT_TILE - 1) / SORT_TILE;
+        const int32_t c = (len + tile - 1) / tile;
         int32_t inc = c;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) { const int32_t v = __shfl_up_sync(0xffffffffU, inc, o); if (lane >= o) inc += v; }
@@ -92,7 +93,7 @@ __device__ __forceinline__ int find_segment(const int32_t* __restrict__ base, in
 template <bool PAIRS>
 __global__ void __launch_bounds__(SORT_THREADS)
 k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base,
-            int T, int shift, uint32_t* __restrict__ hist) {
+            int T, int shift, uint32_t* __restrict__ hist, int tile_keys) {
     // one warp per tile: its own 256 counters, eight key loads in flight per lane, no block-wide barrier
     constexpr int WARPS = SORT_THREADS / 32;
     constexpr int STRIDE = PAIRS ? 2 : 1;
@@ -103,8 +104,8 @@ k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_s
         const int t = find_segment(tile_base, T, tile);
         const int local = tile - tile_base[t];
         const int nt = tile_base[t + 1] - tile_base[t];
-        const int32_t start = seg_start[t] + local * SORT_TILE;
-        const int32_t end = min(start + SORT_TILE, seg_start[t + 1]);
+        const int32_t start = seg_start[t] + local * tile_keys;
+        const int32_t end = min(start + tile_keys, seg_start[t + 1]);
 #pragma unroll
         for (int i = 0; i < 8; ++i) cnt[warp][i * 32 + lane] = 0;
         __syncwarp();
@@ -200,13 +201,14 @@ k_sort_offsets(uint32_t* __restrict__ hist, const int32_t* __restrict__ seg_star
 // FIRST: the input is the bare key array and the payload is the element's position.
 // LAST: the output is split into the sorted keys and the sorted payloads (out_keys / out_vals), which is what the
 // kernels after the sort read.
-template <bool FIRST, bool LAST>
+template <bool FIRST, bool LAST, int SORT_ITEMS>
 __global__ void __launch_bounds__(SORT_THREADS, MPE_SORT_MINB)
 k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint2* __restrict__ pairs_in, uint2* __restrict__ pairs_out,
                uint32_t* __restrict__ out_keys, uint32_t* __restrict__ out_vals,
                const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base, int T, int shift,
                const uint32_t* __restrict__ hist_scanned) {
     constexpr int WARPS = SORT_THREADS / 32;
+    constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;
     __shared__ uint32_t wcnt[WARPS][256];      // per-warp digit counters, then tile-local position of the warp's first key of each digit
     __shared__ uint32_t goff[256];             // first global position of each digit of this tile minus its tile-local start
     __shared__ uint2 skv[SORT_TILE];
