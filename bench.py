@@ -168,8 +168,9 @@ def byte_model(cfg, L, U, U_hit, occ_hit, admissions, evictions, hot_occ, passes
     m["policy"] = (U_miss * (4 if cfg.policy == wl.LFU else 0) + admissions * 8 * cfg.ways,) * 2 + ("method (priority values of candidates and sets)",)
     sort_rw = passes_main * 16 * L + passes_cand * 16 * U
     m["sort_scatter"] = (sort_rw, sort_rw, "radix-sort pass: key + payload read and written")
-    m["sort_hist"] = (passes_main * 4 * L + passes_cand * 4 * U,) * 2 + ("radix-sort pass: keys read",)
+    m["sort_digits"] = (4 * L + 8 * U,) * 2 + ("radix sort: the keys read once, ahead of the passes",)
     m["make_keys"] = (4 * L + 4 * T * B, 4 * L + 4 * T * B, "indices and offsets read")
+    m["unique"] = (4 * L + 4 * U, 4 * L + 4 * U, "sorted keys read, distinct rows written")
     m["unique_count"] = (4 * L, 4 * L, "sorted keys read")
     m["unique_write"] = (4 * L + 4 * U, 4 * L + 4 * U, "sorted keys read, distinct rows written")
     m["broadcast"] = (8 * L, 8 * L, "bookkeeping: per-index slot and sample id written")

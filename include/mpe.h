@@ -41,7 +41,8 @@ enum {
     MPE_ERR_INDEX = -5,        /* device saw row ids outside [0, num_rows) (detail = how many); they were dropped */
     MPE_ERR_OFFSETS = -6,      /* device saw offsets that are not 0 = o[0] <= o[1] <= ... <= o[T*B] = total */
     MPE_ERR_NOMEM = -7,        /* allocation failed */
-    MPE_ERR_TOO_LARGE = -8     /* mpe_forward_static: the batch does not fit the fixed scratch */
+    MPE_ERR_TOO_LARGE = -8,    /* mpe_forward_static: the batch does not fit the fixed scratch */
+    MPE_ERR_TIMEOUT = -9       /* a bounded wait between thread blocks of one kernel ran out (detail = how many); the step was abandoned */
 };
 
 /*
@@ -237,7 +238,10 @@ int mpe_destroy(mpe_handle* h);
 
 /* ---- observation (all of these wait for the handle's stream) --------------------------------- */
 /* Sticky device-detected condition since the last call of this function: *code is MPE_OK,
- * MPE_ERR_INDEX or MPE_ERR_OFFSETS; *detail counts the offending items.  Clears the condition. */
+ * MPE_ERR_INDEX, MPE_ERR_OFFSETS or MPE_ERR_TIMEOUT; *detail counts the offending items.  Clears the
+ * condition.  (MPE_ERR_TIMEOUT: the sort's tiles learn their output positions from the tiles before them;
+ * every such wait gives up after about a second, the step that met it changes nothing from there on and
+ * the handle stays usable.  It is not expected to occur.) */
 int mpe_last_error(mpe_handle* h, int32_t* code, int64_t* detail);
 /* Counters of table `table` accumulated by mpe_backward: out8 = {lookups, hits (per index),
  * unique rows, unique hits, admissions, evictions, bypasses, steps}. */

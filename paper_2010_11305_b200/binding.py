@@ -18,7 +18,7 @@ LRU, LFU = 0, 1
 SGD, ROWWISE_ADAGRAD = 0, 1
 ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
 TABLE_DEVICE, TABLE_HOST = 0, 1
-OK, ERR_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_SEQUENCE, ERR_INDEX, ERR_OFFSETS, ERR_NOMEM, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6, -7, -8
+OK, ERR_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_SEQUENCE, ERR_INDEX, ERR_OFFSETS, ERR_NOMEM, ERR_TOO_LARGE, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7, -8, -9
 STATIC_MAX_INDICES, STATIC_MAX_BAGS, STATIC_MAX_TABLES = 32768, 32768, 64
 
 EXPORTS = [

@@ -39,14 +39,18 @@ struct mpe_handle {
     uint64_t ws_bytes = 0;                  // bytes of the per-step workspace
     uint32_t *sortA = nullptr, *sortB = nullptr;   // two buffers of 2 * sort_n words: (key, payload) records, or keys | payloads
     int64_t sort_n = 0;
-    uint32_t *hist = nullptr, *block_sums = nullptr;
+    uint32_t *ghist = nullptr, *block_sums = nullptr;      // the sort's per-table digit counts; candidates per chunk of distinct rows (large steps)
+    unsigned long long* sort_status = nullptr;             // the sort's per-tile words
+    SortCtl* sort_ctl = nullptr;
+    uint64_t sort_passes_bound = 0;                        // no more than this many sort passes have run on either workspace
     std::vector<void*> ws_allocs;
     cudaEvent_t ev_free = nullptr;          // recorded behind the last kernel that uses this workspace
     // A second workspace, allocated on the first mpe_prepare: the next batch is sorted and de-duplicated there while the
     // kernels of the current step still run.  `alt` holds exactly the members above that belong to a workspace.
     struct WsSet {
         Work wk{};
-        uint32_t *sortA = nullptr, *sortB = nullptr, *hist = nullptr, *block_sums = nullptr;
+        uint32_t *sortA = nullptr, *sortB = nullptr, *ghist = nullptr, *block_sums = nullptr;
+        unsigned long long* sort_status = nullptr; SortCtl* sort_ctl = nullptr;
         int64_t sort_n = 0;
         const uint32_t *skey = nullptr, *spos = nullptr;
         std::vector<void*> allocs;
@@ -172,7 +176,8 @@ void drop_graphs(mpe_handle* h) {
 void swap_sets(mpe_handle* h) {
     std::swap(h->wk, h->alt.wk);
     std::swap(h->sortA, h->alt.sortA); std::swap(h->sortB, h->alt.sortB);
-    std::swap(h->hist, h->alt.hist); std::swap(h->block_sums, h->alt.block_sums);
+    std::swap(h->ghist, h->alt.ghist); std::swap(h->block_sums, h->alt.block_sums);
+    std::swap(h->sort_status, h->alt.sort_status); std::swap(h->sort_ctl, h->alt.sort_ctl);
     std::swap(h->sort_n, h->alt.sort_n);
     std::swap(h->skey, h->alt.skey); std::swap(h->spos, h->alt.spos);
     std::swap(h->ws_allocs, h->alt.allocs);
@@ -199,6 +204,26 @@ void free_workspace(mpe_handle* h) {
 constexpr int64_t GRAPH_MAX_INDICES = 4 << 20;
 
 int alloc_set(mpe_handle* h, int64_t L, int64_t bags);
+
+int64_t sort_max_tiles(const mpe_handle* h, int64_t L) {
+    const int tile = sort_tile(L <= GRAPH_MAX_INDICES);
+    return (L + tile - 1) / tile + h->T + 1;
+}
+
+// The sort's per-tile words carry a 30-bit pass number.  Long before it can come round to a value that old words still
+// hold (hundreds of millions of steps), everything is brought to rest once and the words and the counter start over.
+int renew_sort_tags(mpe_handle* h) {
+    CK(h, cudaDeviceSynchronize());
+    for (int set = 0; set < 2; ++set) {
+        if (h->sort_status) {
+            CK(h, cudaMemset(h->sort_status, 0, sizeof(unsigned long long) * 256 * sort_max_tiles(h, h->cap_L)));
+            CK(h, cudaMemset(h->sort_ctl, 0, sizeof(SortCtl)));
+        }
+        swap_sets(h);
+    }
+    h->sort_passes_bound = 0;
+    return MPE_OK;
+}
 
 int alloc_workspace(mpe_handle* h, int64_t L, int64_t bags) {
     free_workspace(h);
@@ -229,9 +254,13 @@ int alloc_set(mpe_handle* h, int64_t L, int64_t bags) {
     A(h->sortA, 2 * h->sort_n); A(h->sortB, 2 * h->sort_n);
     // small batches (the ones that are replayed from a graph) get small tiles, so that every SM has one
     w.sort_tile = sort_tile(L <= GRAPH_MAX_INDICES);
-    const int64_t max_tiles = (L + w.sort_tile - 1) / w.sort_tile + T + 1;
-    A(h->hist, 256 * max_tiles);
-    A(h->block_sums, std::max<int64_t>(256 * max_tiles, n) / std::min<int64_t>(SCAN_TILE, PRI_CHUNK) + 2);
+    const int64_t max_tiles = sort_max_tiles(h, L);
+    A(h->sort_status, 256 * max_tiles); A(h->ghist, (int64_t)T * SORT_MAX_PASSES * 256); A(h->sort_ctl, 1);
+    // the sort keeps these consistent by itself from one pass to the next; they start from zero
+    CK(h, cudaMemset(h->sort_status, 0, sizeof(unsigned long long) * 256 * max_tiles));
+    CK(h, cudaMemset(h->ghist, 0, sizeof(uint32_t) * T * SORT_MAX_PASSES * 256));
+    CK(h, cudaMemset(h->sort_ctl, 0, sizeof(SortCtl)));
+    A(h->block_sums, n / std::min<int64_t>(SCAN_TILE, PRI_CHUNK) + 2);
     A(w.ctr, 1); A(w.args, 1);
     A(w.table_start, T + 1); A(w.tile_base, T + 1); A(w.ustart, T + 1); A(w.ctile_base, T + 1);
     A(w.bag_of, n); A(w.kidx, n); A(w.occ_loc, n); A(w.occ_b, n);
@@ -251,7 +280,7 @@ int alloc_set(mpe_handle* h, int64_t L, int64_t bags) {
 // The sort's memory: two buffers of 2 * n words each.  The keys to sort are expected in the first n words of B
 // (sort_input()); between passes the elements are (key, payload) records that alternate between A and B; the last
 // pass leaves the sorted keys in the first n words and the sorted payloads in the second n words of its buffer.
-struct SortBufs { uint32_t *A, *B; int64_t n; uint32_t *hist, *block_sums; int tile; };
+struct SortBufs { uint32_t *A, *B; int64_t n; uint32_t* ghist; unsigned long long* status; SortCtl* ctl; uint32_t* abort_flag; int tile; };
 uint32_t* sort_input(const SortBufs& b) { return b.B; }
 
 // stable sort of every segment [seg_start[t], seg_start[t+1]) by the low `key_bits` bits of the key, the payload being
@@ -261,22 +290,27 @@ void seg_sort(mpe_handle* h, const SortBufs& b, const int32_t* seg_start, const 
               int key_bits, int64_t n_upper, const uint32_t** skey, const uint32_t** sval, bool input_pairs = false) {
     const int T = h->T;
     const int64_t max_tiles = (n_upper + b.tile - 1) / b.tile + T;
-    const int g = grid_for(h, max_tiles, 1, MPE_SORT_MINB);
-    const int gh = grid_for(h, max_tiles, SORT_THREADS / 32, 8);
     const int passes = (key_bits + 7) / 8;
+    const int gh = grid_for(h, max_tiles, SORT_THREADS / 32, 4);
+    if (input_pairs) LAUNCH(h, "sort_digits", k_sort_digits<true>, gh, SORT_THREADS, 0, (const uint32_t*)b.B, seg_start, tile_base, T, passes, b.ghist, b.tile);
+    else LAUNCH(h, "sort_digits", k_sort_digits<false>, gh, SORT_THREADS, 0, (const uint32_t*)b.B, seg_start, tile_base, T, passes, b.ghist, b.tile);
     for (int p = 0; p < passes; ++p) {
         const bool first = p == 0 && !input_pairs, last = p == passes - 1;    // input_pairs: B holds (key, payload) records already
         uint32_t* src = (p & 1) ? b.A : b.B;                      // pass p reads B and writes A when p is even, the other way round when odd
         uint32_t* dst = (p & 1) ? b.B : b.A;
-        if (first) LAUNCH(h, "sort_hist", k_sort_hist<false>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist, b.tile);
-        else LAUNCH(h, "sort_hist", k_sort_hist<true>, gh, SORT_THREADS, 0, (const uint32_t*)src, seg_start, (const int32_t*)tile_base, T, 8 * p, b.hist, b.tile);
-        LAUNCH(h, "sort_offsets", k_sort_offsets, std::min(T, h->num_sms * 2), OFFS_THREADS, 0, b.hist, seg_start, (const int32_t*)tile_base, T);
         const uint32_t* kin = src; const uint2* pin = reinterpret_cast<const uint2*>(src);
         uint2* pout = reinterpret_cast<uint2*>(dst); uint32_t* ok = dst; uint32_t* ov = dst + b.n;
-#define SCATTER(F, L) do { if (b.tile == sort_tile(true)) LAUNCH(h, "sort_scatter", (k_sort_scatter<F, L, SORT_ITEMS_SMALL>), g, SORT_THREADS, 0, kin, pin, pout, ok, ov, seg_start, \
-                                                               (const int32_t*)tile_base, T, 8 * p, (const uint32_t*)b.hist); \
-                           else LAUNCH(h, "sort_scatter", (k_sort_scatter<F, L, SORT_ITEMS_LARGE>), g, SORT_THREADS, 0, kin, pin, pout, ok, ov, seg_start, \
-                                       (const int32_t*)tile_base, T, 8 * p, (const uint32_t*)b.hist); } while (0)
+        // tiles are handed out by ticket, so the grid only has to be large enough to fill the GPU
+#define SCATTER(F, L) do { \
+        if (b.tile == sort_tile(true)) { \
+            auto kern = k_sort_scatter<F, L, SORT_ITEMS_SMALL>; \
+            LAUNCH(h, "sort_scatter", kern, grid_for(h, max_tiles, 1, resident_blocks(h, kern, SORT_THREADS, 0)), SORT_THREADS, 0, kin, pin, pout, ok, ov, \
+                   seg_start, tile_base, T, p, b.ghist, b.status, b.ctl, b.abort_flag); \
+        } else { \
+            auto kern = k_sort_scatter<F, L, SORT_ITEMS_LARGE>; \
+            LAUNCH(h, "sort_scatter", kern, grid_for(h, max_tiles, 1, resident_blocks(h, kern, SORT_THREADS, 0)), SORT_THREADS, 0, kin, pin, pout, ok, ov, \
+                   seg_start, tile_base, T, p, b.ghist, b.status, b.ctl, b.abort_flag); \
+        } } while (0)
         if (first && last) SCATTER(true, true);
         else if (first) SCATTER(true, false);
         else if (last) SCATTER(false, true);
@@ -477,16 +511,20 @@ void enqueue_index_chain(mpe_handle* h, int64_t L_grid, int64_t bags_grid, bool 
     Work& w = h->wk;
     const int T = h->T;
     LAUNCH(h, "prelude", (ind ? k_prelude<true> : k_prelude<false>), 1, 32, 0, w, T, av);
-    const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->hist, h->block_sums, h->wk.sort_tile};
+    const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->ghist, h->sort_status, h->sort_ctl, &h->wk.ctr->abort, h->wk.sort_tile};
     LAUNCH(h, "make_keys", (ind ? k_make_keys<true> : k_make_keys<false>), grid_for(h, bags_grid, 32, 8), 256, 0, s, w, sort_input(sb), av);
     // sort the row indices of the mini-batch (Section 5.1), table by table
     seg_sort(h, sb, w.table_start, w.tile_base, bits_for((uint32_t)h->max_rows), L_grid, &h->skey, &h->spos);
     // distinct rows
     const int gs = grid_for(h, L_grid, SCAN_TILE, 8);
-    LAUNCH(h, "unique_count", k_unique<false>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
-    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);
-    LAUNCH(h, "unique_write", k_unique<true>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
-    LAUNCH(h, "ustart", k_ustart, 1, 256, 0, w, T);
+    if (ind) {
+        LAUNCH(h, "unique", k_unique, gs, SCAN_THREADS, 0, w, T, h->skey, h->sort_status, h->sort_ctl);
+    } else {
+        LAUNCH(h, "unique_count", k_unique_pass<false>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
+        LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);
+        LAUNCH(h, "unique_write", k_unique_pass<true>, gs, SCAN_THREADS, 0, w, T, h->skey, h->block_sums);
+        LAUNCH(h, "ustart", k_ustart, 1, 256, 0, w, T);
+    }
 }
 
 // Second half: tag lookup, then fetch + pool.
@@ -524,13 +562,16 @@ int enqueue_backward(mpe_handle* h, int64_t L, bool ind) {
         LAUNCH_ON(h, h->side, "hot_partial", hot, grid_for(h, hot_capacity(L), 1, 2), 8 * LANES, 32 * s.dim * sizeof(float), s, w, av);
     });
     CK(h, cudaEventRecord(h->ev_join, h->side));
-    const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->hist, h->block_sums, h->wk.sort_tile};
-    LAUNCH(h, "priority", (ind ? k_priority<true> : k_priority<false>), grid_for(h, L, PRI_CHUNK, 8), 256, 0, s, w, h->block_sums, av);
+    const SortBufs sb{h->sortA, h->sortB, h->sort_n, h->ghist, h->sort_status, h->sort_ctl, &h->wk.ctr->abort, h->wk.sort_tile};
+    // new priority values; the rows that may be admitted (few, once the caches are warm) are gathered in row order ...
+    LAUNCH(h, "priority", (ind ? k_priority<true> : k_priority<false>), grid_for(h, L, PRI_CHUNK, 8), 256, 0, s, w,
+           h->max_sets > 0 ? reinterpret_cast<uint2*>(sb.B) : (uint2*)nullptr, h->sort_status, h->sort_ctl, h->block_sums, av);
     if (h->max_sets > 0) {
-        // the rows that may be admitted (few, once the caches are warm) are gathered in row order ...
-        LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, (const uint32_t*)&w.ctr->U, (uint32_t)PRI_CHUNK, &w.ctr->n_cand);
-        LAUNCH(h, "cand_write", k_cand_write, grid_for(h, L, PRI_CHUNK, 8), 256, 0, s, w, (const uint32_t*)h->block_sums, reinterpret_cast<uint2*>(sb.B));
-        LAUNCH(h, "cand_starts", k_cand_starts, 1, 32, 0, w, h->T);
+        if (!ind) {        // large steps: the list is made by three small kernels
+            LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, h->block_sums, (const uint32_t*)&w.ctr->U, (uint32_t)PRI_CHUNK, &w.ctr->n_cand);
+            LAUNCH(h, "cand_write", k_cand_write, grid_for(h, L, PRI_CHUNK, 8), 256, 0, s, w, (const uint32_t*)h->block_sums, reinterpret_cast<uint2*>(sb.B));
+            LAUNCH(h, "cand_starts", k_cand_starts, 1, 32, 0, w, h->T);
+        }
         // ... and grouped by cache set, keeping ascending row id inside a set
         const uint32_t *ck = nullptr, *cv = nullptr;
         seg_sort(h, sb, w.cstart, w.ctile_base, bits_for((uint32_t)h->max_sets), L, &ck, &cv, true);
@@ -604,6 +645,8 @@ int forward_impl(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offse
         int rc = mpe_reserve(h, batch, total_indices);
         if (rc != MPE_OK) return rc;
     }
+    h->sort_passes_bound += 4 * SORT_MAX_PASSES;       // this step's two sorts, and those of a batch prepared meanwhile
+    if (h->sort_passes_bound > SORT_TAG_MASK - 1024) { int rc = renew_sort_tags(h); if (rc != MPE_OK) return rc; }
     Work& w = h->wk;
     uint32_t L = (uint32_t)total_indices;
     h->B = batch; h->L = total_indices; ++h->epoch;
@@ -990,7 +1033,16 @@ int mpe_last_error(mpe_handle* h, int32_t* code, int64_t* detail) {
         CK(h, cudaMemset(&h->alt.wk.ctr->err[0], 0, sizeof(c2.err)));
         c.err[ERR_OFFSETS] += c2.err[ERR_OFFSETS]; c.err[ERR_INDEX] += c2.err[ERR_INDEX];
     }
-    if (c.err[ERR_OFFSETS]) { *code = MPE_ERR_OFFSETS; *detail = (int64_t)c.err[ERR_OFFSETS]; }
+    // a wait inside the sort that ran out (its step was abandoned) outranks the conditions of the inputs
+    uint32_t timeouts = 0;
+    for (SortCtl* ctl : {h->sort_ctl, h->prepared ? nullptr : h->alt.sort_ctl}) {
+        if (!ctl) continue;
+        SortCtl sc;
+        CK(h, cudaMemcpy(&sc, ctl, sizeof(sc), cudaMemcpyDeviceToHost));
+        if (sc.timeout) { timeouts += sc.timeout; CK(h, cudaMemset(&ctl->timeout, 0, sizeof(uint32_t))); }
+    }
+    if (timeouts) { *code = MPE_ERR_TIMEOUT; *detail = (int64_t)timeouts; }
+    else if (c.err[ERR_OFFSETS]) { *code = MPE_ERR_OFFSETS; *detail = (int64_t)c.err[ERR_OFFSETS]; }
     else if (c.err[ERR_INDEX]) { *code = MPE_ERR_INDEX; *detail = (int64_t)c.err[ERR_INDEX]; }
     return MPE_OK;
 }
@@ -1176,9 +1228,8 @@ constexpr int STATIC_MAX_TABLES = MPE_STATIC_MAX_TABLES;
 constexpr size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 constexpr size_t STATIC_SCRATCH_BYTES =
     2 * align256(2 * (STATIC_MAX_INDICES + 4) * 4) + 12 * align256((STATIC_MAX_INDICES + 4) * 4) +                                 // keys, payloads, per-index and per-row maps
-    align256(256 * ((STATIC_MAX_INDICES + sort_tile(true) - 1) / sort_tile(true) + STATIC_MAX_TABLES + 1) * 4) +   // sort histograms
-    align256((256 * ((STATIC_MAX_INDICES + sort_tile(true) - 1) / sort_tile(true) + STATIC_MAX_TABLES + 1) / SCAN_TILE + 2 +
-              STATIC_MAX_INDICES / SCAN_TILE + 2) * 4) +                                               // block sums
+    align256(256 * ((STATIC_MAX_INDICES + sort_tile(true) - 1) / sort_tile(true) + STATIC_MAX_TABLES + 1) * 8) +   // the sort's per-tile words
+    align256(STATIC_MAX_TABLES * SORT_MAX_PASSES * 256 * 4) + align256(sizeof(SortCtl)) +              // its per-table digit counts and its counters
     4 * align256((STATIC_MAX_TABLES + 1) * 4) +                                                        // per-table starts
     2 * align256(hot_capacity(STATIC_MAX_INDICES) * 4) +                                             // hot-row lists
     align256(sizeof(Counters)) + align256(sizeof(StepArgs));
@@ -1188,6 +1239,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_B
 
 constexpr int MAX_DEVICES = 64;
 unsigned char* g_scratch_addr[MAX_DEVICES] = {};     // device address of g_static_scratch, per device, filled on first use
+uint64_t g_scratch_passes[MAX_DEVICES] = {};         // sort passes run in the array so far, per device (an upper bound)
 std::mutex g_scratch_lock;                           // first calls from several host threads fill the table one at a time
 
 struct Carver {
@@ -1207,6 +1259,7 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     if (h->device < 0 || h->device >= MAX_DEVICES) return MPE_ERR_ARG;
     DeviceGuard guard(h->device);
     unsigned char* scratch = nullptr;
+    bool renew_tags = false;          // the pass numbers in the sort's per-tile words are about to come round: start them over
     {
         std::lock_guard<std::mutex> lock(g_scratch_lock);
         if (!g_scratch_addr[h->device]) {
@@ -1216,6 +1269,9 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
             g_scratch_addr[h->device] = static_cast<unsigned char*>(addr);
         }
         scratch = g_scratch_addr[h->device];
+        g_scratch_passes[h->device] += SORT_MAX_PASSES;
+        renew_tags = g_scratch_passes[h->device] > SORT_TAG_MASK - 1024;
+        if (renew_tags) g_scratch_passes[h->device] = 0;
     }
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     if (stream != h->stream) { CK(h, cudaStreamSynchronize(h->stream)); h->stream = stream; }
@@ -1229,8 +1285,9 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     w.uniq_row = c.take<int32_t>(n); w.uniq_t = c.take<int32_t>(n); w.seg = c.take<int32_t>(n); w.loc = c.take<int32_t>(n);
     w.final_loc = c.take<int32_t>(n); w.uset = c.take<int32_t>(n); w.hot_base = c.take<int32_t>(n); w.victim = c.take<int32_t>(n);
     const size_t max_tiles = (STATIC_MAX_INDICES + sort_tile(true) - 1) / sort_tile(true) + STATIC_MAX_TABLES + 1;
-    uint32_t* hist = c.take<uint32_t>(256 * max_tiles);
-    uint32_t* block_sums = c.take<uint32_t>(256 * max_tiles / SCAN_TILE + 2 + STATIC_MAX_INDICES / SCAN_TILE + 2);
+    unsigned long long* sort_status = c.take<unsigned long long>(256 * max_tiles);
+    uint32_t* ghist = c.take<uint32_t>((size_t)STATIC_MAX_TABLES * SORT_MAX_PASSES * 256);
+    SortCtl* sort_ctl = c.take<SortCtl>(1);
     w.table_start = c.take<int32_t>(STATIC_MAX_TABLES + 1); w.tile_base = c.take<int32_t>(STATIC_MAX_TABLES + 1);
     w.ustart = c.take<int32_t>(STATIC_MAX_TABLES + 1); w.ctile_base = c.take<int32_t>(STATIC_MAX_TABLES + 1);
     w.hot_k = c.take<int32_t>(hot_capacity(STATIC_MAX_INDICES)); w.task_k = c.take<int32_t>(hot_capacity(STATIC_MAX_INDICES));
@@ -1244,20 +1301,21 @@ extern "C" int mpe_forward_static(mpe_handle* h, const int32_t* d_indices, const
     ++h->epoch;
     // the array keeps whatever the previous call left: the counters are the only part that must start from zero
     CK(h, cudaMemsetAsync(w.ctr, 0, sizeof(Counters), stream));
+    if (renew_tags) {
+        CK(h, cudaMemsetAsync(sort_status, 0, sizeof(unsigned long long) * 256 * max_tiles, stream));
+        CK(h, cudaMemsetAsync(sort_ctl, 0, sizeof(SortCtl), stream));
+    }
     StepArgs av{};
     av.indices = d_indices; av.offsets = d_offsets; av.out = d_out; av.B = batch; av.L = L; av.epoch = h->epoch;
     w.sort_tile = sort_tile(true);
-    const SortBufs sb{sortA, sortB, (int64_t)n, hist, block_sums, w.sort_tile};
+    const SortBufs sb{sortA, sortB, (int64_t)n, ghist, sort_status, sort_ctl, &w.ctr->abort, w.sort_tile};
     LAUNCH(h, "prelude", k_prelude<false>, 1, 32, 0, w, T, av);
     LAUNCH(h, "make_keys", k_make_keys<false>, grid_for(h, bags, 32, 8), 256, 0, s, w, sort_input(sb), av);
     // segmented radix sort, as in mpe_forward, on the carved buffers
     const uint32_t *skey = nullptr, *spos = nullptr;
     seg_sort(h, sb, w.table_start, w.tile_base, bits_for((uint32_t)h->max_rows), total_indices, &skey, &spos);
     const int gs = grid_for(h, total_indices, SCAN_TILE, 8);
-    LAUNCH(h, "unique_count", k_unique<false>, gs, SCAN_THREADS, 0, w, T, skey, block_sums);
-    LAUNCH(h, "scan_block_sums", k_scan_block_sums, 1, BSUM_THREADS, 0, block_sums, (const uint32_t*)&w.ctr->L, (uint32_t)SCAN_TILE, &w.ctr->U);
-    LAUNCH(h, "unique_write", k_unique<true>, gs, SCAN_THREADS, 0, w, T, skey, block_sums);
-    LAUNCH(h, "ustart", k_ustart, 1, 256, 0, w, T);
+    LAUNCH(h, "unique", k_unique, gs, SCAN_THREADS, 0, w, T, skey, sort_status, sort_ctl);
     LAUNCH(h, "probe", k_probe<false>, grid_for(h, total_indices, 256, 8), 256, 0, s, w, av);
     LAUNCH(h, "broadcast", k_broadcast<false>, grid_for(h, total_indices, 256, 8), 256, 0, s, w, spos, av);
     const int gp = grid_for(h, bags, 256 / s.lanes, 8);

@@ -91,8 +91,8 @@ struct Work {
     int32_t *uniq_row, *uniq_t, *seg, *loc, *final_loc, *victim, *hot_base, *uset;   // per unique row
     int32_t* task_k;       // [hot tasks]
     int32_t* hot_k;        // [hot rows]
-    uint32_t* cand_key;    // [distinct rows] the row's set if it is a candidate for admission, else the table's number of sets
-    int32_t* cand_cnt;     // [T] candidates of each table (counted by k_priority, cleared by k_cand_starts)
+    uint32_t* cand_key;    // [distinct rows] large steps: the row's set if it is a candidate for admission, else the table's number of sets
+    int32_t* cand_cnt;     // [T] candidates of each table (counted by k_priority, cleared once the candidates' segments are known)
     int32_t* cstart;       // [T+1] where each table's candidates begin in the compacted candidate list
     int32_t* defer_k;      // [deferred newcomers]
     int32_t* heads;        // [sets with candidates] position of the set's first candidate in the set-sorted list
@@ -187,9 +187,106 @@ k_make_keys(State s, Work w, uint32_t* __restrict__ keys, StepArgs av) {
 // ---------------------------------------------------------------------------------------------
 // distinct rows of the sorted batch (I_U), multiplicities, element -> distinct-row map
 // ---------------------------------------------------------------------------------------------
+// Small steps (the ones replayed from a graph, where every launch counts), one pass: a tile of the sorted batch flags the first element of every run of equal (table, row), learns how many
+// distinct rows the tiles before it hold (look-back over one word per tile), and writes its part of the lists.  The block
+// that ends the pass fills in where each table's distinct rows begin.
+__global__ void __launch_bounds__(SCAN_THREADS)
+k_unique(Work w, int T, const uint32_t* __restrict__ skey, unsigned long long* __restrict__ words, SortCtl* __restrict__ ctl) {
+    __shared__ uint32_t tmp[SCAN_THREADS / 32 + 1];
+    __shared__ uint32_t s_turn[2];
+    __shared__ uint32_t s_prefix[2];
+    const bool off = w.ctr->abort != 0;                 // an abandoned step has no tiles
+    const uint32_t n = off ? 0u : w.ctr->L;
+    const uint32_t nblk = (n + SCAN_TILE - 1) / SCAN_TILE;
+    uint32_t b, tag;
+    while (draw_tile(ctl, nblk, s_turn, &b, &tag)) {
+        const uint32_t base = b * SCAN_TILE + threadIdx.x * SCAN_ITEMS;
+        uint32_t flag[SCAN_ITEMS];
+        int tcur[SCAN_ITEMS];
+        uint32_t sum = 0;
+        uint32_t keyv[SCAN_ITEMS];
+        if (base < n) {
+            int t = find_segment(w.table_start, T, (int32_t)base);
+            while (w.table_start[t + 1] <= (int32_t)base) ++t;     // skip empty tables that start here
+            uint32_t prev = base > 0 ? skey[base - 1] : 0;
+            if (base + SCAN_ITEMS <= n) {                           // 16 keys as four 16-byte loads
+#pragma unroll
+                for (int i = 0; i < SCAN_ITEMS; i += 4) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(skey + base + i);
+                    keyv[i] = v.x; keyv[i + 1] = v.y; keyv[i + 2] = v.z; keyv[i + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < SCAN_ITEMS; ++i) keyv[i] = base + i < n ? skey[base + i] : 0;
+            }
+#pragma unroll
+            for (int i = 0; i < SCAN_ITEMS; ++i) {
+                const uint32_t e = base + i;
+                flag[i] = 0; tcur[i] = t;
+                if (e < n) {
+                    while (w.table_start[t + 1] <= (int32_t)e) ++t;
+                    tcur[i] = t;
+                    const uint32_t k = keyv[i];
+                    flag[i] = (e == (uint32_t)w.table_start[t] || k != prev) ? 1u : 0u;
+                    prev = k;
+                    sum += flag[i];
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < SCAN_ITEMS; ++i) { flag[i] = 0; tcur[i] = 0; keyv[i] = 0; }
+        }
+        uint32_t total;
+        uint32_t ex = block_exclusive_scan<SCAN_THREADS>(sum, &total, tmp);
+        if (threadIdx.x < 32) {
+            if (threadIdx.x == 0) tile_publish(words, b, total, tag);
+            bool poison;
+            const uint32_t before = tile_look_back(words, b, total, tag, &poison);
+            if (threadIdx.x == 0) { s_prefix[0] = before; s_prefix[1] = poison; }
+        }
+        __syncthreads();
+        if (s_prefix[1]) {                                         // a look-back gave up: write nothing, abandon the step
+            if (threadIdx.x == 0) { atomicAdd(&ctl->timeout, 1u); w.ctr->abort = 1; }
+            continue;
+        }
+        ex += s_prefix[0];
+        if (b == nblk - 1 && threadIdx.x == 0) w.ctr->U = s_prefix[0] + total;
+        uint32_t kout[SCAN_ITEMS];
+#pragma unroll
+        for (int i = 0; i < SCAN_ITEMS; ++i) {
+            const uint32_t e = base + i;
+            ex += flag[i];
+            kout[i] = ex - 1;
+            if (e < n && flag[i]) { w.uniq_row[kout[i]] = (int32_t)keyv[i]; w.uniq_t[kout[i]] = tcur[i]; w.seg[kout[i]] = (int32_t)e; }
+        }
+        if (base + SCAN_ITEMS <= n) {
+#pragma unroll
+            for (int i = 0; i < SCAN_ITEMS; i += 4)
+                *reinterpret_cast<uint4*>(w.kidx + base + i) = make_uint4(kout[i], kout[i + 1], kout[i + 2], kout[i + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < SCAN_ITEMS; ++i) if (base + i < n) w.kidx[base + i] = kout[i];
+        }
+    }
+    if (last_block_of_pass(ctl, s_turn)) {
+        // every tile is done and its results are visible: where each table's distinct rows begin, and the end mark
+        if (!off && !__ldcg(&w.ctr->abort)) {
+            const uint32_t U = __ldcg(&w.ctr->U);
+            for (int t = threadIdx.x; t <= T; t += blockDim.x) {
+                const int32_t s0 = w.table_start[t];
+                w.ustart[t] = (uint32_t)s0 < n ? (int32_t)__ldcg(w.kidx + s0) : (int32_t)U;
+            }
+            if (threadIdx.x == 0) w.seg[U] = (int32_t)n;
+        }
+        close_pass(ctl, tag);
+    }
+}
+
+// Large steps: the same in two passes over the sorted batch with a prefix sum over the tiles' counts between them
+// (count, k_scan_block_sums, write), and one small kernel for the tables' starts; nothing waits for anything there.
 template <bool WRITE>
 __global__ void __launch_bounds__(SCAN_THREADS)
-k_unique(Work w, int T, const uint32_t* __restrict__ skey, uint32_t* __restrict__ block_sums) {
+k_unique_pass(Work w, int T, const uint32_t* __restrict__ skey, uint32_t* __restrict__ block_sums) {
     __shared__ uint32_t tmp[SCAN_THREADS / 32 + 1];
     if (w.ctr->abort) return;
     const uint32_t n = w.ctr->L;
@@ -481,22 +578,55 @@ k_pool(State s, Work w, StepArgs av) {
 constexpr int PRI_Q = 4;                 // independent rows per thread: the counter updates are random accesses
 constexpr int PRI_CHUNK = PRI_Q * 256;   // rows per block and round
 
+// The rows that may be admitted (few, once the caches are warm) are to become a list of (set, distinct-row index)
+// records in the order of the distinct rows (table, then row id).
+// Small steps (the ones replayed from a graph, where every launch counts): the list leaves this kernel.  A chunk learns
+// how many candidates the chunks before it hold by look-back over one word per chunk, and the block that ends the pass
+// turns the per-table candidate counts into the segments and tiles of the sort by set that follows.
+// Large steps: this kernel leaves each row's candidate key and each chunk's number of candidates, and three small kernels
+// (prefix sum, k_cand_write, k_cand_starts) make the list -- waiting for the chunks before costs more there than
+// reading the keys again.
+// pairs == nullptr: no table has a cache, no list.
 template <bool IND>
-__global__ void __launch_bounds__(256)
-k_priority(State s, Work w, uint32_t* __restrict__ block_sums, StepArgs av) {
+__global__ void __launch_bounds__(256, 3)
+k_priority(State s, Work w, uint2* __restrict__ pairs, unsigned long long* __restrict__ words, SortCtl* __restrict__ ctl,
+           uint32_t* __restrict__ block_sums, StepArgs av) {
+    constexpr bool FUSED = IND;
     StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
-    __shared__ uint32_t chunk_cand;
-    if (w.ctr->abort) return;
+    __shared__ uint32_t wcand[8][PRI_Q];        // candidates per warp and round
+    __shared__ uint32_t s_turn[2];
+    __shared__ uint32_t s_prefix[2];
+    __shared__ uint2 stash[2][PRI_CHUNK];       // the candidates of this chunk and of the one before, in row order
+    const bool off = w.ctr->abort != 0;         // an abandoned step has no chunks
     const uint32_t step = (uint32_t)a.step;
     constexpr int Q = PRI_Q;
-    const int64_t U = w.ctr->U;
-    uint32_t* __restrict__ ckey = w.cand_key;
-    if (threadIdx.x == 0) chunk_cand = 0;
-    __syncthreads();
+    const int64_t U = off ? 0 : w.ctr->U;
+    const uint32_t nchunk = (uint32_t)((U + PRI_CHUNK - 1) / PRI_CHUNK);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // A chunk's candidates wait in shared memory while the block works on its next chunk, and go out once that is done:
+    // by then the chunks before it have said how many candidates they hold, so the look-back finds its answer at once.
+    bool have_prev = false; uint32_t prev_chunk = 0, prev_total = 0; int buf = 0;
+    auto write_out = [&](uint32_t chunk_id, uint32_t total, int b) {
+        if (warp == 0) {
+            bool poison;
+            const uint32_t before = tile_look_back(words, chunk_id, total, s_turn[1], &poison);
+            if (lane == 0) { s_prefix[0] = before; s_prefix[1] = poison; }
+        }
+        __syncthreads();
+        if (s_prefix[1]) {                                         // a look-back gave up: write nothing, abandon the step
+            if (threadIdx.x == 0) { atomicAdd(&ctl->timeout, 1u); w.ctr->abort = 1; }
+        } else {
+            for (uint32_t j = threadIdx.x; j < total; j += 256) pairs[s_prefix[0] + j] = stash[b][j];
+        }
+    };
+    uint32_t chunk = blockIdx.x, tag = 0;
     // a block takes PRI_CHUNK consecutive rows at a time, thread i the rows i, i + 256, i + 512, i + 768 of them
-    for (int64_t c0 = (int64_t)blockIdx.x * PRI_CHUNK; c0 < U; c0 += (int64_t)gridDim.x * PRI_CHUNK) {
+    for (;; chunk += gridDim.x) {
+        if (FUSED) { if (!draw_tile(ctl, nchunk, s_turn, &chunk, &tag)) break; }
+        else if (chunk >= nchunk) break;
+        const int64_t c0 = (int64_t)chunk * PRI_CHUNK;
         int t[Q], loc[Q]; int32_t row[Q]; uint32_t mult[Q], old[Q]; int64_t rb[Q], sbase[Q]; int32_t nsets[Q];
-        uint32_t ncand = 0;
+        uint32_t ckey[Q]; uint32_t cmask = 0;
 #pragma unroll
         for (int q = 0; q < Q; ++q) {
             const int64_t k = c0 + q * 256 + threadIdx.x;
@@ -516,32 +646,28 @@ k_priority(State s, Work w, uint32_t* __restrict__ block_sums, StepArgs av) {
         for (int q = 0; q < Q; ++q) {
             const int64_t k = c0 + q * 256 + threadIdx.x;
             unsigned long long m = 0, hitm = 0, uh = 0, un = 0, byp = 0, cand = 0;
-            if (t[q] >= 0) {
-                uint32_t key = (uint32_t)nsets[q];           // not a candidate
-                if (loc[q] != LOC_INVALID) {
-                    m = mult[q]; un = 1;
-                    uint32_t pv = step;                      // the priority value the row has from now on
-                    if (s.policy == 1) {                     // LFU: access count of the row, saturating
-                        pv = old[q] + mult[q] < old[q] ? 0xffffffffU : old[q] + mult[q];
-                        s.cnt[rb[q] + row[q]] = pv;
-                    }
-                    // the cached row's priority value, kept per slot: the LRU time stamp, or a copy of the LFU count (so
-                    // that the policy kernel reads one line per set instead of one counter per resident row)
-                    if (loc[q] >= 0) s.ts[loc[q]] = pv;
-                    if (loc[q] >= 0) { hitm = mult[q]; uh = 1; }
-                    else if (nsets[q] > 0) {
-                        // The lowest priority value in a set never falls (counts and time stamps only grow, a replacement
-                        // puts a larger value in the place of the lowest, no way is ever emptied), so a row that does not
-                        // beat a bound recorded earlier is bypassed whatever happens in this step (Algorithm 2's test).
-                        const int32_t set = w.uset[k];
-                        const bool always = s.ways == 1 && s.policy == 0;
-                        if (!always && pv <= s.floor[sbase[q] + set]) byp = 1;
-                        else { key = (uint32_t)set; cand = 1; }
-                    }
+            ckey[q] = t[q] >= 0 ? (uint32_t)nsets[q] : 0u;           // large steps: "not a candidate"
+            if (t[q] >= 0 && loc[q] != LOC_INVALID) {
+                m = mult[q]; un = 1;
+                uint32_t pv = step;                      // the priority value the row has from now on
+                if (s.policy == 1) {                     // LFU: access count of the row, saturating
+                    pv = old[q] + mult[q] < old[q] ? 0xffffffffU : old[q] + mult[q];
+                    s.cnt[rb[q] + row[q]] = pv;
                 }
-                ckey[k] = key;
+                // the cached row's priority value, kept per slot: the LRU time stamp, or a copy of the LFU count (so
+                // that the policy kernel reads one line per set instead of one counter per resident row)
+                if (loc[q] >= 0) s.ts[loc[q]] = pv;
+                if (loc[q] >= 0) { hitm = mult[q]; uh = 1; }
+                else if (nsets[q] > 0) {
+                    // The lowest priority value in a set never falls (counts and time stamps only grow, a replacement
+                    // puts a larger value in the place of the lowest, no way is ever emptied), so a row that does not
+                    // beat a bound recorded earlier is bypassed whatever happens in this step (Algorithm 2's test).
+                    const int32_t set = w.uset[k];
+                    const bool always = s.ways == 1 && s.policy == 0;
+                    if (!always && pv <= s.floor[sbase[q] + set]) byp = 1;
+                    else { ckey[q] = (uint32_t)set; cand = 1; cmask |= 1u << q; }
+                }
             }
-            ncand += (uint32_t)cand;
             // counters: one atomic per warp when the warp sits inside one table
             if (c0 + q * 256 + (threadIdx.x & ~31) >= U) continue;           // warp-uniform: nothing left for this q
             const int t0 = __shfl_sync(0xffffffffU, t[q], 0);
@@ -552,7 +678,7 @@ k_priority(State s, Work w, uint32_t* __restrict__ block_sums, StepArgs av) {
                     uh += __shfl_xor_sync(0xffffffffU, uh, o); un += __shfl_xor_sync(0xffffffffU, un, o);
                     byp += __shfl_xor_sync(0xffffffffU, byp, o); cand += __shfl_xor_sync(0xffffffffU, cand, o);
                 }
-                if ((threadIdx.x & 31) == 0) {
+                if (lane == 0) {
                     unsigned long long* st = s.stats + (int64_t)t0 * 8;
                     atomicAdd(st + 0, m); atomicAdd(st + 1, hitm); atomicAdd(st + 2, un); atomicAdd(st + 3, uh);
                     if (byp) atomicAdd(st + 6, byp);
@@ -565,12 +691,63 @@ k_priority(State s, Work w, uint32_t* __restrict__ block_sums, StepArgs av) {
                 if (cand) atomicAdd(&w.cand_cnt[t[q]], 1);
             }
         }
-        // candidates of this chunk of rows (for the compaction that follows)
-        ncand = __reduce_add_sync(0xffffffffU, ncand);
-        if ((threadIdx.x & 31) == 0 && ncand) atomicAdd(&chunk_cand, ncand);
+        if (!pairs) continue;
+        if (!FUSED) {
+            // large steps: the keys and the chunk's number of candidates, for the kernels that make the list
+#pragma unroll
+            for (int q = 0; q < Q; ++q) if (t[q] >= 0) w.cand_key[c0 + q * 256 + threadIdx.x] = ckey[q];
+            const uint32_t nc = (uint32_t)__syncthreads_count(cmask & 1u) + (uint32_t)__syncthreads_count(cmask & 2u) +
+                                (uint32_t)__syncthreads_count(cmask & 4u) + (uint32_t)__syncthreads_count(cmask & 8u);
+            if (threadIdx.x == 0) block_sums[chunk] = nc;
+            continue;
+        }
+        // the chunk's candidates in row order: round q's rows come before round q + 1's, a warp's before the next warp's
+        uint32_t below[Q];
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            const uint32_t bq = __ballot_sync(0xffffffffU, (cmask >> q) & 1u);
+            below[q] = (uint32_t)__popc(bq & ((1u << lane) - 1u));
+            if (lane == 0) wcand[warp][q] = (uint32_t)__popc(bq);
+        }
         __syncthreads();
-        if (threadIdx.x == 0) { block_sums[c0 / PRI_CHUNK] = chunk_cand; chunk_cand = 0; }
-        __syncthreads();
+        uint32_t total = 0, mine[Q];
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            mine[q] = total + below[q];
+#pragma unroll
+            for (int v = 0; v < 8; ++v) { const uint32_t c = wcand[v][q]; total += c; if (v < warp) mine[q] += c; }
+        }
+        if (threadIdx.x == 0) tile_publish(words, chunk, total, tag);
+#pragma unroll
+        for (int q = 0; q < Q; ++q)
+            if ((cmask >> q) & 1u) stash[buf][mine[q]] = make_uint2(ckey[q], (uint32_t)(c0 + q * 256 + threadIdx.x));
+        if (have_prev) write_out(prev_chunk, prev_total, buf ^ 1);
+        have_prev = true; prev_chunk = chunk; prev_total = total; buf ^= 1;
+    }
+    if constexpr (FUSED) {
+    if (have_prev) { __syncthreads(); write_out(prev_chunk, prev_total, buf ^ 1); }
+    if (last_block_of_pass(ctl, s_turn)) {
+        // every chunk is done and the per-table candidate counts are complete: where each table's candidates begin in
+        // the list, and the tiles of the sort by set (one warp; the counts are cleared for the next step)
+        if (pairs && warp == 0) {
+            const bool dead = off || __ldcg(&w.ctr->abort) != 0;
+            const int T = s.T;
+            int32_t run = 0;
+            for (int t0 = 0; t0 < T; t0 += 32) {
+                const int tt = t0 + lane;
+                const int32_t c = tt < T ? __ldcg(w.cand_cnt + tt) : 0;
+                int32_t inc = c;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { const int32_t v = __shfl_up_sync(0xffffffffU, inc, o); if (lane >= o) inc += v; }
+                if (tt < T) { w.cstart[tt] = run + inc - c; w.cand_cnt[tt] = 0; }
+                run += __shfl_sync(0xffffffffU, inc, 31);
+            }
+            if (lane == 0) { w.cstart[T] = dead ? 0 : run; w.ctr->n_cand = dead ? 0u : (uint32_t)run; }
+            __syncwarp();
+            warp_tile_bases(w.cstart, T, w.ctile_base, dead, w.sort_tile);
+        }
+        close_pass(ctl, tag);
+    }
     }
 }
 

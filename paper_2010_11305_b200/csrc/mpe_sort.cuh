@@ -1,13 +1,14 @@
-// Segmented stable LSD radix sort and device-wide prefix sums.
+// Segmented stable LSD radix sort, and what a single-pass kernel needs to order its tiles.
 //
 // The batch's indices arrive grouped by table, so sorting "by (table, row)"
 // (Section 5.1: sort the row indices of the mini-batch, then merge duplicates)
 // only has to order the rows inside each table's segment.  Every pass sorts by
 // an 8-bit digit with per-(table, digit, tile) counters, so one pass over the
 // whole array sorts all segments at once and never moves a key out of its
-// segment.  No kernel here waits on another block: a pass is histogram ->
-// offsets (one block per table) -> scatter, three ordinary launches.  A tile is 4096 elements:
-// 16 per thread, ranked by warp (match on the digit, warp-private counters),
+// segment.  One kernel counts the digits of all passes; then a pass is one
+// kernel whose tiles learn their output positions from the tiles before them
+// (bounded look-back over per-tile words).  A tile is 4096 or 2048 elements:
+// 16 or 8 per thread, ranked by warp (match on the digit, warp-private counters),
 // reordered through shared memory so that global writes are runs.
 #pragma once
 #include <cuda_runtime.h>
@@ -88,26 +89,140 @@ __device__ __forceinline__ int find_segment(const int32_t* __restrict__ base, in
     return lo;
 }
 
-// ---- pass 1 of 3: per-(table, digit, tile) counts ------------------------------
-// PAIRS: the keys are the .x members of (key, payload) records (every pass but the first)
+// ---- what one tile tells the tiles behind it ------------------------------------------------
+// A pass hands its tiles out in order (a ticket counter), so a tile's predecessors are always held by blocks that are
+// running.  For each of the 256 digit values a tile publishes one 8-byte word: first how many of its keys have that digit
+// (an "aggregate"), later where its successor's keys of that digit begin (a "prefix").  A tile finds where its own keys
+// begin by walking back over its predecessors' words, adding aggregates until it meets a prefix.  The words carry a tag
+// that changes with every pass, so the array is never cleared: a word with another tag is simply not there yet.
+// Every wait is bounded: a tile that gives up poisons what it publishes, the tiles behind it write nothing, and the
+// step is abandoned with a sticky error.
+constexpr int SORT_MAX_PASSES = 4;
+struct SortCtl {
+    uint32_t seq;        // passes completed on this workspace; pass tags are seq + 1
+    uint32_t ticket;     // next tile to hand out; the block that draws the last ticket of a pass puts it back to 0
+    uint32_t timeout;    // sticky: look-backs that gave up
+    uint32_t done;       // blocks that have finished the current pass
+};
+constexpr uint32_t SORT_TAG_MASK = 0x3fffffffU;
+constexpr unsigned long long SORT_PREFIX = 1ULL << 32, SORT_POISON = 1ULL << 33;
+constexpr int SORT_LOOK = 4;                  // predecessors' words a look-back fetches at a time
+constexpr int SORT_POLL_LIMIT = 1 << 22;      // polls of one word before a look-back gives up (about a second)
+__device__ __forceinline__ unsigned long long sort_word(uint32_t tag, unsigned long long flags, uint32_t value) {
+    return ((unsigned long long)tag << 34) | flags | value;
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+// Hands the calling block its next tile (all threads call); false when none is left.
+// Tickets are drawn when the block is ready for the tile, never ahead of time: the tiles behind a ticket wait for its tile.
+__device__ __forceinline__ bool draw_tile(SortCtl* ctl, uint32_t ntiles, uint32_t* s_turn /* [2], shared */, uint32_t* tile, uint32_t* tag) {
+    __syncthreads();
+    if (threadIdx.x == 0) { s_turn[0] = atomicAdd(&ctl->ticket, 1u); s_turn[1] = (ctl->seq + 1u) & SORT_TAG_MASK; }
+    __syncthreads();
+    *tile = s_turn[0]; *tag = s_turn[1];
+    return *tile < ntiles;
+}
+// After its last draw: true in exactly one block of the grid, the last one to get here.  Every other block's writes are
+// visible to that block (through L2: read them with __ldcg), which ends the pass with close_pass() when it is done.
+__device__ __forceinline__ bool last_block_of_pass(SortCtl* ctl, uint32_t* s_turn) {
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_turn[0] = atomicAdd(&ctl->done, 1u);
+    __syncthreads();
+    return s_turn[0] == gridDim.x - 1u;
+}
+__device__ __forceinline__ void close_pass(SortCtl* ctl, uint32_t tag) {
+    if (threadIdx.x == 0) { ctl->ticket = 0; ctl->done = 0; ctl->seq = tag; }
+}
+
+// One word per tile (the compactions).  tile_publish (one thread): how many items the tile holds, as soon as it is known.
+// tile_look_back (one whole warp, any time later): the sum of `total` over the tiles before `tile`, reading 32 predecessors'
+// words at a time; it leaves the tile's prefix in its word.
+__device__ __forceinline__ void tile_publish(unsigned long long* words, uint32_t tile, uint32_t total, uint32_t tag) {
+    st_relaxed_u64(words + tile, sort_word(tag, tile == 0 ? SORT_PREFIX : 0ULL, total));
+}
+__device__ __forceinline__ uint32_t tile_look_back(unsigned long long* words, uint32_t tile, uint32_t total, uint32_t tag, bool* poison) {
+    const int lane = threadIdx.x & 31;
+    uint32_t sum = 0;
+    bool bad = false;
+    if (tile > 0) {
+        for (int64_t base = (int64_t)tile - 1;; base -= 32) {
+            const int64_t j = base - lane;
+            unsigned long long v = sort_word(tag, SORT_PREFIX, 0);            // before the first tile: nothing
+            if (j >= 0) {
+                v = ld_relaxed_u64(words + j);
+                for (int polls = 0; (uint32_t)(v >> 34) != tag; v = ld_relaxed_u64(words + j)) {
+                    if (++polls > SORT_POLL_LIMIT) { v = SORT_PREFIX | SORT_POISON; break; }
+                    if (polls > 32) __nanosleep(200);
+                }
+            }
+            const uint32_t pm = __ballot_sync(0xffffffffU, (v & SORT_PREFIX) != 0);
+            const int stop = pm ? __ffs(pm) - 1 : 31;                          // nearest predecessor that knows its prefix
+            sum += __reduce_add_sync(0xffffffffU, lane <= stop ? (uint32_t)v : 0u);
+            bad |= __any_sync(0xffffffffU, lane <= stop && (v & SORT_POISON) != 0);
+            if (pm) break;
+        }
+        if (lane == 0) st_relaxed_u64(words + tile, sort_word(tag, SORT_PREFIX | (bad ? SORT_POISON : 0ULL), sum + total));
+    }
+    *poison = bad;
+    return sum;
+}
+
+// Sum of what the `left` tiles before the one that owns `word` hold of this thread's digit, plus where the first of them
+// begins: walks back over their words until it meets a prefix.
+__device__ __forceinline__ uint32_t sort_look_back(const unsigned long long* word, int left, uint32_t tag, bool* poison) {
+    uint32_t sum = 0;
+    bool bad = false;
+    const unsigned long long* q = word - 256;
+    for (bool done = false; !done;) {
+        // several predecessors' words are fetched at once and then read in order, nearest first
+        unsigned long long v[SORT_LOOK];
+#pragma unroll
+        for (int u = 0; u < SORT_LOOK; ++u) v[u] = u < left ? ld_relaxed_u64(q - 256 * u) : 0ULL;
+#pragma unroll
+        for (int u = 0; u < SORT_LOOK; ++u) {
+            if (done) break;
+            for (int polls = 0; (uint32_t)(v[u] >> 34) != tag; v[u] = ld_relaxed_u64(q - 256 * u)) {
+                if (++polls > SORT_POLL_LIMIT) { v[u] = SORT_PREFIX | SORT_POISON; break; }
+                if (polls > 32) __nanosleep(200);
+            }
+            sum += (uint32_t)v[u];
+            bad |= (v[u] & SORT_POISON) != 0;
+            done = (v[u] & SORT_PREFIX) != 0;
+        }
+        q -= 256 * SORT_LOOK; left -= SORT_LOOK;
+    }
+    *poison = bad;
+    return sum;
+}
+
+// ---- before the passes: how many keys of each table have each digit value, for every pass at once ----
+// The counts do not depend on the order of the keys, so one read of the unsorted keys serves all passes.
+// ghist[t][pass][digit] must be zero on entry; the pass that uses a row of it clears it again.
+// PAIRS: the keys are the .x members of (key, payload) records
 template <bool PAIRS>
 __global__ void __launch_bounds__(SORT_THREADS)
-k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base,
-            int T, int shift, uint32_t* __restrict__ hist, int tile_keys) {
-    // one warp per tile: its own 256 counters, eight key loads in flight per lane, no block-wide barrier
+k_sort_digits(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base,
+              int T, int passes, uint32_t* __restrict__ ghist, int tile_keys) {
+    // one warp per tile: its own counters, eight key loads in flight per lane, no block-wide barrier
     constexpr int WARPS = SORT_THREADS / 32;
     constexpr int STRIDE = PAIRS ? 2 : 1;
-    __shared__ uint32_t cnt[WARPS][256];
+    __shared__ uint32_t cnt[WARPS][SORT_MAX_PASSES * 256];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int ntiles = tile_base[T];
     for (int tile = blockIdx.x * WARPS + warp; tile < ntiles; tile += gridDim.x * WARPS) {
         const int t = find_segment(tile_base, T, tile);
         const int local = tile - tile_base[t];
-        const int nt = tile_base[t + 1] - tile_base[t];
         const int32_t start = seg_start[t] + local * tile_keys;
         const int32_t end = min(start + tile_keys, seg_start[t + 1]);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) cnt[warp][i * 32 + lane] = 0;
+        for (int i = lane; i < passes * 256; i += 32) cnt[warp][i] = 0;
         __syncwarp();
         for (int32_t i0 = start + lane; i0 < end; i0 += 32 * 8) {
             uint32_t k[8];
@@ -115,83 +230,16 @@ k_sort_hist(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_s
             for (int q = 0; q < 8; ++q) k[q] = i0 + 32 * q < end ? keys[(size_t)(i0 + 32 * q) * STRIDE] : 0u;
 #pragma unroll
             for (int q = 0; q < 8; ++q)
-                if (i0 + 32 * q < end) atomicAdd(&cnt[warp][(k[q] >> shift) & 255u], 1u);
+                if (i0 + 32 * q < end)
+                    for (int p = 0; p < passes; ++p) atomicAdd(&cnt[warp][p * 256 + ((k[q] >> (8 * p)) & 255u)], 1u);
         }
         __syncwarp();
-        uint32_t* out = hist + (size_t)256 * tile_base[t] + local;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) out[(size_t)(i * 32 + lane) * nt] = cnt[warp][i * 32 + lane];
+        uint32_t* out = ghist + (size_t)t * (SORT_MAX_PASSES * 256);
+        for (int i = lane; i < passes * 256; i += 32) {
+            const uint32_t c = cnt[warp][i];
+            if (c) atomicAdd(out + i, c);
+        }
         __syncwarp();
-    }
-}
-
-// ---- pass 2 of 3: counts -> first global position of every (table, digit, tile) ----------------
-// One block per table.  The counts of table t sit as 256 rows (one per digit value) of nt tiles; the first key of
-// (digit d, tile j) goes to  seg_start[t] + (all keys of the table with a smaller digit) + (keys with digit d in the
-// tiles before j).  A warp takes rows d = warp, warp + 32, ...: an exclusive prefix sum along the row, the row totals
-// to shared memory, then the prefix sum over the 256 totals, then the rows again to add their base.
-constexpr int OFFS_THREADS = 1024;
-constexpr int OFFS_SMALL_NT = 32;        // up to this many tiles in a table: one thread per digit value
-__global__ void __launch_bounds__(OFFS_THREADS)
-k_sort_offsets(uint32_t* __restrict__ hist, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base, int T) {
-    __shared__ uint32_t total[256];
-    __shared__ uint32_t scan_tmp[OFFS_THREADS / 32 + 1];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int t = blockIdx.x; t < T; t += gridDim.x) {
-        const int nt = tile_base[t + 1] - tile_base[t];
-        if (nt == 0) continue;                                   // block-uniform
-        uint32_t* __restrict__ rows = hist + (size_t)256 * tile_base[t];
-        if (nt <= OFFS_SMALL_NT) {
-            // few tiles: one thread per digit value walks its row (eight loads in flight at a time)
-            uint32_t* __restrict__ row = rows + (size_t)threadIdx.x * nt;
-            uint32_t sum = 0;
-            if (threadIdx.x < 256) {
-                for (int j0 = 0; j0 < nt; j0 += 8) {
-                    uint32_t v[8];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) v[q] = j0 + q < nt ? row[j0 + q] : 0u;
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) { if (j0 + q < nt) row[j0 + q] = sum; sum += v[q]; }
-                }
-            }
-            uint32_t all;
-            const uint32_t base = block_exclusive_scan<OFFS_THREADS>(threadIdx.x < 256 ? sum : 0u, &all, scan_tmp) + (uint32_t)seg_start[t];
-            if (threadIdx.x < 256) {
-                for (int j0 = 0; j0 < nt; j0 += 8) {
-                    uint32_t v[8];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) v[q] = j0 + q < nt ? row[j0 + q] : 0u;
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) if (j0 + q < nt) row[j0 + q] = v[q] + base;
-                }
-            }
-            continue;
-        }
-        for (int d = warp; d < 256; d += OFFS_THREADS / 32) {
-            uint32_t* __restrict__ row = rows + (size_t)d * nt;
-            uint32_t carry = 0;
-            for (int j0 = 0; j0 < nt; j0 += 32) {
-                const uint32_t v = j0 + lane < nt ? row[j0 + lane] : 0u;
-                uint32_t inc = v;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) { const uint32_t n = __shfl_up_sync(0xffffffffU, inc, o); if (lane >= o) inc += n; }
-                if (j0 + lane < nt) row[j0 + lane] = carry + inc - v;
-                carry += __shfl_sync(0xffffffffU, inc, 31);
-            }
-            if (lane == 0) total[d] = carry;
-        }
-        __syncthreads();
-        uint32_t all;
-        const uint32_t mine = threadIdx.x < 256 ? total[threadIdx.x] : 0u;
-        const uint32_t ex = block_exclusive_scan<OFFS_THREADS>(mine, &all, scan_tmp);
-        if (threadIdx.x < 256) total[threadIdx.x] = ex + (uint32_t)seg_start[t];
-        __syncthreads();
-        for (int d = warp; d < 256; d += OFFS_THREADS / 32) {
-            uint32_t* __restrict__ row = rows + (size_t)d * nt;
-            const uint32_t base = total[d];
-            for (int j = lane; j < nt; j += 32) row[j] += base;
-        }
-        __syncthreads();
     }
 }
 
@@ -205,22 +253,31 @@ template <bool FIRST, bool LAST, int SORT_ITEMS>
 __global__ void __launch_bounds__(SORT_THREADS, MPE_SORT_MINB)
 k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint2* __restrict__ pairs_in, uint2* __restrict__ pairs_out,
                uint32_t* __restrict__ out_keys, uint32_t* __restrict__ out_vals,
-               const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base, int T, int shift,
-               const uint32_t* __restrict__ hist_scanned) {
+               const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base, int T, int pass,
+               uint32_t* __restrict__ ghist, unsigned long long* __restrict__ status, SortCtl* __restrict__ ctl,
+               uint32_t* __restrict__ abort_flag) {
     constexpr int WARPS = SORT_THREADS / 32;
     constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;
     __shared__ uint32_t wcnt[WARPS][256];      // per-warp digit counters, then tile-local position of the warp's first key of each digit
     __shared__ uint32_t goff[256];             // first global position of each digit of this tile minus its tile-local start
     __shared__ uint2 skv[SORT_TILE];
     __shared__ uint32_t scan_tmp[SORT_THREADS / 32 + 1];
+    __shared__ uint32_t s_ticket[2];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
     const int ntiles = tile_base[T];
+    const int shift = 8 * pass;
     volatile uint32_t* myc = wcnt[warp];
-    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    for (;;) {
+        uint32_t ticket, tag;
+        if (!draw_tile(ctl, (uint32_t)ntiles, s_ticket, &ticket, &tag)) {
+            // every block draws one ticket too many; the block that draws the last of those ends the pass
+            if (ticket == (uint32_t)ntiles + gridDim.x - 1u) close_pass(ctl, tag);
+            break;
+        }
+        const int tile = (int)ticket;
         const int t = find_segment(tile_base, T, tile);
         const int local = tile - tile_base[t];
-        const int nt = tile_base[t + 1] - tile_base[t];
         const int32_t start = seg_start[t] + local * SORT_TILE;
         const int32_t count = min(SORT_TILE, seg_start[t + 1] - start);
         // warp w owns elements [w*32*ITEMS, (w+1)*32*ITEMS) of the tile, item i of lane l is w*32*ITEMS + i*32 + l,
@@ -245,7 +302,6 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint2* __restrict__ p
                 }
             }
         }
-        const uint32_t gb = hist_scanned[(size_t)256 * tile_base[t] + (size_t)threadIdx.x * nt + local];   // digit threadIdx.x
 #pragma unroll
         for (int i = 0; i < 8; ++i) wcnt[warp][i * 32 + lane] = 0;
         __syncwarp();
@@ -269,6 +325,9 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint2* __restrict__ p
         uint32_t tot = 0;
 #pragma unroll
         for (int w = 0; w < WARPS; ++w) tot += wcnt[w][threadIdx.x];
+        // tell the tiles behind this one how many keys of digit d it holds, as early as possible
+        unsigned long long* word = status + (size_t)tile * 256 + threadIdx.x;
+        if (local != 0) st_relaxed_u64(word, sort_word(tag, 0, tot));
         uint32_t all;
         const uint32_t ds = block_exclusive_scan<SORT_THREADS>(tot, &all, scan_tmp);
         uint32_t run = ds;
@@ -278,7 +337,6 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint2* __restrict__ p
             wcnt[w][threadIdx.x] = run;
             run += c;
         }
-        goff[threadIdx.x] = gb - ds;                                           // global position = goff + tile-local position
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < SORT_ITEMS; ++i) {
@@ -286,7 +344,25 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint2* __restrict__ p
             const uint32_t r = (i & 1) ? rank[i >> 1] >> 16 : rank[i >> 1] & 0xffffu;
             skv[wcnt[warp][dg] + r] = make_uint2(key[i], val[i]);
         }
-        __syncthreads();
+        // where this tile's keys of digit d begin in the output (the tile is in order in shared memory by now, so the
+        // waiting is done with nothing else left to do)
+        uint32_t gb;
+        bool poison = false;
+        if (local == 0) {
+            // first tile of its table: the table's start plus its keys with a smaller digit
+            uint32_t* g = ghist + ((size_t)t * SORT_MAX_PASSES + pass) * 256 + threadIdx.x;
+            const uint32_t mine = *g;
+            *g = 0;
+            gb = (uint32_t)seg_start[t] + block_exclusive_scan<SORT_THREADS>(mine, &all, scan_tmp);
+        } else {
+            gb = sort_look_back(word, local, tag, &poison);
+        }
+        st_relaxed_u64(word, sort_word(tag, SORT_PREFIX | (poison ? SORT_POISON : 0ULL), gb + tot));
+        goff[threadIdx.x] = gb - ds;                                           // global position = goff + tile-local position
+        if (__syncthreads_or(poison)) {                                        // a look-back gave up: write nothing, abandon the step
+            if (threadIdx.x == 0) { atomicAdd(&ctl->timeout, 1u); *abort_flag = 1; }
+            continue;
+        }
         // padding keys follow every real key of the tile, so positions [0,count) are real
         for (int j = threadIdx.x; j < count; j += SORT_THREADS) {
             const uint2 kv = skv[j];
@@ -294,7 +370,6 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint2* __restrict__ p
             if (LAST) { out_keys[dst] = kv.x; out_vals[dst] = kv.y; }
             else pairs_out[dst] = kv;
         }
-        __syncthreads();
     }
 }
 
