@@ -588,7 +588,7 @@ constexpr int PRI_CHUNK = PRI_Q * 256;   // rows per block and round
 // reading the keys again.
 // pairs == nullptr: no table has a cache, no list.
 template <bool IND>
-__global__ void __launch_bounds__(256, 3)
+__global__ void __launch_bounds__(256, IND ? 2 : 3)
 k_priority(State s, Work w, uint2* __restrict__ pairs, unsigned long long* __restrict__ words, SortCtl* __restrict__ ctl,
            uint32_t* __restrict__ block_sums, StepArgs av) {
     constexpr bool FUSED = IND;
@@ -692,15 +692,14 @@ k_priority(State s, Work w, uint2* __restrict__ pairs, unsigned long long* __res
             }
         }
         if (!pairs) continue;
-        if (!FUSED) {
+        if constexpr (!FUSED) {
             // large steps: the keys and the chunk's number of candidates, for the kernels that make the list
 #pragma unroll
             for (int q = 0; q < Q; ++q) if (t[q] >= 0) w.cand_key[c0 + q * 256 + threadIdx.x] = ckey[q];
             const uint32_t nc = (uint32_t)__syncthreads_count(cmask & 1u) + (uint32_t)__syncthreads_count(cmask & 2u) +
                                 (uint32_t)__syncthreads_count(cmask & 4u) + (uint32_t)__syncthreads_count(cmask & 8u);
             if (threadIdx.x == 0) block_sums[chunk] = nc;
-            continue;
-        }
+        } else {
         // the chunk's candidates in row order: round q's rows come before round q + 1's, a warp's before the next warp's
         uint32_t below[Q];
 #pragma unroll
@@ -723,6 +722,7 @@ k_priority(State s, Work w, uint2* __restrict__ pairs, unsigned long long* __res
             if ((cmask >> q) & 1u) stash[buf][mine[q]] = make_uint2(ckey[q], (uint32_t)(c0 + q * 256 + threadIdx.x));
         if (have_prev) write_out(prev_chunk, prev_total, buf ^ 1);
         have_prev = true; prev_chunk = chunk; prev_total = total; buf ^= 1;
+        }
     }
     if constexpr (FUSED) {
     if (have_prev) { __syncthreads(); write_out(prev_chunk, prev_total, buf ^ 1); }

@@ -205,7 +205,8 @@ __device__ __forceinline__ uint32_t sort_look_back(const unsigned long long* wor
 
 // ---- before the passes: how many keys of each table have each digit value, for every pass at once ----
 // The counts do not depend on the order of the keys, so one read of the unsorted keys serves all passes.
-// ghist[t][pass][digit] must be zero on entry; the pass that uses a row of it clears it again.
+// ghist[t][pass][digit] must be zero on entry; the pass that uses a row of it clears it again, and a pass that finds the
+// step abandoned clears all of its rows.
 // PAIRS: the keys are the .x members of (key, payload) records
 template <bool PAIRS>
 __global__ void __launch_bounds__(SORT_THREADS)
@@ -265,14 +266,19 @@ k_sort_scatter(const uint32_t* __restrict__ keys_in, const uint2* __restrict__ p
     __shared__ uint32_t s_ticket[2];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
-    const int ntiles = tile_base[T];
+    const bool off = *abort_flag != 0;          // the step was abandoned before this pass: nothing to sort
+    const int ntiles = off ? 0 : tile_base[T];
     const int shift = 8 * pass;
     volatile uint32_t* myc = wcnt[warp];
     for (;;) {
         uint32_t ticket, tag;
         if (!draw_tile(ctl, (uint32_t)ntiles, s_ticket, &ticket, &tag)) {
             // every block draws one ticket too many; the block that draws the last of those ends the pass
-            if (ticket == (uint32_t)ntiles + gridDim.x - 1u) close_pass(ctl, tag);
+            if (ticket == (uint32_t)ntiles + gridDim.x - 1u) {
+                if (off)            // the digit counts of this pass were never used: they must not meet the next step's
+                    for (int i = threadIdx.x; i < T * 256; i += SORT_THREADS) ghist[((size_t)(i >> 8) * SORT_MAX_PASSES + pass) * 256 + (i & 255)] = 0;
+                close_pass(ctl, tag);
+            }
             break;
         }
         const int tile = (int)ticket;
