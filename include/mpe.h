@@ -253,6 +253,18 @@ int mpe_memory_bytes(mpe_handle* h, uint64_t* out6);
 /* Device memory the handle holds beyond the model state: out2 = {bytes of the per-step workspace (sized by
  * mpe_reserve or by the largest batch seen; twice that once mpe_prepare has been used), bytes of the two staging sets of mpe_step_host / _submit}. */
 int mpe_workspace_bytes(mpe_handle* h, uint64_t* out2);
+
+/* Self-checks of the library's own safety nets, for tests.  They change no table, cache or policy state and need the
+ * workspace to exist (after mpe_reserve or a forward; else MPE_ERR_SEQUENCE).
+ *   MPE_SELFTEST_LOOK_BACK_TIMEOUT: on the handle's stream, one warp performs the sort's look-back for a tile whose
+ *     predecessor belongs to nobody, with the wait cut to a few thousand polls (about a millisecond).  The wait gives
+ *     up as designed: the next mpe_last_error reports MPE_ERR_TIMEOUT with detail 1, exactly as after a real one, and
+ *     the handle goes on working.  Nothing hangs or faults.  Not between a forward and its backward.
+ *   MPE_SELFTEST_RENEW_TAGS: the next mpe_forward starts the sort's pass numbers over (waits for the device, clears the
+ *     per-tile words), which otherwise happens once in hundreds of millions of steps. */
+#define MPE_SELFTEST_LOOK_BACK_TIMEOUT 1
+#define MPE_SELFTEST_RENEW_TAGS 2
+int mpe_selftest(mpe_handle* h, int32_t which);
 /* Geometry of table `table`'s cache. */
 int mpe_cache_geometry(mpe_handle* h, int32_t table, int32_t* n_sets, int32_t* ways);
 /* Figures of the last step: out6 = {valid indices, distinct rows, dropped indices, rows whose gradient

@@ -18,12 +18,13 @@ LRU, LFU = 0, 1
 SGD, ROWWISE_ADAGRAD = 0, 1
 ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
 TABLE_DEVICE, TABLE_HOST = 0, 1
+SELFTEST_LOOK_BACK_TIMEOUT, SELFTEST_RENEW_TAGS = 1, 2
 OK, ERR_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_SEQUENCE, ERR_INDEX, ERR_OFFSETS, ERR_NOMEM, ERR_TOO_LARGE, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6, -7, -8, -9
 STATIC_MAX_INDICES, STATIC_MAX_BAGS, STATIC_MAX_TABLES = 32768, 32768, 64
 
 EXPORTS = [
     "mpe_create", "mpe_create_placed", "mpe_reserve", "mpe_prepare", "mpe_forward", "mpe_forward_static", "mpe_backward", "mpe_set_rounding", "mpe_step_host", "mpe_step_host_submit", "mpe_step_host_wait", "mpe_flush", "mpe_destroy",
-    "mpe_last_error", "mpe_stats", "mpe_memory_bytes", "mpe_workspace_bytes", "mpe_cache_geometry", "mpe_step_info", "mpe_export_rows",
+    "mpe_last_error", "mpe_stats", "mpe_memory_bytes", "mpe_workspace_bytes", "mpe_selftest", "mpe_cache_geometry", "mpe_step_info", "mpe_export_rows",
     "mpe_export_cache", "mpe_export_aux", "mpe_use_graphs", "mpe_kernel_launches", "mpe_profile", "mpe_profile_read",
     "mpe_forward_routed", "mpe_gather_grad", "mpe_peer_buffer_alloc", "mpe_peer_buffer_open", "mpe_peer_buffer_close", "mpe_peer_buffer_free",
     "mpe_error_string",
@@ -59,6 +60,7 @@ _lib.mpe_last_error.argtypes = [_vp, C.POINTER(_i32), C.POINTER(_i64)]
 _lib.mpe_stats.argtypes = [_vp, _i32, _vp]
 _lib.mpe_memory_bytes.argtypes = [_vp, _vp]
 _lib.mpe_workspace_bytes.argtypes = [_vp, _vp]
+_lib.mpe_selftest.argtypes = [_vp, C.c_int32]
 _lib.mpe_cache_geometry.argtypes = [_vp, _i32, C.POINTER(_i32), C.POINTER(_i32)]
 _lib.mpe_step_info.argtypes = [_vp, _vp]
 _lib.mpe_export_rows.argtypes = [_vp, _i32, _vp, _i64, _vp, _vp, _vp]
@@ -184,6 +186,9 @@ class Mpe:
         code, detail = _i32(), _i64()
         _check(_lib.mpe_last_error(self._h, C.byref(code), C.byref(detail)), "mpe_last_error")
         return code.value, detail.value
+
+    def selftest(self, which):
+        _check(_lib.mpe_selftest(self._h, which), "mpe_selftest")
 
     def stats(self, table):
         out = np.zeros(8, np.uint64)

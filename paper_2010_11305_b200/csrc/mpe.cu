@@ -365,6 +365,7 @@ const char* mpe_error_string(int code) {
         case MPE_ERR_OFFSETS: return "inconsistent offsets";
         case MPE_ERR_NOMEM: return "out of memory";
         case MPE_ERR_TOO_LARGE: return "batch larger than the fixed scratch of mpe_forward_static";
+        case MPE_ERR_TIMEOUT: return "a bounded wait between thread blocks ran out";
         default: return "unknown error";
     }
 }
@@ -1069,6 +1070,23 @@ int mpe_memory_bytes(mpe_handle* h, uint64_t* out6) {
     out6[4] = h->optimizer == MPE_ROWWISE_ADAGRAD ? N * 4 : 0;
     out6[5] = N * 4 * d;
     return MPE_OK;
+}
+
+int mpe_selftest(mpe_handle* h, int32_t which) {
+    if (!h) return MPE_ERR_ARG;
+    if (!h->sort_ctl) return MPE_ERR_SEQUENCE;          // the workspace comes with mpe_reserve or the first forward
+    DeviceGuard guard(h->device);
+    if (which == MPE_SELFTEST_LOOK_BACK_TIMEOUT) {
+        if (h->have_forward) return MPE_ERR_SEQUENCE;
+        LAUNCH(h, "selftest", k_selftest_look_back, 1, 32, 0, h->sort_status, h->sort_ctl);
+        ++h->sort_passes_bound;
+        return check_launch(h);
+    }
+    if (which == MPE_SELFTEST_RENEW_TAGS) {
+        h->sort_passes_bound = SORT_TAG_MASK;           // the next forward starts the pass numbers over
+        return MPE_OK;
+    }
+    return MPE_ERR_ARG;
 }
 
 int mpe_workspace_bytes(mpe_handle* h, uint64_t* out2) {

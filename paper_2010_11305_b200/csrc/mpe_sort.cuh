@@ -148,7 +148,8 @@ __device__ __forceinline__ void close_pass(SortCtl* ctl, uint32_t tag) {
 __device__ __forceinline__ void tile_publish(unsigned long long* words, uint32_t tile, uint32_t total, uint32_t tag) {
     st_relaxed_u64(words + tile, sort_word(tag, tile == 0 ? SORT_PREFIX : 0ULL, total));
 }
-__device__ __forceinline__ uint32_t tile_look_back(unsigned long long* words, uint32_t tile, uint32_t total, uint32_t tag, bool* poison) {
+__device__ __forceinline__ uint32_t tile_look_back(unsigned long long* words, uint32_t tile, uint32_t total, uint32_t tag, bool* poison,
+                                                   int poll_limit = SORT_POLL_LIMIT) {
     const int lane = threadIdx.x & 31;
     uint32_t sum = 0;
     bool bad = false;
@@ -159,7 +160,7 @@ __device__ __forceinline__ uint32_t tile_look_back(unsigned long long* words, ui
             if (j >= 0) {
                 v = ld_relaxed_u64(words + j);
                 for (int polls = 0; (uint32_t)(v >> 34) != tag; v = ld_relaxed_u64(words + j)) {
-                    if (++polls > SORT_POLL_LIMIT) { v = SORT_PREFIX | SORT_POISON; break; }
+                    if (++polls > poll_limit) { v = SORT_PREFIX | SORT_POISON; break; }
                     if (polls > 32) __nanosleep(200);
                 }
             }
@@ -402,6 +403,21 @@ k_scan_block_sums(uint32_t* __restrict__ block_sums, const uint32_t* __restrict_
         carry += total;
     }
     if (threadIdx.x == 0 && total_out) *total_out = carry;
+}
+
+// ---- self-check of the bounded wait ----------------------------------------------------------
+// One warp plays tile 1 of a pass whose tile 0 belongs to nobody, with the wait cut to a few thousand polls (about a
+// millisecond): the look-back has to give up and say so.  The pass number moves on afterwards, so the word it leaves
+// can never be taken for one of a real pass.
+__global__ void k_selftest_look_back(unsigned long long* words, SortCtl* ctl) {
+    if (blockIdx.x != 0 || threadIdx.x >= 32) return;
+    const uint32_t tag = (ctl->seq + 1u) & SORT_TAG_MASK;
+    bool poison = false;
+    tile_look_back(words, 1u, 0u, tag, &poison, 4096);
+    if (threadIdx.x == 0) {
+        if (poison) atomicAdd(&ctl->timeout, 1u);
+        ctl->seq = tag;
+    }
 }
 
 }  // namespace mpe

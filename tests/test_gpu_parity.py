@@ -439,6 +439,82 @@ def test_launch_mode_cannot_change_between_a_forward_and_its_backward():
     assert h.last_error() == (0, 0)
 
 
+def test_a_look_back_that_gives_up_is_reported_and_the_handle_goes_on():
+    """The sort's tiles learn their output positions from the tiles before them; every such wait is bounded.  The
+    library's self-check makes one wait run out (a tile nobody owns, the limit cut to a millisecond): the condition must
+    arrive through mpe_last_error, be cleared by it, and leave the handle training exactly as the oracle does."""
+    from parity_util import make_pair, compare_state
+    from paper_2010_11305_b200 import binding as mpe
+    cfg = _cfg(num_rows=[6000, 700], dim=16, bits=8, batch=96, bag=("poisson", 5.0), zipf=[1.1, 1.0], policy=wl.LRU, ways=4,
+               cache_fraction=0.1, seed=21)
+    rng = np.random.default_rng(0)
+    for graphs in (True, False):
+        h, o = make_pair(cfg)
+        h.use_graphs(graphs)
+        st = wl.Stream(cfg, "cpu")
+        with pytest.raises(mpe.MpeError) as e:          # no workspace yet
+            h.selftest(mpe.SELFTEST_LOOK_BACK_TIMEOUT)
+        assert e.value.code == mpe.ERR_SEQUENCE
+        for step in range(1, 7):
+            idx, off, grad = st.batch(step)
+            out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, device="cuda")
+            h.forward(idx.cuda(), off.cuda(), cfg.batch, out)
+            if step == 3:
+                with pytest.raises(mpe.MpeError) as e:  # not in the middle of a step
+                    h.selftest(mpe.SELFTEST_LOOK_BACK_TIMEOUT)
+                assert e.value.code == mpe.ERR_SEQUENCE
+            h.backward(grad.cuda(), cfg.lr, step)
+            assert np.array_equal(out.cpu().numpy(), o.forward(idx.numpy(), off.numpy(), cfg.batch))
+            o.backward(grad.numpy(), cfg.lr, step)
+            if step in (2, 4):
+                assert h.last_error() == (0, 0)
+                h.selftest(mpe.SELFTEST_LOOK_BACK_TIMEOUT)
+                if step == 4:
+                    h.selftest(mpe.SELFTEST_LOOK_BACK_TIMEOUT)
+                assert h.last_error() == (mpe.ERR_TIMEOUT, 1 if step == 2 else 2)
+                assert h.last_error() == (0, 0)
+        compare_state(h, o, cfg, [0, 1], rng)
+        assert h.last_error() == (0, 0)
+        h.close()
+
+
+def test_sort_pass_numbers_can_start_over_at_any_step():
+    """The per-tile words of the sort carry a pass number that is started over long before it can repeat; forcing that
+    between arbitrary steps (also with a batch prepared ahead in the second workspace) must not change any result."""
+    from parity_util import make_pair, compare_state
+    from paper_2010_11305_b200 import binding as mpe
+    cfg = _cfg(num_rows=[9000, 1200, 50], dim=32, bits=4, batch=300, bag=("poisson", 6.0), zipf=[1.1, 1.0, None], policy=wl.LFU,
+               ways=8, cache_fraction=0.1, seed=22)
+    rng = np.random.default_rng(0)
+    for graphs in (True, False):
+        h, o = make_pair(cfg)
+        h.use_graphs(graphs)
+        st = wl.Stream(cfg, "cpu")
+        side = torch.cuda.Stream()
+        batches = [tuple(x.cuda() for x in st.batch(step)) for step in range(1, 10)]
+        host = [st.batch(step) for step in range(1, 10)]
+        for i, step in enumerate(range(1, 10)):
+            idx, off, grad = batches[i]
+            if step in (1, 4, 5, 8):
+                if step > 1:
+                    h.selftest(mpe.SELFTEST_RENEW_TAGS)
+                else:
+                    h.reserve(cfg.batch, max(int(b[0].numel()) for b in batches))
+                    h.selftest(mpe.SELFTEST_RENEW_TAGS)
+            out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, device="cuda")
+            h.forward(idx, off, cfg.batch, out)
+            if i + 1 < len(batches):
+                h.prepare(batches[i + 1][0], batches[i + 1][1], cfg.batch, side.cuda_stream)
+            h.backward(grad, cfg.lr, step)
+            hi, ho, hg = host[i]
+            assert np.array_equal(out.cpu().numpy(), o.forward(hi.numpy(), ho.numpy(), cfg.batch))
+            o.backward(hg.numpy(), cfg.lr, step)
+        compare_state(h, o, cfg, [0, 1, 2], rng)
+        assert h.last_error() == (0, 0)
+        torch.cuda.synchronize()
+        h.close()
+
+
 def test_graph_replay_and_plain_launches_agree_with_the_oracle():
     """Small steps are replayed from a captured CUDA graph; the same handle must give the oracle's results when
     the batch shrinks and grows under one graph, when the workspace regrows, and with graphs switched off."""
