@@ -291,9 +291,10 @@ void seg_sort(mpe_handle* h, const SortBufs& b, const int32_t* seg_start, const 
     const int T = h->T;
     const int64_t max_tiles = (n_upper + b.tile - 1) / b.tile + T;
     const int passes = (key_bits + 7) / 8;
-    const int gh = grid_for(h, max_tiles, SORT_THREADS / 32, 4);
-    if (input_pairs) LAUNCH(h, "sort_digits", k_sort_digits<true>, gh, SORT_THREADS, 0, (const uint32_t*)b.B, seg_start, tile_base, T, passes, b.ghist, b.tile);
-    else LAUNCH(h, "sort_digits", k_sort_digits<false>, gh, SORT_THREADS, 0, (const uint32_t*)b.B, seg_start, tile_base, T, passes, b.ghist, b.tile);
+    const int split = b.tile == sort_tile(true) ? 4 : 1;         // pieces of a tile the digit count hands to its warps
+    const int gh = grid_for(h, max_tiles * split, SORT_THREADS / 32, 4);
+    if (input_pairs) LAUNCH(h, "sort_digits", k_sort_digits<true>, gh, SORT_THREADS, 0, (const uint32_t*)b.B, seg_start, tile_base, T, passes, b.ghist, b.tile, split);
+    else LAUNCH(h, "sort_digits", k_sort_digits<false>, gh, SORT_THREADS, 0, (const uint32_t*)b.B, seg_start, tile_base, T, passes, b.ghist, b.tile, split);
     for (int p = 0; p < passes; ++p) {
         const bool first = p == 0 && !input_pairs, last = p == passes - 1;    // input_pairs: B holds (key, payload) records already
         uint32_t* src = (p & 1) ? b.A : b.B;                      // pass p reads B and writes A when p is even, the other way round when odd

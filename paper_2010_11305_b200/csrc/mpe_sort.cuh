@@ -212,18 +212,23 @@ __device__ __forceinline__ uint32_t sort_look_back(const unsigned long long* wor
 template <bool PAIRS>
 __global__ void __launch_bounds__(SORT_THREADS)
 k_sort_digits(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ tile_base,
-              int T, int passes, uint32_t* __restrict__ ghist, int tile_keys) {
-    // one warp per tile: its own counters, eight key loads in flight per lane, no block-wide barrier
+              int T, int passes, uint32_t* __restrict__ ghist, int tile_keys, int split) {
+    // one warp per piece of a tile (`split` pieces per tile: whole tiles in large steps, where the cost of emptying the
+    // counters wants many keys to spread over; quarters in small steps, where whole tiles would leave most SMs idle):
+    // its own counters, eight key loads in flight per lane, no block-wide barrier
     constexpr int WARPS = SORT_THREADS / 32;
     constexpr int STRIDE = PAIRS ? 2 : 1;
     __shared__ uint32_t cnt[WARPS][SORT_MAX_PASSES * 256];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int ntiles = tile_base[T];
-    for (int tile = blockIdx.x * WARPS + warp; tile < ntiles; tile += gridDim.x * WARPS) {
+    const int npieces = tile_base[T] * split;
+    const int piece_keys = tile_keys / split;
+    for (int piece = blockIdx.x * WARPS + warp; piece < npieces; piece += gridDim.x * WARPS) {
+        const int tile = piece / split;
         const int t = find_segment(tile_base, T, tile);
         const int local = tile - tile_base[t];
-        const int32_t start = seg_start[t] + local * tile_keys;
-        const int32_t end = min(start + tile_keys, seg_start[t + 1]);
+        const int32_t start = seg_start[t] + local * tile_keys + (piece - tile * split) * piece_keys;
+        const int32_t end = min(start + piece_keys, seg_start[t + 1]);
+        if (start >= end) continue;                    // warp-uniform: the table's last tile is not full
         for (int i = lane; i < passes * 256; i += 32) cnt[warp][i] = 0;
         __syncwarp();
         for (int32_t i0 = start + lane; i0 < end; i0 += 32 * 8) {
