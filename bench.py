@@ -44,10 +44,10 @@ KERNEL_EVIDENCE = {
     "hot_partial": {"dram_bytes_per_index": 20.9, "bound": "l2-latency",
                     "evidence": "gradient rows come from L2 (83 % hits, 36 % of its throughput), 11.2 long-scoreboard stall cycles per issue at 24 % of the warp slots (kept small on purpose: it runs beside other kernels)",
                     "profile": "profiles/k_hot_partial_cfg4_8tables.md"},
-    # on the 8-table case a pass of the sort is L2 resident, so its DRAM traffic does not scale to the full size: none given
-    "sort_scatter": {"dram_bytes_per_index": None, "bound": "shared-memory latency",
-                     "evidence": "10.5 short-scoreboard stall cycles per issue (ranking through shared-memory counters), 28 % of the issue slots; 83 % of each store's sectors useful",
-                     "profile": "profiles/k_sort_scatter_cfg4_8tables.md"},
+    # on the small case a pass of the sort is L2 resident, so its DRAM traffic does not scale to the full size: none given
+    "sort_scatter": {"dram_bytes_per_index": None, "bound": "latency",
+                     "evidence": "short scoreboard 6.1 (ranking through shared-memory counters), long scoreboard 5.6 (tile load, look-back) and barrier 2.6 stall cycles per issue; 35 % of the issue slots; DRAM 14 %, L2 24 % of peak",
+                     "profile": "profiles/k_sort_scatter_cfg4_9tables.md"},
     "broadcast": {"dram_bytes_per_index": 14.1, "bound": "l2",
                   "evidence": "64 % of the L2 throughput (4-byte scatters and gathers inside a table's window), 80 long-scoreboard and 13.6 lg_throttle stall cycles per issue",
                   "profile": "profiles/k_broadcast_cfg4_8tables.md"},
@@ -407,6 +407,7 @@ def run_ours(args, cfg, rank, world, local_rank):
         "per_step": {"indices": L, "distinct_rows": U, "distinct_hits": U_hit, "index_hit_rate": occ_hit / max(L, 1),
                      "admissions": adm, "evictions": evi, "hot_rows": hot_rows, "hot_row_indices": hot_occ},
         "kernels_ms_per_step": {k: v[0] / K for k, v in ranked},
+        "memory_bytes": {"workspace_and_staging": list(h.workspace_bytes())},
     }
     return result
 

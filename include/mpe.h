@@ -202,9 +202,9 @@ int mpe_step_host_wait(mpe_handle* h);
  * does.)
  *
  * Same inputs, outputs, layouts and result as mpe_forward -- the pooled FP32 sums of the bags, bit for bit
- * -- but every intermediate array of the step (sort keys and payloads, histograms, prefix sums, the
+ * -- but every intermediate array of the step (sort keys and payloads, digit counts, per-tile words, the
  * distinct-row list and its maps) lives in ONE fixed array compiled into the library
- * (`static __device__`, about 2.2 MB; every GPU that loads the library holds it until the process exits).
+ * (`static __device__`, about 2.5 MB; every GPU that loads the library holds it until the process exits).
  * Limits: total_indices <= MPE_STATIC_MAX_INDICES, num_tables * batch <= MPE_STATIC_MAX_BAGS,
  * num_tables <= MPE_STATIC_MAX_TABLES; a larger call returns MPE_ERR_TOO_LARGE and does nothing.
  * It calls no cudaMalloc / cudaFree and no allocating library routine.
