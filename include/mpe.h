@@ -114,6 +114,8 @@ int mpe_forward(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offset
  * The first call allocates the second workspace
  * (cudaMalloc; as large as the first, see mpe_workspace_bytes).
  * Typical loop:  forward(k); prepare(k+1, other_stream); backward(k); forward(k+1); ...
+ * It pays to give the training step's stream a higher priority than other_stream (cudaStreamCreateWithPriority):
+ * the step's kernels then get the SMs first and the preparation fills the gaps (measured: 1.6 % of the step).
  */
 int mpe_prepare(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offsets, int32_t batch, int64_t total_indices,
                 void* cuda_stream);
