@@ -193,7 +193,8 @@ class Oracle:
             self._h = None
 
     def __del__(self):
-        self.close()
+        if _destroy is not None:        # at interpreter exit the module's names may be gone already
+            self.close()
 
     def set_rounding(self, mode):
         _set_rounding(self._h, mode)
