@@ -290,7 +290,11 @@ int mpe_export_aux(mpe_handle* h, int32_t table, const int64_t* h_rows, int64_t 
  * the step is captured once into a CUDA graph (sized for the reserved workspace) and replayed; the per-call
  * arguments reach the kernels through device memory.  enable = 0 switches to plain launches (larger steps and
  * steps issued while profiling or while the caller captures the stream always use plain launches).  A backward
- * is replayed only if its forward was.  Not allowed between a forward and its backward (MPE_ERR_SEQUENCE). */
+ * is replayed only if its forward was.  Not allowed between a forward and its backward (MPE_ERR_SEQUENCE).
+ * A graph the CALLER captured around steps of this library may be replayed about 10^8 times in a row: the pass
+ * numbers in the sort's per-tile words (30 bits) are started over by mpe_forward's host code, which counts the calls
+ * it sees, not by the captured kernels.  For more replays, every 10^8 of them call
+ * mpe_selftest(h, MPE_SELFTEST_RENEW_TAGS) and then one mpe_forward / mpe_backward outside the graph. */
 int mpe_use_graphs(mpe_handle* h, int32_t enable);
 
 /* ---- instrumentation ---------------------------------------------------------------------------- */
