@@ -250,7 +250,7 @@ k_sort_digits(const uint32_t* __restrict__ keys, const int32_t* __restrict__ seg
     }
 }
 
-// ---- pass 3 of 3: stable scatter ------------------------------------------------
+// ---- one pass: stable scatter ---------------------------------------------------
 // Between passes an element travels as one 8-byte (key, payload) record, so a pass reads and writes it with one
 // instruction each and a digit's run of a tile is one contiguous piece of memory.
 // FIRST: the input is the bare key array and the payload is the element's position.
