@@ -46,3 +46,26 @@ def test_create_fails_loudly_without_a_gpu():
         assert e.code == binding.ERR_CUDA
     else:
         raise AssertionError("mpe_create must not succeed without a CUDA device")
+
+
+def test_error_codes_of_header_and_binding_agree():
+    from paper_2010_11305_b200 import binding
+    text = open(os.path.join(ROOT, "include", "mpe.h")).read()
+    codes = dict(re.findall(r"\b(MPE_(?:OK|ERR_[A-Z_]+))\s*=\s*(-?\d+)", text))
+    assert len(codes) >= 10
+    for name, value in codes.items():
+        short = name[len("MPE_"):]
+        assert getattr(binding, short) == int(value), name
+
+
+def test_bench_evidence_points_at_committed_summaries():
+    """Every kernel record of the benchmark names the ncu summary its `bound` comes from: the file must be there, and it
+    must be a text summary, nothing that runs."""
+    import sys
+    sys.path.insert(0, ROOT)
+    import bench
+    assert {"update", "pool", "hot_partial", "sort_scatter", "broadcast"} <= set(bench.KERNEL_EVIDENCE)
+    for name, ev in bench.KERNEL_EVIDENCE.items():
+        path = os.path.join(ROOT, ev["profile"])
+        assert os.path.isfile(path) and path.endswith(".md"), f"{name}: {ev['profile']}"
+        assert "--clock-control none" in open(path).read(), f"{name}: the summary does not give its command"
