@@ -657,17 +657,17 @@ int forward_impl(mpe_handle* h, const int32_t* d_indices, const int32_t* d_offse
     int rc = MPE_OK;
     if (may_use_graph(h)) {
         if (!h->x_fwd) {
-            rc = capture(h, &h->g_fwd, &h->x_fwd, &h->n_fwd, &h->k_fwd, (const void*)k_set_args_forward, [&]() {
-                LAUNCH(h, "set_args", k_set_args_forward, 1, 1, 0, w.args, d_indices, d_offsets, d_out, batch, L, h->epoch, route);
+            // the graph's first kernel, k_prelude, is the one whose parameters change from call to call
+            rc = capture(h, &h->g_fwd, &h->x_fwd, &h->n_fwd, &h->k_fwd, (const void*)k_prelude<true>, [&]() {
                 return enqueue_forward(h, h->cap_L, h->cap_bags, true);
             });
             if (rc != MPE_OK) { drop_graphs(h); h->graphs_enabled = false; }      // fall back to plain launches for good
         }
         if (rc == MPE_OK) {
-            StepArgs* a = w.args;
-            void* params[] = {&a, &d_indices, &d_offsets, &d_out, &batch, &L, &h->epoch, &route};
+            Work wv = w; int T = h->T; StepArgs av = h->args;
+            void* params[] = {&wv, &T, &av};
             cudaKernelNodeParams kp{};
-            kp.func = (void*)k_set_args_forward; kp.gridDim = dim3(1); kp.blockDim = dim3(1); kp.kernelParams = params;
+            kp.func = (void*)k_prelude<true>; kp.gridDim = dim3(1); kp.blockDim = dim3(32); kp.kernelParams = params;
             CK(h, cudaGraphExecKernelNodeSetParams(h->x_fwd, h->n_fwd, &kp));
             CK(h, cudaGraphLaunch(h->x_fwd, h->stream));
             h->launches += h->k_fwd;

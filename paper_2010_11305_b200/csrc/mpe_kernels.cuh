@@ -103,10 +103,6 @@ struct Work {
 // ---------------------------------------------------------------------------------------------
 // step prologue
 // ---------------------------------------------------------------------------------------------
-__global__ void k_set_args_forward(StepArgs* a, const int32_t* indices, const int32_t* offsets, float* out, int32_t B, uint32_t L,
-                                   uint32_t epoch, const Route* route) {
-    a->indices = indices; a->offsets = offsets; a->out = out; a->B = B; a->L = L; a->epoch = epoch; a->route = route;
-}
 __global__ void k_set_route(Route* dst, Route r) {
     for (int g = threadIdx.x; g < MAX_RANKS; g += blockDim.x) dst->out[g] = r.out[g];
     if (threadIdx.x == 0) { dst->B_local = r.B_local; dst->T_global = r.T_global; dst->t_base = r.t_base; dst->n_ranks = r.n_ranks; }
@@ -117,11 +113,17 @@ __global__ void k_set_args_backward(StepArgs* a, const float* grad, float lr, un
 
 // one warp: resets the step's counters and reads where each table's bags begin (the offsets of bags 0, B, 2B, ...), 32
 // tables at a time so that the loads overlap; offsets that do not start at 0, end at L or grow abandon the step
+// In a replayed step this is the graph's first kernel and the one whose parameters change from call to call: it passes the
+// forward's arguments on to the kernels behind it through the block in device memory.
 template <bool IND>
 __global__ void k_prelude(Work w, int T, StepArgs av) {
-    StepArgs a = av; if (IND) a = *w.args;      // replayed from a graph: the arguments come from device memory
+    const StepArgs a = av;
     if (blockIdx.x != 0 || threadIdx.x >= 32) return;
     const int lane = threadIdx.x;
+    if (IND && lane == 0) {
+        StepArgs* d = w.args;
+        d->indices = a.indices; d->offsets = a.offsets; d->out = a.out; d->B = a.B; d->L = a.L; d->epoch = a.epoch; d->route = a.route;
+    }
     const int32_t* __restrict__ offsets = a.offsets;
     const int B = a.B;
     const uint32_t L = a.L;
