@@ -310,18 +310,29 @@ def test_memory_accounting_matches_the_appendix_table():
 # Full-size configurations, in the launch configuration the benchmark times.  The oracle follows a
 # sample of the tables (tables are independent); everything observable of those tables is compared.
 # ---------------------------------------------------------------------------------------------
-def _full_size(cfg, tables, steps, check_at=()):
+def _full_size(cfg, tables, steps, check_at=(), prepare_ahead=False):
     """A configuration at its full size in the launch configuration the benchmark times; the oracle follows the
-    sampled tables only.  State is compared at the steps in check_at, at the last step, and again after a flush."""
+    sampled tables only.  State is compared at the steps in check_at, at the last step, and again after a flush.
+    prepare_ahead: as the benchmark does for steps too large to be replayed from a graph, the next batch is sorted and
+    de-duplicated on a second stream while the current step runs."""
     from parity_util import make_pair, compare_state
     h, o = make_pair(cfg, tables)
     st = wl.Stream(cfg, "cuda")
     rng = np.random.default_rng(0)
     cols = np.concatenate([np.arange(t * cfg.dim, (t + 1) * cfg.dim) for t in tables])
+    side = torch.cuda.Stream()
+    nxt = st.batch(1)
+    if prepare_ahead:
+        h.reserve(cfg.batch, int(nxt[0].numel() * 1.05))
     for step in range(1, steps + 1):
-        idx, off, grad = st.batch(step)
+        idx, off, grad = nxt
         out = torch.empty(cfg.batch, cfg.num_tables * cfg.dim, device="cuda")
         h.forward(idx, off, cfg.batch, out)
+        if step < steps:
+            nxt = st.batch(step + 1)
+            if prepare_ahead:
+                side.wait_stream(torch.cuda.current_stream())      # the next batch has been generated on the current stream
+                h.prepare(nxt[0], nxt[1], cfg.batch, side.cuda_stream)
         ref = o.forward(idx.cpu().numpy(), off.cpu().numpy(), cfg.batch)
         assert np.array_equal(out[:, torch.as_tensor(cols, device="cuda")].cpu().numpy(), ref[:, cols]), f"step {step}: pooled outputs"
         h.backward(grad, cfg.lr, step)
@@ -343,9 +354,10 @@ def test_full_size_config4_all_twenty_steps():
     assert cfg.steps == 20
     z = np.array(cfg.zipf)
     tables = sorted({int(z.argmax()), int(z.argmin()), 37})
-    h = _full_size(cfg, tables, cfg.steps, check_at=(3, 10))
+    h = _full_size(cfg, tables, cfg.steps, check_at=(3, 10), prepare_ahead=True)
     info = h.step_info()
     assert info[0] > 25_000_000 and info[3] > 500      # ~31M indices, thousands of hot rows
+    assert h.workspace_bytes()[0] > 4_000_000_000      # two workspaces: batches were prepared ahead
     s = h.stats(tables[0])
     assert s[4] > 0 and s[5] > 0 and s[6] > 0          # past the fill phase: admissions, evictions and bypasses all happen
     h.close()
